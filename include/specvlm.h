@@ -1,0 +1,188 @@
+/*
+ * specvlm.h -- C ABI of the B200 (sm_100a) hot path of SpecVLM's pruned-draft speculative
+ * decoding step (arXiv 2508.16201).
+ *
+ * One speculative step of the paper runs, in this order:
+ *   specvlm_stage1_scores   token rating A from the verifier's language-to-video attention
+ *   specvlm_select          Stage I retention (top-k of A) + Stage II spatially uniform reduction
+ *   specvlm_gather_kv       compaction of the surviving video tokens' K/V into the draft cache
+ *   specvlm_draft_decode_attn   (gamma times) draft decode attention over the pruned cache
+ *   specvlm_verify_attn     (gamma+1)-query causal verification attention over the full cache
+ *   specvlm_accept          greedy acceptance length and next token
+ *
+ * Conventions (all entry points)
+ *   - Return value: SPECVLM_OK (0) or a negative specvlm_status code.  Argument errors are
+ *     detected on the host and nothing is launched.
+ *   - Pointers marked "device" are device memory owned by the caller; pointers marked "host"
+ *     are ordinary host memory read during the call.  Unless an entry point says otherwise the
+ *     library allocates nothing and keeps no state between calls.
+ *   - Work is enqueued on the CUDA stream passed as `stream` (a cudaStream_t cast to void*;
+ *     NULL = the legacy default stream).  No call synchronises the host with the device.
+ *   - `d_status` (device int32_t*, optional): a kernel that gives up a bounded wait stores
+ *     SPECVLM_ERR_TIMEOUT there and returns; it is never written otherwise.
+ *   - Scratch memory comes from the caller: `ws` (device, 256-byte aligned) of at least the
+ *     size the matching *_workspace_bytes query returns.  Its contents need not be initialised
+ *     and are unspecified afterwards.  Calls that share a workspace must not overlap on the GPU.
+ *   - bf16 = 2-byte bfloat16.  "Token row" = head_dim consecutive bf16 values.
+ */
+#ifndef SPECVLM_H_
+#define SPECVLM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum specvlm_status {
+  SPECVLM_OK = 0,
+  SPECVLM_ERR_INVALID_ARG = -1,       /* null pointer, negative size, inconsistent arguments   */
+  SPECVLM_ERR_UNSUPPORTED_SHAPE = -2, /* a shape outside the documented supported set          */
+  SPECVLM_ERR_WORKSPACE_TOO_SMALL = -3,
+  SPECVLM_ERR_CUDA = -4,              /* a CUDA runtime / driver call failed                   */
+  SPECVLM_ERR_TIMEOUT = -5            /* device-side bounded wait expired (via d_status only)  */
+} specvlm_status;
+
+/*
+ * A K/V cache, contiguous or paged (the caches of Section 3.1 of the paper: the draft's pruned
+ * cache and the target's full cache).  Token p of sequence b lives in logical block
+ * p / block_tokens at offset p % block_tokens; the physical block is block_table[b][logical]
+ * when block_table is non-NULL, else block b itself (then block_tokens >= max_seq_len, i.e. one
+ * block per sequence = a contiguous cache).  The element (layer l, physical block n, KV head g,
+ * offset t, channel c) is at
+ *     k[l*stride_layer + n*stride_block + g*stride_head + t*stride_token + c]      (bf16 units).
+ * Requirements: head_dim in {64, 128}; every stride a multiple of 8 elements (16 bytes);
+ * k and v 16-byte aligned; with a block table, block_tokens a multiple of 64.
+ * The struct itself is host memory; k, v, block_table, seq_lens are device pointers.
+ */
+typedef struct specvlm_kv {
+  void* k;
+  void* v;
+  int64_t stride_layer, stride_block, stride_head, stride_token;
+  int32_t n_layers, n_kv_heads, head_dim;
+  int32_t block_tokens;         /* tokens per block                                          */
+  int32_t n_blocks;             /* blocks in the pool (paged) / sequences (contiguous)       */
+  int32_t max_blocks;           /* row length of block_table                                 */
+  const int32_t* block_table;   /* device [batch][max_blocks] or NULL                        */
+  const int32_t* seq_lens;      /* device [batch]: valid tokens per sequence                 */
+  int32_t max_seq_len;          /* host-side upper bound on seq_lens (sizes the launch)      */
+} specvlm_kv_t;
+
+const char* specvlm_version(void);
+const char* specvlm_status_string(int32_t status);
+
+/* ---------------------------------------------------------------------------------------------
+ * Step 1a -- token rating (Section 4.1, Eq. 4-5).
+ * For every verifier layer l, query head h and language query i, the full causal softmax row
+ * over the keys 0..p_i (p_i = absolute position of query i) is formed with logits
+ * sm_scale * <q, K>; G_{i,j} is its value at video token j (Eq. 4); the score of video token j is
+ * the mean of G_{i,j} over the language queries (Eq. 5) and over all layers and query heads.
+ *
+ *   target_kv   host struct; K of the verifier (V is not read).  All layers are used.
+ *   q_text      device bf16 [n_layers][sum_text][n_q_heads][head_dim], language queries of all
+ *               sequences concatenated (sequence b owns rows text_cu[b] .. text_cu[b+1]-1)
+ *   text_cu     host int32 [batch+1]
+ *   text_start  host int32 [batch]: absolute position of sequence b's first language query; its
+ *               i-th query is at text_start[b]+i and sees keys 0 .. text_start[b]+i
+ *   video_start, video_len   host int32 [batch]; video_start+video_len <= text_start
+ *   video_cu    host int32 [batch+1]: offsets of each sequence's scores in `scores`
+ *   scores      device fp32 [video_cu[batch]] out
+ *   ws          device scratch, specvlm_stage1_scores_workspace_bytes(...)
+ * Deterministic: the reduction order over rows, heads and layers is fixed.
+ * Supported: head_dim 128 or 64, n_q_heads / n_kv_heads in 1..16.
+ */
+size_t specvlm_stage1_scores_workspace_bytes(const specvlm_kv_t* target_kv, const int32_t* text_cu,
+                                             const int32_t* video_len, int32_t batch,
+                                             int32_t n_q_heads);
+int32_t specvlm_stage1_scores(const specvlm_kv_t* target_kv, const void* q_text,
+                              const int32_t* text_cu, const int32_t* text_start,
+                              const int32_t* video_start, const int32_t* video_len,
+                              const int32_t* video_cu, int32_t batch, int32_t n_q_heads,
+                              float sm_scale, float* scores, void* ws, size_t ws_bytes,
+                              int32_t* d_status, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Steps 1b + 2 -- two-stage selection (Section 4.2).
+ * Stage I keeps the k_stage1[b] highest-scored video tokens V_R (ranking "sort A, add in order"
+ * of the paragraph before Eq. 6; order key: score descending, index ascending, compared on the
+ * fp32 bit patterns; scores must be finite and >= 0).  Stage II keeps, from V \ V_R, tokens at a
+ * fixed interval (Eq. 7) with budget n_U = k_total[b] - k_stage1[b] so that the final set has
+ * exactly k_total[b] tokens: frame f's remaining tokens (raster order, c_f of them, C_f before
+ * it, m in total) get the quota floor(C_{f+1} n_U / m) - floor(C_f n_U / m) and the picks are
+ * the remaining tokens of rank floor(t c_f / n_f), t = 0..n_f-1.
+ *
+ *   scores      device fp32, sequence b at video_cu[b] .. ; length n_frames[b]*tokens_per_frame
+ *   video_cu, n_frames, k_stage1, k_total, kept_cu    host int32 arrays ([batch+1] for *_cu)
+ *   kept_idx    device int32 out: sequence b's kept video indices (sequence-local, ascending) at
+ *               kept_cu[b] .. kept_cu[b]+k_total[b]-1
+ * Requires 0 <= k_stage1 <= k_total <= n_video <= 57344 per sequence, n_frames <= 1024.
+ * Uses no scratch memory.
+ */
+int32_t specvlm_select(const float* scores, const int32_t* video_cu, const int32_t* n_frames,
+                       int32_t tokens_per_frame, const int32_t* k_stage1, const int32_t* k_total,
+                       const int32_t* kept_cu, int32_t batch, int32_t* kept_idx, int32_t* d_status,
+                       void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Step 3 -- pruned draft context (end of Section 4.2: the draft sees V_R u V_U and the language
+ * prompt, its cache reduced to 1-r of the original).
+ * For every layer and KV head, copies the token rows
+ *   [0, video_start)  ++  video_start + kept_idx[...]  ++  [video_start+video_len, src seq_len)
+ * of sequence b from `src` to positions 0,1,2,... of sequence b in `dst`, K and V alike, bit for
+ * bit.  The caller sets dst->seq_lens (= src length - video_len + kept count) itself.
+ *   src, dst    host structs with the same n_layers, n_kv_heads, head_dim; either may be paged
+ *   kept_idx    device int32 (as written by specvlm_select); kept_cu, video_start, video_len,
+ *               src_len host int32 ([batch+1] / [batch]); src_len[b] = tokens of sequence b in src
+ */
+int32_t specvlm_gather_kv(const specvlm_kv_t* src, const int32_t* kept_idx, const int32_t* kept_cu,
+                          const int32_t* video_start, const int32_t* video_len,
+                          const int32_t* src_len, int32_t batch, const specvlm_kv_t* dst,
+                          int32_t* d_status, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Steps 4a / 4b -- attention (Section 3.1: each draft step streams the draft's whole KV cache;
+ * the target verifies the gamma drafted tokens in one memory-bound pass).
+ *   o[l][b][t][h] = softmax_k( sm_scale * <q[l][b][t][h], K[l][b][g(h)][k]> ) V[l][b][g(h)][k]
+ * with g(h) = h / (n_q_heads / n_kv_heads).  The cache already contains the K/V of the n_q new
+ * tokens at its end (kv->seq_lens counts them); query t sees keys 0 .. seq_len - n_q + t.
+ * specvlm_draft_decode_attn is the n_q = 1 case, specvlm_verify_attn has n_q = gamma + 1.
+ *
+ *   q, out      device bf16 [n_layers][batch][n_q][n_q_heads][head_dim]
+ *   lse_or_null device fp32 [n_layers][batch][n_q][n_q_heads]: natural-log sum-exp of the logits
+ *   ws          device scratch, specvlm_attn_workspace_bytes(kv, batch, n_q_heads, gamma)
+ * fp32 softmax and accumulation; probabilities are rounded to bf16 before the PV product.
+ * Supported: head_dim 64/128; group = n_q_heads/n_kv_heads in 1..16; 0 <= gamma <= 8;
+ * group * (gamma+1) <= 96.
+ */
+size_t specvlm_attn_workspace_bytes(const specvlm_kv_t* kv, int32_t batch, int32_t n_q_heads,
+                                    int32_t gamma);
+int32_t specvlm_draft_decode_attn(const specvlm_kv_t* kv, const void* q, int32_t batch,
+                                  int32_t n_q_heads, float sm_scale, void* out, float* lse_or_null,
+                                  void* ws, size_t ws_bytes, int32_t* d_status, void* stream);
+int32_t specvlm_verify_attn(const specvlm_kv_t* kv, const void* q, int32_t batch,
+                            int32_t n_q_heads, int32_t gamma, float sm_scale, void* out,
+                            float* lse_or_null, void* ws, size_t ws_bytes, int32_t* d_status,
+                            void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Step 4c -- greedy acceptance (Section 3.1 and the experimental set-up: the target decodes
+ * greedily and speculative decoding is lossless).
+ *   g[b][t] = argmax_v target_logits[b][t][v]   (lowest index among equal maxima)
+ *   accept_len[b] = number of leading positions t < gamma with draft_tokens[b][t] == g[b][t]
+ *   next_token[b] = g[b][accept_len[b]]
+ *   target_logits  device fp32 [batch][gamma+1][vocab] (finite values)
+ *   draft_tokens   device int32 [batch][gamma]
+ *   accept_len, next_token   device int32 [batch] out
+ *   target_argmax_or_null    device int32 [batch][gamma+1] out (optional)
+ *   ws             device scratch, specvlm_accept_workspace_bytes(batch, gamma, vocab)
+ */
+size_t specvlm_accept_workspace_bytes(int32_t batch, int32_t gamma, int32_t vocab);
+int32_t specvlm_accept(const float* target_logits, const int32_t* draft_tokens, int32_t batch,
+                       int32_t gamma, int32_t vocab, int32_t* accept_len, int32_t* next_token,
+                       int32_t* target_argmax_or_null, void* ws, size_t ws_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECVLM_H_ */

@@ -1,0 +1,131 @@
+// Step 4c: greedy acceptance.  Kernel 1 streams the fp32 logits once (16-byte loads) and leaves
+// one (max, lowest index) candidate per (row, vocab chunk); kernel 2 finishes the argmax of the
+// gamma+1 rows of a sequence and counts the leading draft tokens that equal it.
+#include "common.cuh"
+#include "host_util.h"
+
+namespace specvlm {
+
+constexpr int kAcceptChunk = 4096;     // logits per CTA in kernel 1
+constexpr int kAcceptThreads = 256;
+
+struct Cand {
+  float v;
+  int32_t i;
+};
+
+// a is replaced by b when b is larger, or equal with a lower index
+__device__ __forceinline__ void take_better(float& av, int& ai, float bv, int bi) {
+  if (bv > av || (bv == av && bi < ai)) {
+    av = bv;
+    ai = bi;
+  }
+}
+
+__global__ void __launch_bounds__(kAcceptThreads)
+accept_partial_kernel(const float* __restrict__ logits, int vocab, int n_chunks, Cand* __restrict__ part) {
+  const int row = blockIdx.y, chunk = blockIdx.x;
+  const float* base = logits + (size_t)row * vocab;
+  const int lo = chunk * kAcceptChunk;
+  const int hi = lo + kAcceptChunk < vocab ? lo + kAcceptChunk : vocab;
+  float bv = -INFINITY;
+  int bi = 0x7fffffff;
+  if (((reinterpret_cast<uintptr_t>(base + lo)) & 15u) == 0) {
+    const int n4 = (hi - lo) >> 2;
+    const float4* b4 = reinterpret_cast<const float4*>(base + lo);
+    for (int k = threadIdx.x; k < n4; k += kAcceptThreads) {
+      const float4 x = __ldcs(b4 + k);
+      const int i0 = lo + 4 * k;
+      // ascending index with strict '>' keeps the lowest index among equals
+      if (x.x > bv) { bv = x.x; bi = i0; }
+      if (x.y > bv) { bv = x.y; bi = i0 + 1; }
+      if (x.z > bv) { bv = x.z; bi = i0 + 2; }
+      if (x.w > bv) { bv = x.w; bi = i0 + 3; }
+    }
+    for (int i = lo + 4 * n4 + threadIdx.x; i < hi; i += kAcceptThreads) take_better(bv, bi, base[i], i);
+  } else {
+    for (int i = lo + threadIdx.x; i < hi; i += kAcceptThreads) take_better(bv, bi, base[i], i);
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+    const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+    take_better(bv, bi, ov, oi);
+  }
+  __shared__ float sv[kAcceptThreads / 32];
+  __shared__ int si[kAcceptThreads / 32];
+  if ((threadIdx.x & 31) == 0) {
+    sv[threadIdx.x >> 5] = bv;
+    si[threadIdx.x >> 5] = bi;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < kAcceptThreads / 32; ++w) take_better(bv, bi, sv[w], si[w]);
+    part[(size_t)row * n_chunks + chunk] = Cand{bv, bi};
+  }
+}
+
+// one warp per (sequence, t); one CTA of (gamma+1) warps per sequence
+__global__ void accept_finish_kernel(const Cand* __restrict__ part, int n_chunks,
+                                     const int32_t* __restrict__ draft, int gamma,
+                                     int32_t* __restrict__ accept_len, int32_t* __restrict__ next_token,
+                                     int32_t* __restrict__ g_out) {
+  __shared__ int g_sm[16];
+  const int b = blockIdx.x, t = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const Cand* row = part + ((size_t)b * (gamma + 1) + t) * n_chunks;
+  float bv = -INFINITY;
+  int bi = 0x7fffffff;
+  for (int c = lane; c < n_chunks; c += 32) take_better(bv, bi, row[c].v, row[c].i);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+    const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+    take_better(bv, bi, ov, oi);
+  }
+  if (lane == 0) {
+    g_sm[t] = bi;
+    if (g_out) g_out[(size_t)b * (gamma + 1) + t] = bi;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int n = 0;
+    while (n < gamma && draft[(size_t)b * gamma + n] == g_sm[n]) ++n;
+    accept_len[b] = n;
+    next_token[b] = g_sm[n];
+  }
+}
+
+}  // namespace specvlm
+
+using namespace specvlm;
+
+extern "C" size_t specvlm_accept_workspace_bytes(int32_t batch, int32_t gamma, int32_t vocab) {
+  if (batch < 1 || gamma < 0 || vocab < 1) return 0;
+  const size_t n_chunks = ((size_t)vocab + kAcceptChunk - 1) / kAcceptChunk;
+  return round_up((size_t)batch * (gamma + 1) * n_chunks * sizeof(Cand), 256);
+}
+
+extern "C" int32_t specvlm_accept(const float* target_logits, const int32_t* draft_tokens,
+                                  int32_t batch, int32_t gamma, int32_t vocab, int32_t* accept_len,
+                                  int32_t* next_token, int32_t* target_argmax_or_null, void* ws,
+                                  size_t ws_bytes, void* stream) {
+  if (!target_logits || !accept_len || !next_token || batch < 1 || gamma < 0 || vocab < 1 || !ws)
+    return SPECVLM_ERR_INVALID_ARG;
+  if (gamma > 0 && !draft_tokens) return SPECVLM_ERR_INVALID_ARG;
+  if (gamma > 15) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  if ((int64_t)batch * (gamma + 1) > 65535) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(target_logits) & 3u) || (reinterpret_cast<uintptr_t>(ws) & 7u))
+    return SPECVLM_ERR_INVALID_ARG;
+  if (ws_bytes < specvlm_accept_workspace_bytes(batch, gamma, vocab)) return SPECVLM_ERR_WORKSPACE_TOO_SMALL;
+  const int n_chunks = (vocab + kAcceptChunk - 1) / kAcceptChunk;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  Cand* part = static_cast<Cand*>(ws);
+  accept_partial_kernel<<<dim3((unsigned)n_chunks, (unsigned)(batch * (gamma + 1))), kAcceptThreads, 0, st>>>(
+      target_logits, vocab, n_chunks, part);
+  int32_t rc = launch_status();
+  if (rc != SPECVLM_OK) return rc;
+  accept_finish_kernel<<<(unsigned)batch, 32 * (gamma + 1), 0, st>>>(part, n_chunks, draft_tokens, gamma,
+                                                                     accept_len, next_token,
+                                                                     target_argmax_or_null);
+  return launch_status();
+}

@@ -1,0 +1,616 @@
+// Step 1a: token rating from the verifier's language-to-video attention.
+//
+// The rating of video token j is the mean, over layers, query heads and language queries, of the
+// causal softmax probability the query puts on j.  This is a dense contraction (every language
+// query row against every key), so it runs on the tensor cores, in two passes over QK^T:
+//   pass 1 (row-centric)   the log-sum-exp of every language query row over all its causal keys;
+//   pass 2 (column-centric) P = 2^(s - lse) recomputed tile by tile and summed down the rows.
+// The full attention matrix is never stored.  All reductions run in a fixed order: per-layer
+// partial column sums, then one ordered sum over layers.
+//
+// Rows of a (layer, KV head) problem are the language queries times the group's heads, in the
+// order r = i * group + head_in_group; a row tile holds QT = floor(128 / group) queries.
+#include "common.cuh"
+#include "host_util.h"
+
+namespace specvlm {
+
+constexpr int kScoresMaxBatch = 64;
+constexpr int kKeyTile = 128;          // keys per CTA tile (two cache pages)
+
+struct ScoreSeq {
+  int32_t text_off, n_text, text_start, video_start, n_video, score_off;
+  int32_t tile_off;                    // first CTA index (pass 1: row tiles, pass 2: key blocks)
+};
+
+struct ScoreParams {
+  const __nv_bfloat16* q;              // [L][sum_text][Hq][D]
+  float* lse2;                         // [L][Hkv][sum_text * group]  (log2 units, of scaled logits)
+  float* partial;                      // [L][sum_video]
+  const int32_t* block_table;
+  int32_t* d_status;
+  int32_t batch, n_layers, n_q_heads, n_kv_heads, group, qt, sum_text, sum_video;
+  int32_t max_blocks, block_tokens;
+  float scale_log2;
+  ScoreSeq seq[kScoresMaxBatch];
+};
+
+__device__ __forceinline__ int find_seq(const ScoreParams& p, int cta) {
+  int b = 0;
+  while (b + 1 < p.batch && p.seq[b + 1].tile_off <= cta) ++b;
+  return b;
+}
+
+// issue the TMA loads of one 128-key K tile (two 64-token pages, D/64 channel halves each)
+template <int D>
+__device__ __forceinline__ void load_key_tile(const CUtensorMap* tm_k, const ScoreParams& p, int b,
+                                              int g, int layer, int key0, uint32_t dst, uint32_t bar,
+                                              uint64_t policy) {
+#pragma unroll
+  for (int pg = 0; pg < 2; ++pg) {
+    const int tok0 = key0 + pg * 64;
+    int blk = b, tok = tok0;
+    if (p.block_table) {
+      const int lblk = tok0 / p.block_tokens;
+      // past the sequence's last page: an out-of-range block coordinate reads zeros
+      blk = lblk < p.max_blocks ? p.block_table[(size_t)b * p.max_blocks + lblk] : -1;
+      tok = tok0 % p.block_tokens;
+    }
+#pragma unroll
+    for (int h = 0; h < D / 64; ++h)
+      tma_load_5d(dst + h * (kKeyTile * 128) + pg * (64 * 128), tm_k, bar, h * 64, tok, g, blk, layer,
+                  policy);
+  }
+}
+// byte offset of (row r of a 128-row tile, 16-byte chunk c16); halves of 64 channels are 16 KB apart
+template <int D>
+__device__ __forceinline__ uint32_t tile128_offset(int r, int c16) {
+  return static_cast<uint32_t>((c16 >> 3) * (kKeyTile * 128) + r * 128 + (((c16 & 7) ^ (r & 7)) << 4));
+}
+
+// ---------------------------------------------------------------------------------------------
+// Pass 1.  CTA = (row tile, KV head, layer).  8 compute warps = 4 (32 rows each) x 2 (64 of the
+// tile's 128 keys each); warp 8 streams K tiles.  Q fragments stay in registers.
+// ---------------------------------------------------------------------------------------------
+template <int D, int STAGES>
+__global__ void __launch_bounds__(288, 1)
+scores_lse_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ ScoreParams p) {
+  constexpr int TILE_BYTES = kKeyTile * D * 2;
+  constexpr int KSTEPS = D / 16;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t base = (raw_addr + 1023u) & ~1023u;
+  uint8_t* const smem = smem_raw + (base - raw_addr);
+  const uint32_t bar_full = base + STAGES * TILE_BYTES;
+  const uint32_t bar_empty = bar_full + 8 * STAGES;
+  volatile int* const abort_flag =
+      reinterpret_cast<volatile int*>(smem + STAGES * TILE_BYTES + 16 * STAGES);
+  float* const red = reinterpret_cast<float*>(smem + STAGES * TILE_BYTES + 16 * STAGES + 16);  // [2][128][2]
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int b = find_seq(p, blockIdx.x);
+  const ScoreSeq sq = p.seq[b];
+  const int qtile = blockIdx.x - sq.tile_off;
+  const int g = blockIdx.y, layer = blockIdx.z;
+  const int i_first = qtile * p.qt;
+  const int n_i = min(p.qt, sq.n_text - i_first);               // queries in this tile
+  const int rows_valid = n_i * p.group;
+  const int key_end = sq.text_start + i_first + n_i;            // keys [0, key_end) are needed
+  const int n_kt = (key_end + kKeyTile - 1) / kKeyTile;
+
+  if (tid == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 8);
+    }
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  __syncthreads();
+
+  if (warp == 8) {
+    if (lane == 0) {
+      tma_prefetch_desc(&tm_k);
+      const uint64_t policy = l2_policy_evict_last();           // K is re-read by the other row tiles
+      int issued = 0;
+      bool ok = true;
+      for (int i = 0; i < n_kt; ++i) {
+        const int s = i % STAGES;
+        if (i >= STAGES) ok = mbar_wait(bar_empty + 8 * s, ((i / STAGES) - 1) & 1, abort_flag);
+        if (!ok) break;
+        mbar_arrive_expect_tx(bar_full + 8 * s, TILE_BYTES);
+        load_key_tile<D>(&tm_k, p, b, g, layer, i * kKeyTile, base + s * TILE_BYTES, bar_full + 8 * s,
+                         policy);
+        issued = i + 1;
+      }
+      if (!ok) {
+        if (p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
+        for (int i = issued > STAGES ? issued - STAGES : 0; i < issued; ++i) {
+          const uint64_t t0 = global_timer_ns();
+          while (!mbar_try_wait(bar_full + 8 * (i % STAGES), (i / STAGES) & 1) &&
+                 global_timer_ns() - t0 < kWaitLimitNs) {
+          }
+        }
+      }
+    }
+    return;
+  }
+
+  const int wm = warp >> 1, wn = warp & 1;        // 4 row groups x 2 key halves
+  const int col = (lane & 3) * 2;
+  // the four rows this thread holds: mt*16 + (lane>>2) + {0, 8}
+  uint32_t qf[2][KSTEPS][4];
+  int lim[2][2];
+#pragma unroll
+  for (int mt = 0; mt < 2; ++mt) {
+#pragma unroll
+    for (int hf = 0; hf < 2; ++hf) {
+      const int r = wm * 32 + mt * 16 + (lane >> 2) + hf * 8;
+      const __nv_bfloat16* qp = nullptr;
+      lim[mt][hf] = 0;
+      if (r < rows_valid) {
+        const int il = r / p.group, hg = r - il * p.group;
+        qp = p.q + (((size_t)layer * p.sum_text + sq.text_off + i_first + il) * p.n_q_heads +
+                    g * p.group + hg) * D;
+        lim[mt][hf] = sq.text_start + i_first + il + 1;
+      }
+#pragma unroll
+      for (int ks = 0; ks < KSTEPS; ++ks) {
+        qf[mt][ks][hf] = qp ? *reinterpret_cast<const uint32_t*>(qp + ks * 16 + col) : 0u;
+        qf[mt][ks][2 + hf] = qp ? *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8 + col) : 0u;
+      }
+    }
+  }
+  float m[2][2], l[2][2];
+#pragma unroll
+  for (int mt = 0; mt < 2; ++mt) m[mt][0] = m[mt][1] = -INFINITY, l[mt][0] = l[mt][1] = 0.f;
+
+  const int mi = lane >> 3, r8 = lane & 7;
+  bool alive = true;
+  for (int i = 0; i < n_kt; ++i) {
+    const int s = i % STAGES;
+    if (!mbar_wait(bar_full + 8 * s, (i / STAGES) & 1, abort_flag)) {
+      alive = false;
+      break;
+    }
+    const uint32_t k_base = base + s * TILE_BYTES;
+    const int key0 = i * kKeyTile + wn * 64;
+    if (key0 < key_end) {
+      float sc[2][8][4];
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) sc[mt][nt][0] = sc[mt][nt][1] = sc[mt][nt][2] = sc[mt][nt][3] = 0.f;
+#pragma unroll
+      for (int ks = 0; ks < KSTEPS; ++ks) {
+#pragma unroll
+        for (int np = 0; np < 4; ++np) {       // 16 keys per ldmatrix.x4
+          uint32_t b0, b1, b2, b3;
+          const int kr = wn * 64 + np * 16 + (mi >> 1) * 8 + r8;
+          ldmatrix_x4(k_base + tile128_offset<D>(kr, 2 * ks + (mi & 1)), b0, b1, b2, b3);
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt) {
+            mma_bf16_16816(sc[mt][2 * np], qf[mt][ks], b0, b1);
+            mma_bf16_16816(sc[mt][2 * np + 1], qf[mt][ks], b2, b3);
+          }
+        }
+      }
+      const bool need_mask = key0 + 64 > sq.text_start + i_first + 1;   // tile reaches past the first limit
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          float mx = -INFINITY;
+#pragma unroll
+          for (int nt = 0; nt < 8; ++nt) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              float v = sc[mt][nt][hf * 2 + e] * p.scale_log2;
+              if (need_mask && key0 + nt * 8 + col + e >= lim[mt][hf]) v = -INFINITY;
+              sc[mt][nt][hf * 2 + e] = v;
+              mx = fmaxf(mx, v);
+            }
+          }
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+          const float mn = fmaxf(m[mt][hf], mx);
+          const float mu = mn == -INFINITY ? 0.f : mn;
+          float ps = 0.f;
+#pragma unroll
+          for (int nt = 0; nt < 8; ++nt) ps += fast_exp2(sc[mt][nt][hf * 2] - mu) + fast_exp2(sc[mt][nt][hf * 2 + 1] - mu);
+          l[mt][hf] = l[mt][hf] * fast_exp2(m[mt][hf] - mu) + ps;
+          m[mt][hf] = mn;
+        }
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+  }
+  // combine the quad's partial sums, then the two key halves
+#pragma unroll
+  for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+    for (int hf = 0; hf < 2; ++hf) {
+      l[mt][hf] += __shfl_xor_sync(0xffffffffu, l[mt][hf], 1);
+      l[mt][hf] += __shfl_xor_sync(0xffffffffu, l[mt][hf], 2);
+    }
+  if ((lane & 3) == 0) {
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        const int r = wm * 32 + mt * 16 + (lane >> 2) + hf * 8;
+        red[(wn * 128 + r) * 2] = m[mt][hf];
+        red[(wn * 128 + r) * 2 + 1] = l[mt][hf];
+      }
+  }
+  asm volatile("bar.sync 1, 256;" ::: "memory");
+  if (!alive || *abort_flag) {
+    if (tid == 0 && p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
+    return;
+  }
+  if (tid < rows_valid) {
+    const float ma = red[tid * 2], la = red[tid * 2 + 1];
+    const float mb = red[(128 + tid) * 2], lb2 = red[(128 + tid) * 2 + 1];
+    const float M = fmaxf(ma, mb);
+    const float L = la * fast_exp2(ma - M) + lb2 * fast_exp2(mb - M);
+    p.lse2[((size_t)layer * p.n_kv_heads + g) * ((size_t)p.sum_text * p.group) +
+           (size_t)(sq.text_off + i_first) * p.group + tid] = M + log2f(L);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Pass 2.  CTA = (block of 128 video keys, layer); it loops over the layer's KV heads and, for
+// each, over all row tiles of the sequence.  8 compute warps = 2 (64 rows each) x 4 (32 keys
+// each); a warp keeps its K fragments in registers for the whole head and its 8 column sums in
+// registers for the whole layer.  Warp 8 streams the K block of each head and the Q row tiles.
+// ---------------------------------------------------------------------------------------------
+template <int D, int STAGES>
+__global__ void __launch_bounds__(288, 1)
+scores_colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
+                     const __grid_constant__ ScoreParams p) {
+  constexpr int TILE_BYTES = kKeyTile * D * 2;     // K block and Q tile alike (128 rows)
+  constexpr int KSTEPS = D / 16;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t base = (raw_addr + 1023u) & ~1023u;
+  uint8_t* const smem = smem_raw + (base - raw_addr);
+  const uint32_t k_sm = base;                                    // K block
+  const uint32_t q_sm = base + TILE_BYTES;                       // Q ring
+  const uint32_t bar_qfull = base + (STAGES + 1) * TILE_BYTES;
+  const uint32_t bar_qempty = bar_qfull + 8 * STAGES;
+  const uint32_t bar_kfull = bar_qempty + 8 * STAGES;
+  const uint32_t bar_kempty = bar_kfull + 8;
+  uint8_t* const tail = smem + (STAGES + 1) * TILE_BYTES + 16 * STAGES + 16;
+  volatile int* const abort_flag = reinterpret_cast<volatile int*>(tail);
+  float* const red = reinterpret_cast<float*>(tail + 16);        // [128] column sums of row half 1
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int b = find_seq(p, blockIdx.x);
+  const ScoreSeq sq = p.seq[b];
+  const int kblock = blockIdx.x - sq.tile_off;
+  const int layer = blockIdx.y;
+  const int key0 = sq.video_start + kblock * kKeyTile;           // absolute position of column 0
+  const int n_cols = min(kKeyTile, sq.n_video - kblock * kKeyTile);
+  const int n_qt = (sq.n_text + p.qt - 1) / p.qt;
+  const int n_units = p.n_kv_heads;
+
+  if (tid == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(bar_qfull + 8 * s, 1);
+      mbar_init(bar_qempty + 8 * s, 8);
+    }
+    mbar_init(bar_kfull, 1);
+    mbar_init(bar_kempty, 8);
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  __syncthreads();
+
+  if (warp == 8) {
+    if (lane == 0) {
+      tma_prefetch_desc(&tm_k);
+      tma_prefetch_desc(&tm_q);
+      const uint64_t pol_k = l2_policy_evict_first();
+      const uint64_t pol_q = l2_policy_evict_last();             // Q is re-read by every key block
+      bool ok = true;
+      int qi = 0;                                                 // running Q-tile counter
+      for (int u = 0; u < n_units && ok; ++u) {
+        if (u > 0) ok = mbar_wait(bar_kempty, (u - 1) & 1, abort_flag);
+        if (!ok) break;
+        mbar_arrive_expect_tx(bar_kfull, TILE_BYTES);
+        load_key_tile<D>(&tm_k, p, b, u, layer, key0, k_sm, bar_kfull, pol_k);
+        for (int t = 0; t < n_qt && ok; ++t, ++qi) {
+          const int s = qi % STAGES;
+          if (qi >= STAGES) ok = mbar_wait(bar_qempty + 8 * s, ((qi / STAGES) - 1) & 1, abort_flag);
+          if (!ok) break;
+          // box = (64 channels, group heads, 1 KV head, QT queries, 1 layer); rows land in the
+          // order r = query * group + head.  When group does not divide 128 the box has fewer
+          // than 128 rows; the barrier expects exactly the box bytes.
+          mbar_arrive_expect_tx(bar_qfull + 8 * s, (D / 64) * p.qt * p.group * 128);
+#pragma unroll
+          for (int h = 0; h < D / 64; ++h)
+            tma_load_5d(q_sm + s * TILE_BYTES + h * (kKeyTile * 128), &tm_q, bar_qfull + 8 * s, h * 64, 0,
+                        u, sq.text_off + t * p.qt, layer, pol_q);
+        }
+      }
+      if (!ok) {
+        // a wait expired: report, then stay until the copies already issued have landed
+        if (p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
+        const uint64_t t0 = global_timer_ns();
+        for (int i = qi > STAGES ? qi - STAGES : 0; i < qi; ++i)
+          while (!mbar_try_wait(bar_qfull + 8 * (i % STAGES), (i / STAGES) & 1) &&
+                 global_timer_ns() - t0 < kWaitLimitNs) {
+          }
+      }
+    }
+    return;
+  }
+
+  const int wm = warp >> 2, wn = warp & 3;          // 2 row halves x 4 key quarters
+  const int col = (lane & 3) * 2;
+  const int mi = lane >> 3, r8 = lane & 7;
+  float colsum[4][2];
+#pragma unroll
+  for (int nt = 0; nt < 4; ++nt) colsum[nt][0] = colsum[nt][1] = 0.f;
+
+  bool alive = true;
+  int qi = 0;
+  for (int u = 0; u < n_units && alive; ++u) {
+    if (!mbar_wait(bar_kfull, u & 1, abort_flag)) {
+      alive = false;
+      break;
+    }
+    uint32_t kf[KSTEPS][4][2];                      // B fragments: 4 n-tiles of 8 keys
+#pragma unroll
+    for (int ks = 0; ks < KSTEPS; ++ks) {
+#pragma unroll
+      for (int np = 0; np < 2; ++np) {
+        const int kr = wn * 32 + np * 16 + (mi >> 1) * 8 + r8;
+        ldmatrix_x4(k_sm + tile128_offset<D>(kr, 2 * ks + (mi & 1)), kf[ks][2 * np][0], kf[ks][2 * np][1],
+                    kf[ks][2 * np + 1][0], kf[ks][2 * np + 1][1]);
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar_kempty);
+    const float* lse_u = p.lse2 + ((size_t)layer * p.n_kv_heads + u) * ((size_t)p.sum_text * p.group) +
+                         (size_t)sq.text_off * p.group;
+    for (int t = 0; t < n_qt; ++t, ++qi) {
+      const int s = qi % STAGES;
+      if (!mbar_wait(bar_qfull + 8 * s, (qi / STAGES) & 1, abort_flag)) {
+        alive = false;
+        break;
+      }
+      const uint32_t q_base = q_sm + s * TILE_BYTES;
+      const int rows_valid = min(p.qt, sq.n_text - t * p.qt) * p.group;
+      if (wm * 64 < rows_valid) {
+        float acc[4][4][4];
+#pragma unroll
+        for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+          for (int nt = 0; nt < 4; ++nt) acc[mt][nt][0] = acc[mt][nt][1] = acc[mt][nt][2] = acc[mt][nt][3] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS; ++ks) {
+#pragma unroll
+          for (int mt = 0; mt < 4; ++mt) {
+            uint32_t a[4];
+            // A fragment: (rows 0-7, chunk 2ks), (rows 8-15, chunk 2ks), (rows 0-7, 2ks+1), (rows 8-15, 2ks+1)
+            const int qr = wm * 64 + mt * 16 + (mi & 1) * 8 + r8;
+            ldmatrix_x4(q_base + tile128_offset<D>(qr, 2 * ks + (mi >> 1)), a[0], a[1], a[2], a[3]);
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) mma_bf16_16816(acc[mt][nt], a, kf[ks][nt][0], kf[ks][nt][1]);
+          }
+        }
+        const int row_base = t * p.qt * p.group;     // index into this sequence's lse rows
+#pragma unroll
+        for (int mt = 0; mt < 4; ++mt) {
+#pragma unroll
+          for (int hf = 0; hf < 2; ++hf) {
+            const int r = wm * 64 + mt * 16 + (lane >> 2) + hf * 8;
+            if (r < rows_valid) {
+              const float lse = __ldg(lse_u + row_base + r);
+#pragma unroll
+              for (int nt = 0; nt < 4; ++nt) {
+                colsum[nt][0] += fast_exp2(acc[mt][nt][hf * 2] * p.scale_log2 - lse);
+                colsum[nt][1] += fast_exp2(acc[mt][nt][hf * 2 + 1] * p.scale_log2 - lse);
+              }
+            }
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_qempty + 8 * s);
+    }
+  }
+  // rows: reduce over the 8 lanes that share (lane & 3), then over the two row halves
+#pragma unroll
+  for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      float v = colsum[nt][e];
+      v += __shfl_xor_sync(0xffffffffu, v, 4);
+      v += __shfl_xor_sync(0xffffffffu, v, 8);
+      v += __shfl_xor_sync(0xffffffffu, v, 16);
+      colsum[nt][e] = v;
+    }
+  if (wm == 1 && lane < 4) {
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+      red[wn * 32 + nt * 8 + col] = colsum[nt][0];
+      red[wn * 32 + nt * 8 + col + 1] = colsum[nt][1];
+    }
+  }
+  asm volatile("bar.sync 1, 256;" ::: "memory");
+  if (!alive || *abort_flag) {
+    if (tid == 0 && p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
+    return;
+  }
+  if (wm == 0 && lane < 4) {
+    float* out = p.partial + (size_t)layer * p.sum_video + sq.score_off + kblock * kKeyTile;
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int c = wn * 32 + nt * 8 + col + e;
+        if (c < n_cols) out[c] = colsum[nt][e] + red[c];
+      }
+    }
+  }
+}
+
+// scores[j] = (sum over layers, in order, of partial[l][j]) / (L * Hq * n_text of j's sequence)
+__global__ void scores_finish_kernel(const __grid_constant__ ScoreParams p, float* __restrict__ scores) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= p.sum_video) return;
+  int b = 0;
+  while (b + 1 < p.batch && p.seq[b + 1].score_off <= j) ++b;
+  float acc = 0.f;
+  for (int l = 0; l < p.n_layers; ++l) acc += p.partial[(size_t)l * p.sum_video + j];
+  scores[j] = acc / ((float)p.n_layers * (float)p.n_q_heads * (float)p.seq[b].n_text);
+}
+
+static void ws_layout(int n_layers, int n_kv_heads, int group, int64_t sum_text, int64_t sum_video,
+                      size_t& lse_bytes, size_t& partial_bytes) {
+  lse_bytes = round_up((size_t)n_layers * n_kv_heads * sum_text * group * sizeof(float), 256);
+  partial_bytes = round_up((size_t)n_layers * sum_video * sizeof(float), 256);
+}
+
+}  // namespace specvlm
+
+using namespace specvlm;
+
+extern "C" size_t specvlm_stage1_scores_workspace_bytes(const specvlm_kv_t* target_kv,
+                                                        const int32_t* text_cu, const int32_t* video_len,
+                                                        int32_t batch, int32_t n_q_heads) {
+  if (!target_kv || !text_cu || !video_len || batch < 1 || n_q_heads < 1 || target_kv->n_kv_heads < 1 ||
+      n_q_heads % target_kv->n_kv_heads != 0)
+    return 0;
+  int64_t sum_video = 0;
+  for (int b = 0; b < batch; ++b) sum_video += video_len[b];
+  size_t a, c;
+  ws_layout(target_kv->n_layers, target_kv->n_kv_heads, n_q_heads / target_kv->n_kv_heads, text_cu[batch],
+            sum_video, a, c);
+  return a + c;
+}
+
+extern "C" int32_t specvlm_stage1_scores(const specvlm_kv_t* target_kv, const void* q_text,
+                                         const int32_t* text_cu, const int32_t* text_start,
+                                         const int32_t* video_start, const int32_t* video_len,
+                                         const int32_t* video_cu, int32_t batch, int32_t n_q_heads,
+                                         float sm_scale, float* scores, void* ws, size_t ws_bytes,
+                                         int32_t* d_status, void* stream) {
+  if (!target_kv) return SPECVLM_ERR_INVALID_ARG;
+  specvlm_kv_t kv = *target_kv;
+  static const int32_t dummy = 0;
+  if (!kv.seq_lens) kv.seq_lens = &dummy;             // lengths come from text_start / text_cu here
+  int32_t rc = validate_kv(&kv, batch, false);
+  if (rc != SPECVLM_OK) return rc;
+  if (!q_text || !text_cu || !text_start || !video_start || !video_len || !video_cu || !scores || !ws ||
+      n_q_heads < 1 || !(sm_scale > 0.f) || !aligned16(q_text))
+    return SPECVLM_ERR_INVALID_ARG;
+  if (batch > kScoresMaxBatch) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  if (n_q_heads % kv.n_kv_heads != 0) return SPECVLM_ERR_INVALID_ARG;
+  const int group = n_q_heads / kv.n_kv_heads;
+  if (group > 16) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  if (reinterpret_cast<uintptr_t>(ws) & 255u) return SPECVLM_ERR_INVALID_ARG;
+  if (kv.block_table && kv.block_tokens % 64 != 0) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+
+  ScoreParams p;
+  p.qt = 128 / group;
+  int n_row_tiles = 0, n_key_blocks = 0;
+  int64_t sum_video = 0;
+  for (int b = 0; b < batch; ++b) {
+    const int nt = text_cu[b + 1] - text_cu[b];
+    if (nt < 1 || video_len[b] < 1 || video_start[b] < 0 || video_start[b] + video_len[b] > text_start[b] ||
+        text_start[b] + nt > kv.max_seq_len || video_cu[b + 1] - video_cu[b] < video_len[b] ||
+        video_cu[b] != sum_video)
+      return SPECVLM_ERR_INVALID_ARG;
+    sum_video += video_len[b];
+  }
+  if (video_cu[batch] != sum_video) return SPECVLM_ERR_INVALID_ARG;
+  size_t lse_bytes, partial_bytes;
+  ws_layout(kv.n_layers, kv.n_kv_heads, group, text_cu[batch], sum_video, lse_bytes, partial_bytes);
+  if (ws_bytes < lse_bytes + partial_bytes) return SPECVLM_ERR_WORKSPACE_TOO_SMALL;
+  if (kv.n_layers > 65535 || kv.n_kv_heads > 65535) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+
+  p.q = static_cast<const __nv_bfloat16*>(q_text);
+  p.lse2 = static_cast<float*>(ws);
+  p.partial = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + lse_bytes);
+  p.block_table = kv.block_table;
+  p.d_status = d_status;
+  p.batch = batch;
+  p.n_layers = kv.n_layers;
+  p.n_q_heads = n_q_heads;
+  p.n_kv_heads = kv.n_kv_heads;
+  p.group = group;
+  p.sum_text = text_cu[batch];
+  p.sum_video = (int32_t)sum_video;
+  p.max_blocks = kv.max_blocks;
+  p.block_tokens = kv.block_tokens;
+  p.scale_log2 = sm_scale * kLog2e;
+
+  CUtensorMap tk, tq;
+  rc = encode_kv_map(&tk, &kv, kv.k, 64);
+  if (rc != SPECVLM_OK) return rc;
+  {
+    encode_tiled_fn enc = get_encode_tiled();
+    if (!enc) return SPECVLM_ERR_CUDA;
+    const int D = kv.head_dim;
+    const cuuint64_t dims[5] = {(cuuint64_t)D, (cuuint64_t)group, (cuuint64_t)kv.n_kv_heads,
+                                (cuuint64_t)p.sum_text, (cuuint64_t)kv.n_layers};
+    const cuuint64_t strides[4] = {(cuuint64_t)D * 2, (cuuint64_t)group * D * 2, (cuuint64_t)n_q_heads * D * 2,
+                                   (cuuint64_t)p.sum_text * n_q_heads * D * 2};
+    const cuuint32_t box[5] = {64u, (cuuint32_t)group, 1u, (cuuint32_t)p.qt, 1u};
+    const cuuint32_t estr[5] = {1u, 1u, 1u, 1u, 1u};
+    if (enc(&tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(q_text), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return SPECVLM_ERR_CUDA;
+  }
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // pass 1 tiles: row tiles per sequence; pass 2 tiles: key blocks per sequence.  The two passes
+  // use separate tile_off tables, so fill, launch pass 1 ... both passes are launched from
+  // run_scores with one params struct: store pass-1 offsets in seq[].tile_off and pass-2 offsets
+  // in a second struct.
+  ScoreParams p2 = p;
+  for (int b = 0; b < batch; ++b) {
+    const int nt = text_cu[b + 1] - text_cu[b];
+    ScoreSeq s;
+    s.text_off = text_cu[b];
+    s.n_text = nt;
+    s.text_start = text_start[b];
+    s.video_start = video_start[b];
+    s.n_video = video_len[b];
+    s.score_off = video_cu[b];
+    s.tile_off = n_row_tiles;
+    p.seq[b] = s;
+    s.tile_off = n_key_blocks;
+    p2.seq[b] = s;
+    n_row_tiles += (nt + p.qt - 1) / p.qt;
+    n_key_blocks += (video_len[b] + kKeyTile - 1) / kKeyTile;
+  }
+  // launch (pass 1 with p, pass 2 and the final reduction with p2)
+  auto launch = [&](auto tag) -> int32_t {
+    constexpr int D = decltype(tag)::value;
+    constexpr int STAGES1 = 4, STAGES2 = 3;
+    constexpr int TILE = kKeyTile * D * 2;
+    constexpr int SMEM1 = STAGES1 * TILE + 1024 + 16 * STAGES1 + 16 + 2 * 128 * 2 * 4;
+    constexpr int SMEM2 = (STAGES2 + 1) * TILE + 1024 + 16 * STAGES2 + 16 + 16 + 128 * 4;
+    auto k1 = scores_lse_kernel<D, STAGES1>;
+    auto k2 = scores_colsum_kernel<D, STAGES2>;
+    if (cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM1) != cudaSuccess ||
+        cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2) != cudaSuccess)
+      return SPECVLM_ERR_CUDA;
+    k1<<<dim3((unsigned)n_row_tiles, (unsigned)kv.n_kv_heads, (unsigned)kv.n_layers), 288, SMEM1, st>>>(tk, p);
+    int32_t r = launch_status();
+    if (r != SPECVLM_OK) return r;
+    k2<<<dim3((unsigned)n_key_blocks, (unsigned)kv.n_layers), 288, SMEM2, st>>>(tk, tq, p2);
+    r = launch_status();
+    if (r != SPECVLM_OK) return r;
+    scores_finish_kernel<<<(unsigned)((p2.sum_video + 255) / 256), 256, 0, st>>>(p2, scores);
+    return launch_status();
+  };
+  if (kv.head_dim == 128) return launch(std::integral_constant<int, 128>{});
+  return launch(std::integral_constant<int, 64>{});
+}

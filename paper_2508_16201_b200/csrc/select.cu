@@ -1,0 +1,212 @@
+// Steps 1b + 2: Stage I top-k retention and Stage II spatially uniform reduction, one CTA per
+// sequence with the whole fp32 score vector resident in shared memory.
+//   1. radix select (4 passes of 8 bits, most significant first) finds the k1-th largest key T
+//      and how many keys equal to T belong to the top-k1;
+//   2. ordered block scans give (a) the rank of each key equal to T among its equals, so ties go
+//      to the lower index, (b) the rank of each unselected token among the unselected ones,
+//      hence its rank inside its frame, (c) the output position of each kept token;
+//   3. the Stage-II pick test is integer arithmetic per token.
+// Everything is deterministic: no atomics decide an output.
+#include "common.cuh"
+#include "host_util.h"
+
+namespace specvlm {
+
+constexpr int kSelThreads = 1024;
+constexpr int kSelMaxBatch = 64;
+
+struct SelSeq {
+  int32_t score_off, n_frames, k1, k_total, kept_off;
+};
+struct SelParams {
+  const float* scores;
+  int32_t* kept_idx;
+  int32_t tokens_per_frame;
+  SelSeq seq[kSelMaxBatch];
+};
+
+// exclusive prefix sum over the block of one int per thread; returns the exclusive prefix and
+// stores the block total in *total.  warp_sums: 32 ints of shared memory.
+__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = v;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int n = __shfl_up_sync(0xffffffffu, incl, off);
+    if (lane >= off) incl += n;
+  }
+  __syncthreads();                     // warp_sums may still be read from a previous scan
+  if (lane == 31) warp_sums[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    const int ws = warp_sums[lane];
+    int wi = ws;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int n = __shfl_up_sync(0xffffffffu, wi, off);
+      if (lane >= off) wi += n;
+    }
+    warp_sums[lane] = wi - ws;         // exclusive prefix of the warp totals
+    if (lane == 31) *total = wi;
+  }
+  __syncthreads();
+  return warp_sums[warp] + incl - v;
+}
+
+__global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const __grid_constant__ SelParams p) {
+  extern __shared__ uint32_t sel_smem[];
+  const SelSeq sq = p.seq[blockIdx.x];
+  const int T = p.tokens_per_frame, F = sq.n_frames, n_v = F * T;
+  const int k1 = sq.k1, k_total = sq.k_total;
+  uint32_t* const key = sel_smem;                                  // [n_v] keys, later states
+  int* const cf = reinterpret_cast<int*>(sel_smem + n_v);         // [F + 1] unselected before frame f
+  int* const hist = cf + F + 1;                                    // [256]
+  int* const warp_sums = hist + 256;                               // [32]
+  int* const misc = warp_sums + 32;                                // [8]
+  const int tid = threadIdx.x;
+
+  // order-preserving map float -> uint32 (larger float <=> larger key)
+  const float* sc = p.scores + sq.score_off;
+  for (int j = tid; j < n_v; j += kSelThreads) {
+    const uint32_t u = __float_as_uint(sc[j]);
+    key[j] = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+  }
+
+  // ---- 1. radix select of the k1-th largest key
+  uint32_t prefix = 0, prefix_mask = 0;
+  int k_rem = k1;                      // how many of the keys matching `prefix` are still wanted
+  if (k1 > 0) {
+    for (int shift = 24; shift >= 0; shift -= 8) {
+      for (int i = tid; i < 256; i += kSelThreads) hist[i] = 0;
+      __syncthreads();
+      for (int j0 = 0; j0 < n_v; j0 += kSelThreads) {
+        const int j = j0 + tid;
+        const bool live = j < n_v && (key[j] & prefix_mask) == prefix;
+        const uint32_t digit = live ? (key[j] >> shift) & 255u : 256u;
+        // one shared-memory atomic per distinct digit in the warp
+        const uint32_t peers = __match_any_sync(0xffffffffu, digit);
+        if (live && (tid & 31) == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
+      }
+      __syncthreads();
+      if (tid == 0) {
+        int acc = 0, d = 255;
+        for (; d > 0; --d) {
+          if (acc + hist[d] >= k_rem) break;
+          acc += hist[d];
+        }
+        misc[0] = d;                   // digit of the k_rem-th largest live key
+        misc[1] = k_rem - acc;         // wanted among the keys with that digit
+      }
+      __syncthreads();
+      prefix |= static_cast<uint32_t>(misc[0]) << shift;
+      prefix_mask |= 255u << shift;
+      k_rem = misc[1];
+      __syncthreads();
+    }
+  }
+  const uint32_t thr = prefix;         // key of the k1-th largest element (when k1 > 0)
+
+  // ---- 2a. ties: keys equal to thr are taken in index order until k_rem are taken
+  // each thread owns a contiguous run of tokens so that block scans are ordered by index
+  int per = (n_v + kSelThreads - 1) / kSelThreads;
+  per |= 1;                            // odd run length: conflict-free strided shared-memory access
+  const int j_lo = min(tid * per, n_v), j_hi = min(j_lo + per, n_v);
+  int n_eq = 0;
+  if (k1 > 0)
+    for (int j = j_lo; j < j_hi; ++j) n_eq += key[j] == thr;
+  int eq_rank = block_exclusive_scan(n_eq, warp_sums, &misc[2]);
+  // states: 0 = dropped so far, 1 = in V_R
+  int n_unsel = 0;
+  for (int j = j_lo; j < j_hi; ++j) {
+    const uint32_t kj = key[j];
+    bool sel = false;
+    if (k1 > 0) {
+      if (kj > thr) sel = true;
+      else if (kj == thr) sel = eq_rank++ < k_rem;
+    }
+    key[j] = sel ? 1u : 0u;
+    n_unsel += !sel;
+  }
+  // ---- 2b. rank among the unselected tokens; unselected count before each frame
+  int m_total;
+  int e = block_exclusive_scan(n_unsel, warp_sums, &misc[3]);
+  m_total = misc[3];
+  {
+    int run = e;
+    for (int j = j_lo; j < j_hi; ++j) {
+      if (j % T == 0) cf[j / T] = run;
+      run += key[j] == 0u;
+    }
+    if (tid == 0) cf[F] = m_total;
+  }
+  __syncthreads();
+  // ---- 3. Stage II pick test, then compaction
+  const long long n_u = k_total - k1;
+  int n_keep = 0;
+  {
+    int run = e;
+    for (int j = j_lo; j < j_hi; ++j) {
+      if (key[j] == 0u) {
+        const int f = j / T;
+        const int c0 = cf[f], c1 = cf[f + 1];
+        const int c_f = c1 - c0;
+        const int rank = run - c0;
+        const int n_f = static_cast<int>((c1 * n_u) / m_total - (c0 * n_u) / m_total);
+        if (n_f > 0) {
+          const long long t = ((long long)rank * n_f + c_f - 1) / c_f;
+          if (t < n_f && (t * c_f) / n_f == rank) key[j] = 2u;
+        }
+        ++run;
+      }
+      n_keep += key[j] != 0u;
+    }
+  }
+  int pos = block_exclusive_scan(n_keep, warp_sums, &misc[4]);
+  int32_t* out = p.kept_idx + sq.kept_off;
+  for (int j = j_lo; j < j_hi; ++j)
+    if (key[j] != 0u) out[pos++] = j;
+}
+
+}  // namespace specvlm
+
+using namespace specvlm;
+
+extern "C" int32_t specvlm_select(const float* scores, const int32_t* video_cu, const int32_t* n_frames,
+                                  int32_t tokens_per_frame, const int32_t* k_stage1,
+                                  const int32_t* k_total, const int32_t* kept_cu, int32_t batch,
+                                  int32_t* kept_idx, int32_t* d_status, void* stream) {
+  (void)d_status;
+  if (!scores || !video_cu || !n_frames || !k_stage1 || !k_total || !kept_cu || !kept_idx ||
+      batch < 1 || tokens_per_frame < 1)
+    return SPECVLM_ERR_INVALID_ARG;
+  size_t max_smem = 0;
+  for (int b = 0; b < batch; ++b) {
+    const int64_t n_v = (int64_t)n_frames[b] * tokens_per_frame;
+    if (n_frames[b] < 1 || n_frames[b] > 1024 || n_v > 57344) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+    if (k_stage1[b] < 0 || k_stage1[b] > k_total[b] || k_total[b] > n_v) return SPECVLM_ERR_INVALID_ARG;
+    if (video_cu[b + 1] - video_cu[b] < n_v || kept_cu[b + 1] - kept_cu[b] < k_total[b])
+      return SPECVLM_ERR_INVALID_ARG;
+    const size_t sm = ((size_t)n_v + n_frames[b] + 1 + 256 + 32 + 8) * 4;
+    if (sm > max_smem) max_smem = sm;
+  }
+  if (max_smem > 232448) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  if (cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem) !=
+      cudaSuccess)
+    return SPECVLM_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  SelParams p;
+  p.scores = scores;
+  p.kept_idx = kept_idx;
+  p.tokens_per_frame = tokens_per_frame;
+  for (int b0 = 0; b0 < batch; b0 += kSelMaxBatch) {
+    const int nb = batch - b0 < kSelMaxBatch ? batch - b0 : kSelMaxBatch;
+    for (int i = 0; i < nb; ++i) {
+      const int b = b0 + i;
+      p.seq[i] = SelSeq{video_cu[b], n_frames[b], k_stage1[b], k_total[b], kept_cu[b]};
+    }
+    select_kernel<<<(unsigned)nb, kSelThreads, max_smem, st>>>(p);
+    const int32_t rc = launch_status();
+    if (rc != SPECVLM_OK) return rc;
+  }
+  return SPECVLM_OK;
+}

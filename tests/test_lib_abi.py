@@ -1,0 +1,70 @@
+"""The C-ABI library loads on a machine without a GPU and exports every declared symbol; host-side
+argument validation rejects bad calls before anything is launched."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2508_16201_b200 import specvlm
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    src = open(os.path.join(ROOT, "include", "specvlm.h")).read()
+    return sorted(set(re.findall(r"\b(specvlm_[a-z0-9_]+)\s*\(", src)))
+
+
+def test_library_exports_every_declared_symbol():
+    if not os.path.exists(specvlm.LIB_PATH):
+        from paper_2508_16201_b200 import build
+        build.build()
+    L = specvlm.lib()
+    names = _declared()
+    assert len(names) >= 11
+    for n in names:
+        assert hasattr(L, n), n
+    assert set(names) == set(specvlm.EXPORTS)
+    assert "sm_100a" in specvlm.version()
+    assert specvlm.status_string(0) == "ok"
+    assert specvlm.status_string(-3) == "workspace too small"
+
+
+def test_host_validation_without_gpu():
+    L = specvlm.lib()
+    kv = specvlm.KvStruct()
+    # null cache pointers
+    rc = L.specvlm_draft_decode_attn(ctypes.byref(kv), None, 1, 4, 0.1, None, None, None, 0, None, None)
+    assert rc == specvlm.ERR_INVALID_ARG
+    # unsupported head_dim
+    kv.k = kv.v = 0x1000
+    kv.seq_lens = 0x1000
+    kv.n_layers = kv.n_kv_heads = kv.n_blocks = 1
+    kv.block_tokens = kv.max_seq_len = 128
+    kv.head_dim = 96
+    kv.stride_token = 96
+    kv.stride_head = kv.stride_block = kv.stride_layer = 96 * 128
+    rc = L.specvlm_draft_decode_attn(ctypes.byref(kv), 0x1000, 1, 4, 0.1, 0x1000, None, None, 0, None, None)
+    assert rc == specvlm.ERR_UNSUPPORTED_SHAPE
+    # bad stride alignment
+    kv.head_dim = 64
+    kv.stride_token = 68
+    rc = L.specvlm_draft_decode_attn(ctypes.byref(kv), 0x1000, 1, 4, 0.1, 0x1000, None, None, 0, None, None)
+    assert rc == specvlm.ERR_INVALID_ARG
+    # gamma out of range
+    kv.stride_token = 64
+    kv.stride_head = kv.stride_block = kv.stride_layer = 64 * 128
+    rc = L.specvlm_verify_attn(ctypes.byref(kv), 0x1000, 1, 4, 9, 0.1, 0x1000, None, None, 0, None, None)
+    assert rc == specvlm.ERR_UNSUPPORTED_SHAPE
+    # select: k_stage1 > k_total
+    i32 = lambda *a: (ctypes.c_int32 * len(a))(*a)
+    rc = L.specvlm_select(0x1000, i32(0, 100), i32(1), 100, i32(20), i32(10), i32(0, 10), 1, 0x1000, None, None)
+    assert rc == specvlm.ERR_INVALID_ARG
+    # select: too many tokens for one CTA
+    rc = L.specvlm_select(0x1000, i32(0, 80000), i32(800), 100, i32(10), i32(20), i32(0, 20), 1, 0x1000, None, None)
+    assert rc == specvlm.ERR_UNSUPPORTED_SHAPE
+    # accept: workspace too small
+    rc = L.specvlm_accept(0x1000, 0x1000, 1, 4, 1024, 0x1000, 0x1000, None, 0x1000, 8, None)
+    assert rc == specvlm.ERR_WORKSPACE_TOO_SMALL
+    assert L.specvlm_accept_workspace_bytes(1, 4, 1024) >= 5 * 8
