@@ -303,7 +303,6 @@ attn_rowsN_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   constexpr int NT_W = D / 32;               // n-tiles of 8 channels per warp in PV
   constexpr int GROWS = MT * 16;             // rows per group
   constexpr int P_BYTES = GROWS * 128;       // one group's probability tile (64 tokens bf16 per row)
-  constexpr int CONSUMERS = 128 * NG;
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -429,15 +428,14 @@ attn_rowsN_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   bool alive = true;
   for (int i = 0; i < n_my; ++i) {
     const int s = i % STAGES;
-    if (!mbar_wait(bar_full + 8 * s, (i / STAGES) & 1, abort_flag)) {
-      alive = false;
-      break;
-    }
+    // A warp whose wait expired keeps taking part in the group barriers below (its results are
+    // discarded at the end), so the other warps of the group can never be left waiting for it.
+    if (alive && !mbar_wait(bar_full + 8 * s, (i / STAGES) & 1, abort_flag)) alive = false;
     const uint32_t k_base = base + s * STAGE_BYTES;
     const uint32_t v_base = k_base + TILE_BYTES;
     const int tile_tok0 = (tile_begin + i) * kTileTokens;
     const int tb = tile_tok0 + cw * 16;
-    if (tile_tok0 + kTileTokens > kv_len) {
+    if (alive && tile_tok0 + kTileTokens > kv_len) {
       // clear the V rows past the end of the sequence (see kernel A); this warp clears the rows of
       // its own 16-token slice, the group barrier below publishes them to the other warps
       uint8_t* vt = smem + s * STAGE_BYTES + TILE_BYTES;
@@ -455,7 +453,7 @@ attn_rowsN_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
       for (int nt = 0; nt < 2; ++nt) sc[mt][nt][0] = sc[mt][nt][1] = sc[mt][nt][2] = sc[mt][nt][3] = 0.f;
-    if (tb < kv_len) {
+    if (alive && tb < kv_len) {
 #pragma unroll
       for (int ks = 0; ks < KSTEPS; ++ks) {
         uint32_t b0, b1, b2, b3;
@@ -538,7 +536,7 @@ attn_rowsN_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
       }
     }
     __syncwarp();
-    if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+    if (lane == 0 && alive) mbar_arrive(bar_empty + 8 * s);
   }
 
   // ------------------------------------------------------------ row sums across the group's warps

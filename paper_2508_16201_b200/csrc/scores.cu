@@ -290,8 +290,9 @@ scores_colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
   const ScoreSeq sq = p.seq[b];
   const int kblock = blockIdx.x - sq.tile_off;
   const int layer = blockIdx.y;
-  const int key0 = sq.video_start + kblock * kKeyTile;           // absolute position of column 0
-  const int n_cols = min(kKeyTile, sq.n_video - kblock * kKeyTile);
+  // key blocks start on a page boundary at or before the first video token, so that a 64-token
+  // TMA box never straddles two cache pages; columns outside the video range are dropped
+  const int key0 = (sq.video_start / 64) * 64 + kblock * kKeyTile;   // absolute position of column 0
   const int n_qt = (sq.n_text + p.qt - 1) / p.qt;
   const int n_units = p.n_kv_heads;
 
@@ -446,13 +447,14 @@ scores_colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     return;
   }
   if (wm == 0 && lane < 4) {
-    float* out = p.partial + (size_t)layer * p.sum_video + sq.score_off + kblock * kKeyTile;
+    float* out = p.partial + (size_t)layer * p.sum_video + sq.score_off;
 #pragma unroll
     for (int nt = 0; nt < 4; ++nt) {
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
         const int c = wn * 32 + nt * 8 + col + e;
-        if (c < n_cols) out[c] = colsum[nt][e] + red[c];
+        const int j = key0 + c - sq.video_start;        // video token index of column c
+        if (j >= 0 && j < sq.n_video) out[j] = colsum[nt][e] + red[c];
       }
     }
   }
@@ -588,7 +590,7 @@ extern "C" int32_t specvlm_stage1_scores(const specvlm_kv_t* target_kv, const vo
     s.tile_off = n_key_blocks;
     p2.seq[b] = s;
     n_row_tiles += (nt + p.qt - 1) / p.qt;
-    n_key_blocks += (video_len[b] + kKeyTile - 1) / kKeyTile;
+    n_key_blocks += (video_start[b] % 64 + video_len[b] + kKeyTile - 1) / kKeyTile;
   }
   // launch (pass 1 with p, pass 2 and the final reduction with p2)
   auto launch = [&](auto tag) -> int32_t {
