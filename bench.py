@@ -1,0 +1,511 @@
+#!/usr/bin/env python
+"""Benchmark of the SpecVLM pruned-draft speculative-decoding hot path on B200.
+
+One step = one pass of the whole hot path over the LLaVA-OneVision-72B / 7B shaped workload
+(6272 video + 128 text tokens, batch 1):
+    token-rating row LSE -> token rating -> select -> gather -> gamma x draft decode attention
+    -> verify attention -> accept.
+The headline value is the K/V bandwidth of the memory-bound attention calls (draft decode over the
+pruned cache + verification over the full cache): K/V bytes they must read once / their device
+time.  Prune time (rating + select, gather listed apart) and every call's time are reported too.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+`--impl reference` times the CPU oracle (the plain fp64 restatement of the method) on the host
+cores, on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "draft-decode + verify attention KV GB/s"
+UNIT = "GB/s"
+HBM_NOMINAL_GBS = 8000.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d["bf16_tflops_sustained"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
+# summarised under profiles/; None until a capture exists for the kernel.
+NCU_TRAFFIC_BYTES = {"verify": None, "decode": None, "scores_colsum": None, "scores_lse": None}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------------
+def build_inputs(w, device, n_copies):
+    """Synthetic tensors of the workload, resident on the device."""
+    import torch
+    from paper_2508_16201_b200 import specvlm, synth
+    D, nv, nt, g1 = w.head_dim, w.n_video(), w.n_text[0], w.gamma + 1
+    n_t = nv + nt + g1                      # verifier cache incl. the gamma+1 new tokens
+    inp = {}
+    tk = synth.randn_bf16((w.t_layers, 1, w.t_kv_heads, n_t, D), device, 0, "tK")
+    tv = synth.randn_bf16((w.t_layers, 1, w.t_kv_heads, n_t, D), device, 0, "tV")
+    q_text = synth.randn_bf16((w.t_layers, nt, w.t_q_heads, D), device, 0, "Qtext")
+    synth.plant_salient_(tk[:, 0, :, :nv, :], q_text, synth.salient_set(nv, w.planted_permille, 0))
+    lens_t = torch.tensor([n_t], dtype=torch.int32, device=device)
+    inp["tcache"] = specvlm.KvCache(tk, tv, lens_t, n_t)
+    # rating reads the prompt part only (the same memory, shorter length bound)
+    inp["tcache_prompt"] = specvlm.KvCache(tk, tv, torch.tensor([nv + nt], dtype=torch.int32, device=device),
+                                           nv + nt)
+    inp["q_text"] = q_text
+    # draft: full-length cache (gather source) and gamma+1 pruned copies (copy 0 = gather target)
+    n_d = nv + nt
+    sk = synth.randn_bf16((w.d_layers, 1, w.d_kv_heads, n_d, D), device, 0, "dK")
+    sv = synth.randn_bf16((w.d_layers, 1, w.d_kv_heads, n_d, D), device, 0, "dV")
+    inp["dsrc"] = specvlm.KvCache(sk, sv, torch.tensor([n_d], dtype=torch.int32, device=device), n_d)
+    n_p = w.k_total() + nt
+    lens_p = torch.tensor([n_p], dtype=torch.int32, device=device)
+    inp["dpruned"] = []
+    for c in range(n_copies + 1):
+        pk = torch.zeros((w.d_layers, 1, w.d_kv_heads, n_p, D), dtype=torch.bfloat16, device=device)
+        pv = torch.zeros_like(pk)
+        inp["dpruned"].append(specvlm.KvCache(pk, pv, lens_p, n_p))
+    inp["q_dec"] = [synth.randn_bf16((w.d_layers, 1, w.d_q_heads, D), device, 0, "Qd", c) for c in range(w.gamma)]
+    inp["q_ver"] = synth.randn_bf16((w.t_layers, 1, g1, w.t_q_heads, D), device, 0, "Qv")
+    inp["logits"], inp["drafts"] = synth.logits_and_drafts(1, w.gamma, w.vocab, device, 0)
+    return inp
+
+
+class Path:
+    """Pre-allocated outputs / workspaces and the sequence of C-ABI calls of one step."""
+
+    def __init__(self, w, inp, device):
+        import torch
+        from paper_2508_16201_b200 import specvlm
+        self.w, self.inp, self.sv, self.torch = w, inp, specvlm, torch
+        D, nv, nt = w.head_dim, w.n_video(), w.n_text[0]
+        self.scale = 1.0 / math.sqrt(D)
+        self.kt, self.k1 = w.k_total(), w.k_stage1()
+        self.row_lse = torch.empty((w.t_layers, nt, w.t_q_heads), dtype=torch.float32, device=device)
+        self.scores = torch.empty(nv, dtype=torch.float32, device=device)
+        self.ws_scores = torch.empty(specvlm.stage1_scores_workspace_bytes(inp["tcache_prompt"], [0, nt], [nv],
+                                                                           w.t_q_heads),
+                                     dtype=torch.uint8, device=device)
+        self.kept = torch.empty(self.kt, dtype=torch.int32, device=device)
+        self.o_dec = [torch.empty_like(q) for q in inp["q_dec"]]
+        self.ws_dec = torch.empty(max(256, specvlm.attn_workspace_bytes(inp["dpruned"][0], 1, w.d_q_heads, 0)),
+                                  dtype=torch.uint8, device=device)
+        self.o_ver = torch.empty_like(inp["q_ver"])
+        self.ws_ver = torch.empty(max(256, specvlm.attn_workspace_bytes(inp["tcache"], 1, w.t_q_heads, w.gamma)),
+                                  dtype=torch.uint8, device=device)
+        self.acc = (torch.empty(1, dtype=torch.int32, device=device),
+                    torch.empty(1, dtype=torch.int32, device=device), None)
+        self.ws_acc = torch.empty(specvlm.accept_workspace_bytes(1, w.gamma, w.vocab), dtype=torch.uint8,
+                                  device=device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        # launches of our kernels per step
+        dec_l = 1 + (specvlm.attn_workspace_bytes(inp["dpruned"][0], 1, w.d_q_heads, 0) > 256)
+        ver_l = 1 + (specvlm.attn_workspace_bytes(inp["tcache"], 1, w.t_q_heads, w.gamma) > 256)
+        self.launches_per_step = 1 + 2 + 1 + 1 + w.gamma * dec_l + ver_l + 2
+
+    # the calls, in path order ------------------------------------------------------------------
+    def row_lse_call(self):
+        w, nv, nt = self.w, self.w.n_video(), self.w.n_text[0]
+        self.sv.stage1_row_lse(self.inp["tcache_prompt"], self.inp["q_text"], [0, nt], [nv], self.scale,
+                               row_lse=self.row_lse, d_status=self.status)
+
+    def scores_call(self):
+        nv, nt = self.w.n_video(), self.w.n_text[0]
+        self.sv.stage1_scores(self.inp["tcache_prompt"], self.inp["q_text"], [0, nt], [nv], [0], [nv], [0, nv],
+                              self.scale, scores=self.scores, ws=self.ws_scores, d_status=self.status,
+                              row_lse=self.row_lse)
+
+    def select_call(self):
+        w, nv = self.w, self.w.n_video()
+        self.sv.select(self.scores, [0, nv], [w.n_frames[0]], w.tokens_per_frame, [self.k1], [self.kt],
+                       [0, self.kt], kept_idx=self.kept, d_status=self.status)
+
+    def gather_call(self, dst):
+        nv, nt = self.w.n_video(), self.w.n_text[0]
+        self.sv.gather_kv(self.inp["dsrc"], self.kept, [0, self.kt], [0], [nv], [nv + nt], dst,
+                          d_status=self.status)
+
+    def decode_call(self, c, cache):
+        self.sv.draft_decode_attn(cache, self.inp["q_dec"][c], self.scale, out=self.o_dec[c], ws=self.ws_dec,
+                                  d_status=self.status)
+
+    def verify_call(self):
+        self.sv.verify_attn(self.inp["tcache"], self.inp["q_ver"], self.w.gamma, self.scale, out=self.o_ver,
+                            ws=self.ws_ver, d_status=self.status)
+
+    def accept_call(self):
+        self.sv.accept(self.inp["logits"], self.inp["drafts"], ws=self.ws_acc, out=self.acc)
+
+
+SEGMENTS = ["row_lse", "scores", "select", "gather", "decode", "verify", "accept"]
+
+
+def run_ours(args, rank, world):
+    import torch
+    import torch.distributed as dist
+    from paper_2508_16201_b200 import specvlm, synth
+
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    specvlm.lib()
+    w = synth.workload(2)
+    D, nv, nt, gamma = w.head_dim, w.n_video(), w.n_text[0], w.gamma
+    inp = build_inputs(w, device, n_copies=gamma)
+    path = Path(w, inp, device)
+    E = lambda: torch.cuda.Event(enable_timing=True)
+
+    # one-time: fill every pruned copy with real gathered data (copies 1.. are the decode inputs)
+    path.row_lse_call(); path.scores_call(); path.select_call()
+    for c in inp["dpruned"]:
+        path.gather_call(c)
+    torch.cuda.synchronize()
+
+    def step(ev):
+        """ev: dict name -> list of (start, stop) event pairs appended for this step (or None)."""
+        def seg(name, fn):
+            if ev is None:
+                fn()
+                return
+            a, b = E(), E()
+            a.record()
+            fn()
+            b.record()
+            ev[name].append((a, b))
+        seg("row_lse", path.row_lse_call)
+        seg("scores", path.scores_call)
+        seg("select", path.select_call)
+        seg("gather", lambda: path.gather_call(inp["dpruned"][0]))
+        for c in range(gamma):
+            # each draft step reads its own copy of the pruned cache: nothing is L2-resident
+            seg("decode", lambda c=c: path.decode_call(c, inp["dpruned"][1 + c]))
+        seg("verify", path.verify_call)
+        seg("accept", path.accept_call)
+
+    for _ in range(args.warmup):
+        step(None)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    ev = {k: [] for k in SEGMENTS}
+    t0, t1 = E(), E()
+    torch.cuda.synchronize()
+    t0.record()
+    for _ in range(args.steps):
+        step(ev)
+    t1.record()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    total_ms = t0.elapsed_time(t1)
+    if rank == 0:
+        time.sleep(0.2)
+    clocks = sampler.stop() if rank == 0 else None
+    assert int(path.status.item()) == 0, "a device-side wait timed out"
+    seg_ms = {k: [a.elapsed_time(b) for a, b in v] for k, v in ev.items()}
+    mean = {k: sum(v) / len(v) for k, v in seg_ms.items()}          # per call
+    med = {k: statistics.median(v) for k, v in seg_ms.items()}
+
+    # algorithmic K/V bytes (read once): 2 (K,V) * tokens * kv_heads * d * 2 B * layers
+    n_p = w.k_total() + nt
+    n_t = nv + nt + gamma + 1
+    bytes_dec = 2 * n_p * w.d_kv_heads * D * 2 * w.d_layers
+    bytes_ver = 2 * n_t * w.t_kv_heads * D * 2 * w.t_layers
+    attn_ms = mean["decode"] * gamma + mean["verify"]
+    attn_bytes = bytes_dec * gamma + bytes_ver
+
+    # ---------------- end-to-end leg: inputs from pinned host memory, results read back
+    e2e = run_e2e(args, path, inp, w, device, attn_bytes)
+
+    # ---------------- extras outside the timed region: unpruned draft cache (the SD baseline draft)
+    extra = {}
+    dsrc = inp["dsrc"]
+    ws_u = torch.empty(max(256, specvlm.attn_workspace_bytes(dsrc, 1, w.d_q_heads, 0)), dtype=torch.uint8,
+                       device=device)
+    ts = []
+    for i in range(3 + 10):
+        a, b = E(), E()
+        a.record()
+        specvlm.draft_decode_attn(dsrc, inp["q_dec"][0], path.scale, out=path.o_dec[0], ws=ws_u)
+        b.record()
+        torch.cuda.synchronize()
+        if i >= 3:
+            ts.append(a.elapsed_time(b))
+    bytes_unpruned = 2 * (nv + nt) * w.d_kv_heads * D * 2 * w.d_layers
+    extra["decode_unpruned_us"] = statistics.median(ts) * 1e3
+    extra["decode_unpruned_kv_gbs"] = bytes_unpruned / (statistics.median(ts) * 1e-3) / 1e9
+
+    # max over ranks
+    if world > 1:
+        t = torch.tensor([total_ms, attn_ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, attn_ms = float(t[0]), float(t[1])
+    if rank != 0:
+        return
+    peaks = measured_peaks()
+    value = world * attn_bytes / (attn_ms * 1e-3) / 1e9
+
+    def hbm(name, nbytes, ms, traffic):
+        ach = nbytes / (ms * 1e-3) / 1e9
+        return {"kernel": name, "bound": "hbm", "achieved": round(ach, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": round(ach / peaks["hbm_gbs"], 4), "frac_of_nominal_8000": round(ach / HBM_NOMINAL_GBS, 4),
+                "traffic": traffic, "peak_source": peaks["source"], "launch_ms": round(ms, 5)}
+
+    def tensor(name, flops, ms, traffic):
+        ach = flops / (ms * 1e-3) / 1e12
+        return {"kernel": name, "bound": "tensor", "achieved": round(ach, 1), "peak": peaks["bf16_tflops_sustained"],
+                "unit": "TFLOP/s", "frac": round(ach / peaks["bf16_tflops_sustained"], 4), "traffic": traffic,
+                "peak_source": peaks["source"] + " (sustained bf16)", "launch_ms": round(ms, 5)}
+
+    rows = w.t_layers * w.t_q_heads * nt
+    flops_colsum = 2.0 * rows * nv * D
+    flops_lse = 2.0 * w.t_layers * w.t_q_heads * D * sum(nv + i + 1 for i in range(nt))
+    roofs = {
+        "verify": hbm("attn_rowsN_kernel (verify)", bytes_ver, mean["verify"], NCU_TRAFFIC_BYTES["verify"]),
+        "decode": hbm("attn_rows16_kernel (draft decode, pruned cache)", bytes_dec, mean["decode"],
+                      NCU_TRAFFIC_BYTES["decode"]),
+        "scores_colsum": tensor("scores_colsum_kernel", flops_colsum, mean["scores"],
+                                NCU_TRAFFIC_BYTES["scores_colsum"]),
+        "scores_lse": tensor("scores_lse_kernel", flops_lse, mean["row_lse"], NCU_TRAFFIC_BYTES["scores_lse"]),
+    }
+    dominant = max(("scores_colsum", "scores_lse", "verify", "decode"),
+                   key=lambda k: {"scores_colsum": mean["scores"], "scores_lse": mean["row_lse"],
+                                  "verify": mean["verify"], "decode": mean["decode"] * gamma}[k])
+    out = {
+        "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(total_ms / args.steps, 4), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name + ": verifier 80L 64q/8kv d128, draft 28L 28q/4kv, 6272 video + 128 text "
+                               "tokens, retention 10%, gamma 5, vocab 152064, batch 1, contiguous caches",
+                   "l2": "verify cache 2.1 GB and rating K 1.05 GB exceed L2; each of the gamma draft steps reads "
+                         "its own copy of the 43 MB pruned cache (6 copies, 260 MB), so no call finds its K/V in L2",
+                   "replicas": world},
+        "pct_of_hbm_peak": {"of_measured_%d" % int(peaks["hbm_gbs"]): round(100 * value / world / peaks["hbm_gbs"], 2),
+                            "of_nominal_8000": round(100 * value / world / HBM_NOMINAL_GBS, 2)},
+        "per_call_us": {k: round(mean[k] * 1e3, 2) for k in SEGMENTS},
+        "per_call_us_median": {k: round(med[k] * 1e3, 2) for k in SEGMENTS},
+        "prune_us_per_call": round((mean["row_lse"] + mean["scores"] + mean["select"]) * 1e3, 2),
+        "prune_us_with_caller_lse": round((mean["scores"] + mean["select"]) * 1e3, 2),
+        "prune_total_us_with_gather": round((mean["row_lse"] + mean["scores"] + mean["select"] + mean["gather"]) * 1e3, 2),
+        "kv_gbs": {"decode_pruned": round(bytes_dec / (mean["decode"] * 1e-3) / 1e9, 1),
+                   "verify": round(bytes_ver / (mean["verify"] * 1e-3) / 1e9, 1),
+                   "gather_rw": round(2 * bytes_dec / (mean["gather"] * 1e-3) / 1e9, 1),
+                   "accept_logits": round((gamma + 1) * w.vocab * 4 / (mean["accept"] * 1e-3) / 1e9, 1)},
+        "extra": {k: round(v, 2) for k, v in extra.items()},
+        "roofline": roofs[dominant], "roofline_all": roofs,
+        "e2e": e2e, "gpu_launches": path.launches_per_step * args.steps,
+        "clocks": clocks,
+    }
+    if args.cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(w)
+    print(json.dumps(out))
+
+
+def run_e2e(args, path, inp, w, device, attn_bytes):
+    """Same step, but every call's inputs start in pinned host memory and its result is read back;
+    the copies sit inside the timed regions.  The K/V caches are the serving state and stay on the
+    device."""
+    import torch
+    gamma = w.gamma
+    pin = lambda t: t.detach().cpu().pin_memory()
+    h_qtext, h_qver = pin(inp["q_text"]), pin(inp["q_ver"])
+    h_qdec = [pin(q) for q in inp["q_dec"]]
+    h_logits, h_drafts = pin(inp["logits"]), pin(inp["drafts"])
+    h_kept = torch.empty(path.kt, dtype=torch.int32).pin_memory()
+    h_odec = [torch.empty_like(h) for h in h_qdec]
+    h_odec = [h.pin_memory() for h in h_odec]
+    h_over = torch.empty_like(h_qver).pin_memory()
+    h_acc = torch.empty(2, dtype=torch.int32).pin_memory()
+    h2d = (h_qtext.numel() * 2 + h_qver.numel() * 2 + sum(h.numel() * 2 for h in h_qdec) + h_logits.numel() * 4 +
+           h_drafts.numel() * 4)
+    d2h = h_kept.numel() * 4 + sum(h.numel() * 2 for h in h_odec) + h_over.numel() * 2 + 8
+    E = lambda: torch.cuda.Event(enable_timing=True)
+    attn_ms, step_ms = [], []
+    for it in range(args.warmup + args.steps):
+        s0, s1 = E(), E()
+        s0.record()
+        inp["q_text"].copy_(h_qtext, non_blocking=True)
+        path.row_lse_call(); path.scores_call(); path.select_call()
+        h_kept.copy_(path.kept, non_blocking=True)
+        path.gather_call(inp["dpruned"][0])
+        a0, a1 = E(), E()
+        a0.record()
+        for c in range(gamma):
+            inp["q_dec"][c].copy_(h_qdec[c], non_blocking=True)
+            path.decode_call(c, inp["dpruned"][1 + c])
+            h_odec[c].copy_(path.o_dec[c], non_blocking=True)
+        inp["q_ver"].copy_(h_qver, non_blocking=True)
+        path.verify_call()
+        h_over.copy_(path.o_ver, non_blocking=True)
+        a1.record()
+        inp["logits"].copy_(h_logits, non_blocking=True)
+        inp["drafts"].copy_(h_drafts, non_blocking=True)
+        path.accept_call()
+        h_acc[0:1].copy_(path.acc[0], non_blocking=True)
+        h_acc[1:2].copy_(path.acc[1], non_blocking=True)
+        s1.record()
+        torch.cuda.synchronize()
+        if it >= args.warmup:
+            attn_ms.append(a0.elapsed_time(a1))
+            step_ms.append(s0.elapsed_time(s1))
+    am = sum(attn_ms) / len(attn_ms)
+    return {"value": round(attn_bytes / (am * 1e-3) / 1e9, 1), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+            "d2h_bytes_per_step": int(d2h), "ms_per_step": round(sum(step_ms) / len(step_ms), 4),
+            "attention_ms_per_step": round(am, 4),
+            "note": "pinned host q / logits in, outputs out, inside the timed region; K/V caches resident"}
+
+
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(w, n_verify_layers):
+    """Times the CPU oracle on a bounded sample: gamma draft decode steps over the pruned cache (all
+    draft layers) + verification over n_verify_layers verifier layers.  Returns (KV bytes, seconds)."""
+    import numpy as np
+    import oracle
+    rng = np.random.default_rng(0)
+    D, nv, nt, gamma = w.head_dim, w.n_video(), w.n_text[0], w.gamma
+    n_p, n_t = w.k_total() + nt, nv + nt + gamma + 1
+    scale = 1.0 / math.sqrt(D)
+
+    def bf16(shape):
+        return (rng.standard_normal(shape).astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
+    kd, vd = bf16((w.d_kv_heads, n_p, D)), bf16((w.d_kv_heads, n_p, D))
+    qd = bf16((1, w.d_q_heads, D))
+    kt_, vt_ = bf16((w.t_kv_heads, n_t, D)), bf16((w.t_kv_heads, n_t, D))
+    qv = bf16((gamma + 1, w.t_q_heads, D))
+    t0 = time.perf_counter()
+    for _ in range(gamma):
+        for _l in range(w.d_layers):
+            oracle.attention(qd, kd, vd, n_p, scale)
+    for _l in range(n_verify_layers):
+        oracle.attention(qv, kt_, vt_, n_t, scale)
+    dt = time.perf_counter() - t0
+    nbytes = gamma * w.d_layers * 2 * n_p * w.d_kv_heads * D * 2 + n_verify_layers * 2 * n_t * w.t_kv_heads * D * 2
+    return nbytes, dt
+
+
+def cpu_baseline(w):
+    import oracle
+    n_layers = w.t_layers
+    nbytes, dt = oracle_sample(w, n_layers)
+    return {"value": round(nbytes / dt / 1e9, 4), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "seconds": round(dt, 2),
+            "sample": f"fp64 oracle attention: {w.gamma} draft decode steps over the pruned cache (all {w.d_layers} "
+                      f"draft layers) + verification over {n_layers} of {w.t_layers} verifier layers"}
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    from paper_2508_16201_b200 import synth
+    import oracle
+    w = synth.workload(2)
+    n_layers = 16                           # bounded sample per step
+    for _ in range(args.warmup):
+        oracle_sample(w, 1)
+    tot_b, tot_t = 0, 0.0
+    for _ in range(args.steps):
+        b, t = oracle_sample(w, n_layers)
+        tot_b += b
+        tot_t += t
+    v = round(tot_b / tot_t / 1e9, 4)
+    sample = (f"fp64 oracle attention per step: {w.gamma} draft decode steps over the pruned cache (all "
+              f"{w.d_layers} draft layers) + verification over {n_layers} of {w.t_layers} verifier layers")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(tot_t / args.steps * 1e3, 2), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name + " (bounded sample, see cpu_baseline.sample)"},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    args.warmup = max(args.warmup, 3)
+    if world > 1 or rank != 0:
+        args.cpu_baseline = False
+    run_ours(args, rank, world)
+
+
+if __name__ == "__main__":
+    main()

@@ -88,19 +88,30 @@ const char* specvlm_status_string(int32_t status);
  *   video_start, video_len   host int32 [batch]; video_start+video_len <= text_start
  *   video_cu    host int32 [batch+1]: offsets of each sequence's scores in `scores`
  *   scores      device fp32 [video_cu[batch]] out
+ *   row_lse_or_null  device fp32 [n_layers][sum_text][n_q_heads] or NULL: the natural-log
+ *               sum-exp of each language query's scaled causal logits.  An attention kernel that ran
+ *               the prefill usually has it; when NULL it is computed first (one more pass over QK^T),
+ *               exactly as specvlm_stage1_row_lse would.
  *   ws          device scratch, specvlm_stage1_scores_workspace_bytes(...)
  * Deterministic: the reduction order over rows, heads and layers is fixed.
- * Supported: head_dim 128 or 64, n_q_heads / n_kv_heads in 1..16.
+ * Supported: head_dim 128 or 64, n_q_heads / n_kv_heads in 1..16, batch <= 64.
+ *
+ * specvlm_stage1_row_lse is the first half on its own: it writes row_lse (same layout) and
+ * needs no scratch.
  */
 size_t specvlm_stage1_scores_workspace_bytes(const specvlm_kv_t* target_kv, const int32_t* text_cu,
                                              const int32_t* video_len, int32_t batch,
                                              int32_t n_q_heads);
+int32_t specvlm_stage1_row_lse(const specvlm_kv_t* target_kv, const void* q_text,
+                               const int32_t* text_cu, const int32_t* text_start, int32_t batch,
+                               int32_t n_q_heads, float sm_scale, float* row_lse, int32_t* d_status,
+                               void* stream);
 int32_t specvlm_stage1_scores(const specvlm_kv_t* target_kv, const void* q_text,
                               const int32_t* text_cu, const int32_t* text_start,
                               const int32_t* video_start, const int32_t* video_len,
                               const int32_t* video_cu, int32_t batch, int32_t n_q_heads,
-                              float sm_scale, float* scores, void* ws, size_t ws_bytes,
-                              int32_t* d_status, void* stream);
+                              float sm_scale, const float* row_lse_or_null, float* scores, void* ws,
+                              size_t ws_bytes, int32_t* d_status, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Steps 1b + 2 -- two-stage selection (Section 4.2).

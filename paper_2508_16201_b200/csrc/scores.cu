@@ -25,7 +25,7 @@ struct ScoreSeq {
 
 struct ScoreParams {
   const __nv_bfloat16* q;              // [L][sum_text][Hq][D]
-  float* lse2;                         // [L][Hkv][sum_text * group]  (log2 units, of scaled logits)
+  float* lse;                          // [L][sum_text][Hq]: natural-log sum-exp of the scaled logits
   float* partial;                      // [L][sum_video]
   const int32_t* block_table;
   int32_t* d_status;
@@ -254,8 +254,9 @@ scores_lse_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     const float mb = red[(128 + tid) * 2], lb2 = red[(128 + tid) * 2 + 1];
     const float M = fmaxf(ma, mb);
     const float L = la * fast_exp2(ma - M) + lb2 * fast_exp2(mb - M);
-    p.lse2[((size_t)layer * p.n_kv_heads + g) * ((size_t)p.sum_text * p.group) +
-           (size_t)(sq.text_off + i_first) * p.group + tid] = M + log2f(L);
+    const int il = tid / p.group, hg = tid - il * p.group;
+    p.lse[((size_t)layer * p.sum_text + sq.text_off + i_first + il) * p.n_q_heads + g * p.group + hg] =
+        (M + log2f(L)) * kLn2;
   }
 }
 
@@ -374,8 +375,7 @@ scores_colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(bar_kempty);
-    const float* lse_u = p.lse2 + ((size_t)layer * p.n_kv_heads + u) * ((size_t)p.sum_text * p.group) +
-                         (size_t)sq.text_off * p.group;
+    const float* lse_u = p.lse + ((size_t)layer * p.sum_text + sq.text_off) * p.n_q_heads + u * p.group;
     for (int t = 0; t < n_qt; ++t, ++qi) {
       const int s = qi % STAGES;
       if (!mbar_wait(bar_qfull + 8 * s, (qi / STAGES) & 1, abort_flag)) {
@@ -402,14 +402,14 @@ scores_colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             for (int nt = 0; nt < 4; ++nt) mma_bf16_16816(acc[mt][nt], a, kf[ks][nt][0], kf[ks][nt][1]);
           }
         }
-        const int row_base = t * p.qt * p.group;     // index into this sequence's lse rows
 #pragma unroll
         for (int mt = 0; mt < 4; ++mt) {
 #pragma unroll
           for (int hf = 0; hf < 2; ++hf) {
             const int r = wm * 64 + mt * 16 + (lane >> 2) + hf * 8;
             if (r < rows_valid) {
-              const float lse = __ldg(lse_u + row_base + r);
+              const int il = r / p.group, hg = r - il * p.group;
+              const float lse = __ldg(lse_u + (size_t)(t * p.qt + il) * p.n_q_heads + hg) * kLog2e;
 #pragma unroll
               for (int nt = 0; nt < 4; ++nt) {
                 colsum[nt][0] += fast_exp2(acc[mt][nt][hf * 2] * p.scale_log2 - lse);
@@ -471,73 +471,58 @@ __global__ void scores_finish_kernel(const __grid_constant__ ScoreParams p, floa
   scores[j] = acc / ((float)p.n_layers * (float)p.n_q_heads * (float)p.seq[b].n_text);
 }
 
-static void ws_layout(int n_layers, int n_kv_heads, int group, int64_t sum_text, int64_t sum_video,
-                      size_t& lse_bytes, size_t& partial_bytes) {
-  lse_bytes = round_up((size_t)n_layers * n_kv_heads * sum_text * group * sizeof(float), 256);
+static void ws_layout(int n_layers, int n_q_heads, int64_t sum_text, int64_t sum_video, size_t& lse_bytes,
+                      size_t& partial_bytes) {
+  lse_bytes = round_up((size_t)n_layers * sum_text * n_q_heads * sizeof(float), 256);
   partial_bytes = round_up((size_t)n_layers * sum_video * sizeof(float), 256);
 }
 
-}  // namespace specvlm
+struct ScoreSetup {
+  specvlm_kv_t kv;
+  ScoreParams p1, p2;          // pass-1 (row tiles) and pass-2 (key blocks) CTA tables
+  CUtensorMap tk, tq;
+  int n_row_tiles, n_key_blocks;
+};
 
-using namespace specvlm;
-
-extern "C" size_t specvlm_stage1_scores_workspace_bytes(const specvlm_kv_t* target_kv,
-                                                        const int32_t* text_cu, const int32_t* video_len,
-                                                        int32_t batch, int32_t n_q_heads) {
-  if (!target_kv || !text_cu || !video_len || batch < 1 || n_q_heads < 1 || target_kv->n_kv_heads < 1 ||
-      n_q_heads % target_kv->n_kv_heads != 0)
-    return 0;
-  int64_t sum_video = 0;
-  for (int b = 0; b < batch; ++b) sum_video += video_len[b];
-  size_t a, c;
-  ws_layout(target_kv->n_layers, target_kv->n_kv_heads, n_q_heads / target_kv->n_kv_heads, text_cu[batch],
-            sum_video, a, c);
-  return a + c;
-}
-
-extern "C" int32_t specvlm_stage1_scores(const specvlm_kv_t* target_kv, const void* q_text,
-                                         const int32_t* text_cu, const int32_t* text_start,
-                                         const int32_t* video_start, const int32_t* video_len,
-                                         const int32_t* video_cu, int32_t batch, int32_t n_q_heads,
-                                         float sm_scale, float* scores, void* ws, size_t ws_bytes,
-                                         int32_t* d_status, void* stream) {
+// Validates the arguments common to both entry points and fills the launch tables.
+static int32_t setup_scores(const specvlm_kv_t* target_kv, const void* q_text, const int32_t* text_cu,
+                            const int32_t* text_start, const int32_t* video_start, const int32_t* video_len,
+                            const int32_t* video_cu, int32_t batch, int32_t n_q_heads, float sm_scale,
+                            int32_t* d_status, ScoreSetup& su) {
   if (!target_kv) return SPECVLM_ERR_INVALID_ARG;
-  specvlm_kv_t kv = *target_kv;
+  su.kv = *target_kv;
+  specvlm_kv_t& kv = su.kv;
   static const int32_t dummy = 0;
   if (!kv.seq_lens) kv.seq_lens = &dummy;             // lengths come from text_start / text_cu here
   int32_t rc = validate_kv(&kv, batch, false);
   if (rc != SPECVLM_OK) return rc;
-  if (!q_text || !text_cu || !text_start || !video_start || !video_len || !video_cu || !scores || !ws ||
-      n_q_heads < 1 || !(sm_scale > 0.f) || !aligned16(q_text))
+  if (!q_text || !text_cu || !text_start || n_q_heads < 1 || !(sm_scale > 0.f) || !aligned16(q_text))
     return SPECVLM_ERR_INVALID_ARG;
   if (batch > kScoresMaxBatch) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   if (n_q_heads % kv.n_kv_heads != 0) return SPECVLM_ERR_INVALID_ARG;
   const int group = n_q_heads / kv.n_kv_heads;
   if (group > 16) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
-  if (reinterpret_cast<uintptr_t>(ws) & 255u) return SPECVLM_ERR_INVALID_ARG;
-  if (kv.block_table && kv.block_tokens % 64 != 0) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  if (kv.n_layers > 65535 || kv.n_kv_heads > 65535) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
 
-  ScoreParams p;
+  ScoreParams& p = su.p1;
   p.qt = 128 / group;
-  int n_row_tiles = 0, n_key_blocks = 0;
   int64_t sum_video = 0;
   for (int b = 0; b < batch; ++b) {
     const int nt = text_cu[b + 1] - text_cu[b];
-    if (nt < 1 || video_len[b] < 1 || video_start[b] < 0 || video_start[b] + video_len[b] > text_start[b] ||
-        text_start[b] + nt > kv.max_seq_len || video_cu[b + 1] - video_cu[b] < video_len[b] ||
-        video_cu[b] != sum_video)
-      return SPECVLM_ERR_INVALID_ARG;
-    sum_video += video_len[b];
+    if (nt < 1 || text_start[b] < 0 || text_start[b] + nt > kv.max_seq_len) return SPECVLM_ERR_INVALID_ARG;
+    if (video_len) {
+      if (!video_start || !video_cu || video_len[b] < 1 || video_start[b] < 0 ||
+          video_start[b] + video_len[b] > text_start[b] || video_cu[b] != sum_video)
+        return SPECVLM_ERR_INVALID_ARG;
+      sum_video += video_len[b];
+    }
   }
-  if (video_cu[batch] != sum_video) return SPECVLM_ERR_INVALID_ARG;
-  size_t lse_bytes, partial_bytes;
-  ws_layout(kv.n_layers, kv.n_kv_heads, group, text_cu[batch], sum_video, lse_bytes, partial_bytes);
-  if (ws_bytes < lse_bytes + partial_bytes) return SPECVLM_ERR_WORKSPACE_TOO_SMALL;
-  if (kv.n_layers > 65535 || kv.n_kv_heads > 65535) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  if (video_len && video_cu[batch] != sum_video) return SPECVLM_ERR_INVALID_ARG;
+  if (sum_video > 0x7fffffff) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
 
   p.q = static_cast<const __nv_bfloat16*>(q_text);
-  p.lse2 = static_cast<float*>(ws);
-  p.partial = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + lse_bytes);
+  p.lse = nullptr;
+  p.partial = nullptr;
   p.block_table = kv.block_table;
   p.d_status = d_status;
   p.batch = batch;
@@ -550,69 +535,122 @@ extern "C" int32_t specvlm_stage1_scores(const specvlm_kv_t* target_kv, const vo
   p.max_blocks = kv.max_blocks;
   p.block_tokens = kv.block_tokens;
   p.scale_log2 = sm_scale * kLog2e;
-
-  CUtensorMap tk, tq;
-  rc = encode_kv_map(&tk, &kv, kv.k, 64);
-  if (rc != SPECVLM_OK) return rc;
-  {
-    encode_tiled_fn enc = get_encode_tiled();
-    if (!enc) return SPECVLM_ERR_CUDA;
-    const int D = kv.head_dim;
-    const cuuint64_t dims[5] = {(cuuint64_t)D, (cuuint64_t)group, (cuuint64_t)kv.n_kv_heads,
-                                (cuuint64_t)p.sum_text, (cuuint64_t)kv.n_layers};
-    const cuuint64_t strides[4] = {(cuuint64_t)D * 2, (cuuint64_t)group * D * 2, (cuuint64_t)n_q_heads * D * 2,
-                                   (cuuint64_t)p.sum_text * n_q_heads * D * 2};
-    const cuuint32_t box[5] = {64u, (cuuint32_t)group, 1u, (cuuint32_t)p.qt, 1u};
-    const cuuint32_t estr[5] = {1u, 1u, 1u, 1u, 1u};
-    if (enc(&tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(q_text), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return SPECVLM_ERR_CUDA;
-  }
-
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // pass 1 tiles: row tiles per sequence; pass 2 tiles: key blocks per sequence.  The two passes
-  // use separate tile_off tables, so fill, launch pass 1 ... both passes are launched from
-  // run_scores with one params struct: store pass-1 offsets in seq[].tile_off and pass-2 offsets
-  // in a second struct.
-  ScoreParams p2 = p;
+  su.p2 = p;
+  su.n_row_tiles = su.n_key_blocks = 0;
   for (int b = 0; b < batch; ++b) {
     const int nt = text_cu[b + 1] - text_cu[b];
     ScoreSeq s;
     s.text_off = text_cu[b];
     s.n_text = nt;
     s.text_start = text_start[b];
-    s.video_start = video_start[b];
-    s.n_video = video_len[b];
-    s.score_off = video_cu[b];
-    s.tile_off = n_row_tiles;
-    p.seq[b] = s;
-    s.tile_off = n_key_blocks;
-    p2.seq[b] = s;
-    n_row_tiles += (nt + p.qt - 1) / p.qt;
-    n_key_blocks += (video_start[b] % 64 + video_len[b] + kKeyTile - 1) / kKeyTile;
+    s.video_start = video_len ? video_start[b] : 0;
+    s.n_video = video_len ? video_len[b] : 0;
+    s.score_off = video_len ? video_cu[b] : 0;
+    s.tile_off = su.n_row_tiles;
+    su.p1.seq[b] = s;
+    s.tile_off = su.n_key_blocks;
+    su.p2.seq[b] = s;
+    su.n_row_tiles += (nt + p.qt - 1) / p.qt;
+    su.n_key_blocks += (s.video_start % 64 + s.n_video + kKeyTile - 1) / kKeyTile;
   }
-  // launch (pass 1 with p, pass 2 and the final reduction with p2)
-  auto launch = [&](auto tag) -> int32_t {
-    constexpr int D = decltype(tag)::value;
-    constexpr int STAGES1 = 4, STAGES2 = 3;
-    constexpr int TILE = kKeyTile * D * 2;
-    constexpr int SMEM1 = STAGES1 * TILE + 1024 + 16 * STAGES1 + 16 + 2 * 128 * 2 * 4;
-    constexpr int SMEM2 = (STAGES2 + 1) * TILE + 1024 + 16 * STAGES2 + 16 + 16 + 128 * 4;
-    auto k1 = scores_lse_kernel<D, STAGES1>;
-    auto k2 = scores_colsum_kernel<D, STAGES2>;
-    if (cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM1) != cudaSuccess ||
-        cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2) != cudaSuccess)
-      return SPECVLM_ERR_CUDA;
-    k1<<<dim3((unsigned)n_row_tiles, (unsigned)kv.n_kv_heads, (unsigned)kv.n_layers), 288, SMEM1, st>>>(tk, p);
-    int32_t r = launch_status();
-    if (r != SPECVLM_OK) return r;
-    k2<<<dim3((unsigned)n_key_blocks, (unsigned)kv.n_layers), 288, SMEM2, st>>>(tk, tq, p2);
-    r = launch_status();
-    if (r != SPECVLM_OK) return r;
-    scores_finish_kernel<<<(unsigned)((p2.sum_video + 255) / 256), 256, 0, st>>>(p2, scores);
-    return launch_status();
-  };
-  if (kv.head_dim == 128) return launch(std::integral_constant<int, 128>{});
-  return launch(std::integral_constant<int, 64>{});
+
+  rc = encode_kv_map(&su.tk, &kv, kv.k, 64);
+  if (rc != SPECVLM_OK) return rc;
+  encode_tiled_fn enc = get_encode_tiled();
+  if (!enc) return SPECVLM_ERR_CUDA;
+  const int D = kv.head_dim;
+  const cuuint64_t dims[5] = {(cuuint64_t)D, (cuuint64_t)group, (cuuint64_t)kv.n_kv_heads,
+                              (cuuint64_t)p.sum_text, (cuuint64_t)kv.n_layers};
+  const cuuint64_t strides[4] = {(cuuint64_t)D * 2, (cuuint64_t)group * D * 2, (cuuint64_t)n_q_heads * D * 2,
+                                 (cuuint64_t)p.sum_text * n_q_heads * D * 2};
+  const cuuint32_t box[5] = {64u, (cuuint32_t)group, 1u, (cuuint32_t)p.qt, 1u};
+  const cuuint32_t estr[5] = {1u, 1u, 1u, 1u, 1u};
+  if (enc(&su.tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(q_text), dims, strides, box, estr,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return SPECVLM_ERR_CUDA;
+  return SPECVLM_OK;
+}
+
+template <int D>
+static int32_t launch_lse(ScoreSetup& su, cudaStream_t st) {
+  constexpr int STAGES = 4;
+  constexpr int SMEM = STAGES * kKeyTile * D * 2 + 1024 + 16 * STAGES + 16 + 2 * 128 * 2 * 4;
+  auto k = scores_lse_kernel<D, STAGES>;
+  if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
+    return SPECVLM_ERR_CUDA;
+  k<<<dim3((unsigned)su.n_row_tiles, (unsigned)su.kv.n_kv_heads, (unsigned)su.kv.n_layers), 288, SMEM, st>>>(
+      su.tk, su.p1);
+  return launch_status();
+}
+
+template <int D>
+static int32_t launch_colsum(ScoreSetup& su, float* scores, cudaStream_t st) {
+  constexpr int STAGES = 3;
+  constexpr int SMEM = (STAGES + 1) * kKeyTile * D * 2 + 1024 + 16 * STAGES + 16 + 16 + 128 * 4;
+  auto k = scores_colsum_kernel<D, STAGES>;
+  if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
+    return SPECVLM_ERR_CUDA;
+  k<<<dim3((unsigned)su.n_key_blocks, (unsigned)su.kv.n_layers), 288, SMEM, st>>>(su.tk, su.tq, su.p2);
+  int32_t rc = launch_status();
+  if (rc != SPECVLM_OK) return rc;
+  scores_finish_kernel<<<(unsigned)((su.p2.sum_video + 255) / 256), 256, 0, st>>>(su.p2, scores);
+  return launch_status();
+}
+
+}  // namespace specvlm
+
+using namespace specvlm;
+
+extern "C" size_t specvlm_stage1_scores_workspace_bytes(const specvlm_kv_t* target_kv,
+                                                        const int32_t* text_cu, const int32_t* video_len,
+                                                        int32_t batch, int32_t n_q_heads) {
+  if (!target_kv || !text_cu || !video_len || batch < 1 || n_q_heads < 1) return 0;
+  int64_t sum_video = 0;
+  for (int b = 0; b < batch; ++b) sum_video += video_len[b];
+  size_t a, c;
+  ws_layout(target_kv->n_layers, n_q_heads, text_cu[batch], sum_video, a, c);
+  return a + c;
+}
+
+extern "C" int32_t specvlm_stage1_row_lse(const specvlm_kv_t* target_kv, const void* q_text,
+                                          const int32_t* text_cu, const int32_t* text_start, int32_t batch,
+                                          int32_t n_q_heads, float sm_scale, float* row_lse,
+                                          int32_t* d_status, void* stream) {
+  if (!row_lse) return SPECVLM_ERR_INVALID_ARG;
+  ScoreSetup su;
+  int32_t rc = setup_scores(target_kv, q_text, text_cu, text_start, nullptr, nullptr, nullptr, batch,
+                            n_q_heads, sm_scale, d_status, su);
+  if (rc != SPECVLM_OK) return rc;
+  su.p1.lse = row_lse;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return su.kv.head_dim == 128 ? launch_lse<128>(su, st) : launch_lse<64>(su, st);
+}
+
+extern "C" int32_t specvlm_stage1_scores(const specvlm_kv_t* target_kv, const void* q_text,
+                                         const int32_t* text_cu, const int32_t* text_start,
+                                         const int32_t* video_start, const int32_t* video_len,
+                                         const int32_t* video_cu, int32_t batch, int32_t n_q_heads,
+                                         float sm_scale, const float* row_lse_or_null, float* scores,
+                                         void* ws, size_t ws_bytes, int32_t* d_status, void* stream) {
+  if (!video_start || !video_len || !video_cu || !scores || !ws) return SPECVLM_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(ws) & 255u) return SPECVLM_ERR_INVALID_ARG;
+  ScoreSetup su;
+  int32_t rc = setup_scores(target_kv, q_text, text_cu, text_start, video_start, video_len, video_cu, batch,
+                            n_q_heads, sm_scale, d_status, su);
+  if (rc != SPECVLM_OK) return rc;
+  size_t lse_bytes, partial_bytes;
+  ws_layout(su.kv.n_layers, n_q_heads, su.p1.sum_text, su.p1.sum_video, lse_bytes, partial_bytes);
+  if (ws_bytes < lse_bytes + partial_bytes) return SPECVLM_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const bool d128 = su.kv.head_dim == 128;
+  if (row_lse_or_null) {
+    su.p2.lse = const_cast<float*>(row_lse_or_null);
+  } else {
+    su.p1.lse = su.p2.lse = static_cast<float*>(ws);
+    rc = d128 ? launch_lse<128>(su, st) : launch_lse<64>(su, st);
+    if (rc != SPECVLM_OK) return rc;
+  }
+  su.p2.partial = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + lse_bytes);
+  return d128 ? launch_colsum<128>(su, scores, st) : launch_colsum<64>(su, scores, st);
 }

@@ -46,7 +46,7 @@ _lib = None
 
 EXPORTS = [
     "specvlm_version", "specvlm_status_string",
-    "specvlm_stage1_scores_workspace_bytes", "specvlm_stage1_scores",
+    "specvlm_stage1_scores_workspace_bytes", "specvlm_stage1_row_lse", "specvlm_stage1_scores",
     "specvlm_select", "specvlm_gather_kv",
     "specvlm_attn_workspace_bytes", "specvlm_draft_decode_attn", "specvlm_verify_attn",
     "specvlm_accept_workspace_bytes", "specvlm_accept",
@@ -70,7 +70,11 @@ def lib():
         L.specvlm_stage1_scores_workspace_bytes.argtypes = [kvp, i32p, i32p, c_int32, c_int32]
         L.specvlm_stage1_scores.restype = c_int32
         L.specvlm_stage1_scores.argtypes = [kvp, c_void_p, i32p, i32p, i32p, i32p, i32p, c_int32, c_int32,
-                                            c_float, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]
+                                            c_float, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p,
+                                            c_void_p]
+        L.specvlm_stage1_row_lse.restype = c_int32
+        L.specvlm_stage1_row_lse.argtypes = [kvp, c_void_p, i32p, i32p, c_int32, c_int32, c_float, c_void_p,
+                                             c_void_p, c_void_p]
         L.specvlm_select.restype = c_int32
         L.specvlm_select.argtypes = [c_void_p, i32p, i32p, c_int32, i32p, i32p, i32p, c_int32, c_void_p,
                                      c_void_p, c_void_p]
@@ -213,9 +217,24 @@ def stage1_scores_workspace_bytes(kv: KvCache, text_cu, video_len, n_q_heads: in
                                                            batch, n_q_heads))
 
 
+def stage1_row_lse(kv: KvCache, q_text: torch.Tensor, text_cu, text_start, sm_scale: float,
+                   row_lse: torch.Tensor | None = None, d_status: torch.Tensor | None = None) -> torch.Tensor:
+    """q_text: bf16 [n_layers][sum_text][n_q_heads][head_dim]; returns fp32 [n_layers][sum_text][n_q_heads]."""
+    L, n_text_all, Hq, D = q_text.shape
+    assert q_text.is_contiguous() and q_text.dtype == torch.bfloat16 and n_text_all == text_cu[-1]
+    if row_lse is None:
+        row_lse = torch.empty((L, n_text_all, Hq), dtype=torch.float32, device=q_text.device)
+    rc = lib().specvlm_stage1_row_lse(byref(kv.struct), _ptr(q_text), _i32(text_cu), _i32(text_start),
+                                      len(text_start), Hq, float(sm_scale), _ptr(row_lse), _ptr(d_status),
+                                      _stream())
+    _check(rc, "specvlm_stage1_row_lse")
+    return row_lse
+
+
 def stage1_scores(kv: KvCache, q_text: torch.Tensor, text_cu, text_start, video_start, video_len,
                   video_cu, sm_scale: float, scores: torch.Tensor | None = None,
-                  ws: torch.Tensor | None = None, d_status: torch.Tensor | None = None) -> torch.Tensor:
+                  ws: torch.Tensor | None = None, d_status: torch.Tensor | None = None,
+                  row_lse: torch.Tensor | None = None) -> torch.Tensor:
     """q_text: bf16 [n_layers][sum_text][n_q_heads][head_dim]; returns fp32 [sum_video]."""
     L, n_text_all, Hq, D = q_text.shape
     batch = len(video_len)
@@ -226,8 +245,8 @@ def stage1_scores(kv: KvCache, q_text: torch.Tensor, text_cu, text_start, video_
         ws = _ws(stage1_scores_workspace_bytes(kv, text_cu, video_len, Hq), q_text.device)
     rc = lib().specvlm_stage1_scores(byref(kv.struct), _ptr(q_text), _i32(text_cu), _i32(text_start),
                                      _i32(video_start), _i32(video_len), _i32(video_cu), batch, Hq,
-                                     float(sm_scale), _ptr(scores), _ptr(ws), ws.numel(), _ptr(d_status),
-                                     _stream())
+                                     float(sm_scale), _ptr(row_lse), _ptr(scores), _ptr(ws), ws.numel(),
+                                     _ptr(d_status), _stream())
     _check(rc, "specvlm_stage1_scores")
     return scores
 

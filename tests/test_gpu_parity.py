@@ -350,3 +350,17 @@ def test_pipeline_cfg1_end_to_end():
     assert inter >= 0.9 * kt, f"GPU-score selection overlaps the oracle's in {inter}/{kt}"
     # planted tokens should be over-represented in Stage I (sanity statistic, not a gate)
     assert len(kept_ref) == kt
+
+
+def test_scores_row_lse_entry():
+    from gpu_util import make_cache
+    L, Hq, Hkv, D, nv, nt = 2, 28, 4, 128, 200, 45
+    cache, k_host, _ = make_cache(L, Hkv, D, [nv + nt], paged=True, seed=21)
+    q = synth.randn_bf16((L, nt, Hq, D), "cuda", 21, "Qtext")
+    scale = 1.0 / math.sqrt(D)
+    lse = specvlm.stage1_row_lse(cache, q, [0, nt], [nv], scale)
+    _, _, ref_lse = oracle.stage1_scores(bits(q), k_host[0], 0, nv, nv, scale, want_rows=True)
+    np.testing.assert_allclose(lse.cpu().numpy(), ref_lse.transpose(0, 2, 1), rtol=0, atol=1e-4)
+    a = specvlm.stage1_scores(cache, q, [0, nt], [nv], [0], [nv], [0, nv], scale)
+    b = specvlm.stage1_scores(cache, q, [0, nt], [nv], [0], [nv], [0, nv], scale, row_lse=lse)
+    assert torch.equal(a, b)
