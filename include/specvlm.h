@@ -41,7 +41,8 @@ typedef enum specvlm_status {
   SPECVLM_ERR_UNSUPPORTED_SHAPE = -2, /* a shape outside the documented supported set          */
   SPECVLM_ERR_WORKSPACE_TOO_SMALL = -3,
   SPECVLM_ERR_CUDA = -4,              /* a CUDA runtime / driver call failed                   */
-  SPECVLM_ERR_TIMEOUT = -5            /* device-side bounded wait expired (via d_status only)  */
+  SPECVLM_ERR_TIMEOUT = -5,           /* device-side bounded wait expired (via d_status only)  */
+  SPECVLM_ERR_TOO_LARGE = -6          /* problem exceeds the fixed capacity of a no-allocation call */
 } specvlm_status;
 
 /*
@@ -192,6 +193,33 @@ size_t specvlm_accept_workspace_bytes(int32_t batch, int32_t gamma, int32_t voca
 int32_t specvlm_accept(const float* target_logits, const int32_t* draft_tokens, int32_t batch,
                        int32_t gamma, int32_t vocab, int32_t* accept_len, int32_t* next_token,
                        int32_t* target_argmax_or_null, void* ws, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * specvlm_accept without any caller-provided scratch.  (The paper has no counterpart: this is a
+ * packaging variant of step 4c, same results.)
+ *
+ * For callers that cannot allocate device memory at the point of the call and have no workspace
+ * to hand over: code running inside another framework's pre-planned memory arena, a latency-
+ * critical serving loop that forbids cudaMalloc (it synchronises the device), or a plug-in that
+ * only receives input and output buffers.  The per-(row, vocabulary-chunk) candidates live in a
+ * fixed array inside the library (128 KB of device memory on every GPU that loads the library,
+ * held until the process exits) instead of `ws`.
+ *
+ * Arguments and results are those of specvlm_accept, minus ws / ws_bytes.
+ * Limit: batch * (gamma+1) * ceil(vocab / 4096) <= 16384 candidates (e.g. batch 16, gamma 8,
+ * vocab 152064 needs 5472); larger problems return SPECVLM_ERR_TOO_LARGE and launch nothing.
+ * The call allocates and frees nothing, on the host side or the device side.
+ * The first call on each device looks up the device address of that device's copy of the array
+ * (a cheap runtime query, cached afterwards); make that first call with the device current and
+ * before starting any stream capture.
+ * All calls on a device share the one array: two calls whose kernels may overlap on the GPU
+ * (different streams without an ordering between them) race on it and give wrong results.
+ * Calls ordered on one stream are safe; nothing needs clearing between calls, because each call
+ * overwrites every slot it later reads.
+ */
+int32_t specvlm_accept_noalloc(const float* target_logits, const int32_t* draft_tokens, int32_t batch,
+                               int32_t gamma, int32_t vocab, int32_t* accept_len,
+                               int32_t* next_token, int32_t* target_argmax_or_null, void* stream);
 
 #ifdef __cplusplus
 }

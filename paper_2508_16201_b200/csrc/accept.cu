@@ -1,6 +1,8 @@
 // Step 4c: greedy acceptance.  Kernel 1 streams the fp32 logits once (16-byte loads) and leaves
 // one (max, lowest index) candidate per (row, vocab chunk); kernel 2 finishes the argmax of the
 // gamma+1 rows of a sequence and counts the leading draft tokens that equal it.
+#include <mutex>
+
 #include "common.cuh"
 #include "host_util.h"
 
@@ -95,6 +97,11 @@ __global__ void accept_finish_kernel(const Cand* __restrict__ part, int n_chunks
   }
 }
 
+// Built-in scratch of specvlm_accept_noalloc: room for kStaticCands (row, vocab chunk) candidates.
+// Every GPU that loads the library holds these 128 KB until the process exits.
+constexpr int kStaticCands = 16384;
+static __device__ __align__(256) Cand g_accept_scratch[kStaticCands];
+
 }  // namespace specvlm
 
 using namespace specvlm;
@@ -120,6 +127,48 @@ extern "C" int32_t specvlm_accept(const float* target_logits, const int32_t* dra
   const int n_chunks = (vocab + kAcceptChunk - 1) / kAcceptChunk;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   Cand* part = static_cast<Cand*>(ws);
+  accept_partial_kernel<<<dim3((unsigned)n_chunks, (unsigned)(batch * (gamma + 1))), kAcceptThreads, 0, st>>>(
+      target_logits, vocab, n_chunks, part);
+  int32_t rc = launch_status();
+  if (rc != SPECVLM_OK) return rc;
+  accept_finish_kernel<<<(unsigned)batch, 32 * (gamma + 1), 0, st>>>(part, n_chunks, draft_tokens, gamma,
+                                                                     accept_len, next_token,
+                                                                     target_argmax_or_null);
+  return launch_status();
+}
+
+extern "C" int32_t specvlm_accept_noalloc(const float* target_logits, const int32_t* draft_tokens,
+                                          int32_t batch, int32_t gamma, int32_t vocab, int32_t* accept_len,
+                                          int32_t* next_token, int32_t* target_argmax_or_null, void* stream) {
+  if (!target_logits || !accept_len || !next_token || batch < 1 || gamma < 0 || vocab < 1)
+    return SPECVLM_ERR_INVALID_ARG;
+  if (gamma > 0 && !draft_tokens) return SPECVLM_ERR_INVALID_ARG;
+  if (gamma > 15) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  if ((int64_t)batch * (gamma + 1) > 65535) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  if (reinterpret_cast<uintptr_t>(target_logits) & 3u) return SPECVLM_ERR_INVALID_ARG;
+  const int n_chunks = (vocab + kAcceptChunk - 1) / kAcceptChunk;
+  if ((int64_t)batch * (gamma + 1) * n_chunks > kStaticCands) return SPECVLM_ERR_TOO_LARGE;
+
+  // Set-up, once per device: in host code the array's name is only a handle, the kernels need
+  // the device address of this device's copy.
+  constexpr int kMaxDevices = 64;
+  static Cand* scratch_of[kMaxDevices] = {};
+  static std::mutex mu;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SPECVLM_ERR_CUDA;
+  Cand* part;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (!scratch_of[dev]) {
+      void* addr = nullptr;
+      if (cudaGetSymbolAddress(&addr, g_accept_scratch) != cudaSuccess || !addr) return SPECVLM_ERR_CUDA;
+      scratch_of[dev] = static_cast<Cand*>(addr);
+    }
+    part = scratch_of[dev];
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // every candidate slot that kernel 2 reads is written by kernel 1 of the same call first, so
+  // nothing left over from an earlier call has to be cleared
   accept_partial_kernel<<<dim3((unsigned)n_chunks, (unsigned)(batch * (gamma + 1))), kAcceptThreads, 0, st>>>(
       target_logits, vocab, n_chunks, part);
   int32_t rc = launch_status();

@@ -11,6 +11,7 @@ extern "C" const char* specvlm_status_string(int32_t status) {
     case SPECVLM_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
     case SPECVLM_ERR_CUDA: return "CUDA call failed";
     case SPECVLM_ERR_TIMEOUT: return "device-side wait timed out";
+    case SPECVLM_ERR_TOO_LARGE: return "problem exceeds the built-in scratch of a no-allocation call";
     default: return "unknown status";
   }
 }

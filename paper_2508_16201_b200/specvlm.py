@@ -21,6 +21,7 @@ ERR_UNSUPPORTED_SHAPE = -2
 ERR_WORKSPACE_TOO_SMALL = -3
 ERR_CUDA = -4
 ERR_TIMEOUT = -5
+ERR_TOO_LARGE = -6
 
 
 class SpecvlmError(RuntimeError):
@@ -49,7 +50,7 @@ EXPORTS = [
     "specvlm_stage1_scores_workspace_bytes", "specvlm_stage1_row_lse", "specvlm_stage1_scores",
     "specvlm_select", "specvlm_gather_kv",
     "specvlm_attn_workspace_bytes", "specvlm_draft_decode_attn", "specvlm_verify_attn",
-    "specvlm_accept_workspace_bytes", "specvlm_accept",
+    "specvlm_accept_workspace_bytes", "specvlm_accept", "specvlm_accept_noalloc",
 ]
 
 
@@ -94,6 +95,9 @@ def lib():
         L.specvlm_accept.restype = c_int32
         L.specvlm_accept.argtypes = [c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p,
                                      c_void_p, c_void_p, c_size_t, c_void_p]
+        L.specvlm_accept_noalloc.restype = c_int32
+        L.specvlm_accept_noalloc.argtypes = [c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p,
+                                             c_void_p, c_void_p]
         _lib = L
     return _lib
 
@@ -302,3 +306,18 @@ def accept(target_logits: torch.Tensor, draft_tokens: torch.Tensor, want_argmax:
                               _ptr(next_token), _ptr(g), _ptr(ws), ws.numel(), _stream())
     _check(rc, "specvlm_accept")
     return accept_len, next_token, g
+
+
+def accept_noalloc(target_logits: torch.Tensor, draft_tokens: torch.Tensor, out, want_argmax_into=None):
+    """specvlm_accept_noalloc: like ``accept`` but the library's built-in scratch is used, and this
+    wrapper allocates nothing either: ``out`` = (accept_len, next_token) int32 [B] tensors made by
+    the caller beforehand; ``want_argmax_into`` an optional int32 [B][gamma+1] tensor.
+    Raises SpecvlmError(ERR_TOO_LARGE) beyond the built-in capacity."""
+    B, G1, V = target_logits.shape
+    assert target_logits.dtype == torch.float32 and target_logits.is_contiguous()
+    assert draft_tokens.dtype == torch.int32 and draft_tokens.is_contiguous()
+    accept_len, next_token = out
+    rc = lib().specvlm_accept_noalloc(_ptr(target_logits), _ptr(draft_tokens), B, G1 - 1, V, _ptr(accept_len),
+                                      _ptr(next_token), _ptr(want_argmax_into), _stream())
+    _check(rc, "specvlm_accept_noalloc")
+    return accept_len, next_token
