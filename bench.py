@@ -488,8 +488,67 @@ def run_reference(args, rank):
         "gpu_launches": 0}))
 
 
+def run_case(args):
+    """One call of the path on a reduced number of layers (a small case for `ncu`, or a sweep):
+    prints the median device time of `--iters` launches.  Not the benchmark line."""
+    import dataclasses
+    import torch
+    from paper_2508_16201_b200 import specvlm, synth
+    w = synth.workload(args.workload, gamma=args.gamma)
+    if args.layers:
+        w = dataclasses.replace(w, t_layers=args.layers, d_layers=args.layers)
+    if args.frames:
+        w = dataclasses.replace(w, n_frames=(args.frames,))
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    inp = build_inputs(w, device, n_copies=1)
+    path = Path(w, inp, device)
+    path.row_lse_call(); path.scores_call(); path.select_call()
+    for c in inp["dpruned"]:
+        path.gather_call(c)
+    D, nv, nt, gamma = w.head_dim, w.n_video(), w.n_text[0], w.gamma
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=device)
+    dsrc = inp["dsrc"]
+    ws_u = torch.empty(max(256, specvlm.attn_workspace_bytes(dsrc, 1, w.d_q_heads, 0)), dtype=torch.uint8,
+                       device=device)
+    calls = {
+        "verify": (path.verify_call, 2 * (nv + nt + gamma + 1) * w.t_kv_heads * D * 2 * w.t_layers),
+        "decode": (lambda: path.decode_call(0, inp["dpruned"][1]), 2 * (w.k_total() + nt) * w.d_kv_heads * D * 2 * w.d_layers),
+        "decode_unpruned": (lambda: specvlm.draft_decode_attn(dsrc, inp["q_dec"][0], path.scale, out=path.o_dec[0], ws=ws_u),
+                            2 * (nv + nt) * w.d_kv_heads * D * 2 * w.d_layers),
+        "row_lse": (path.row_lse_call, 0), "scores": (path.scores_call, 0), "select": (path.select_call, 0),
+        "gather": (lambda: path.gather_call(inp["dpruned"][0]), 4 * (w.k_total() + nt) * w.d_kv_heads * D * 2 * w.d_layers),
+        "accept": (path.accept_call, (gamma + 1) * w.vocab * 4),
+    }
+    fn, nbytes = calls[args.case]
+    ts = []
+    for i in range(args.warmup + args.iters):
+        if args.flush:
+            flush.zero_()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        torch.cuda.synchronize()
+        if i >= args.warmup:
+            ts.append(a.elapsed_time(b))
+    assert int(path.status.item()) == 0
+    med = statistics.median(ts)
+    print(json.dumps({"case": args.case, "workload": w.name, "layers": args.layers, "gamma": gamma,
+                      "median_us": round(med * 1e3, 2), "min_us": round(min(ts) * 1e3, 2),
+                      "gbs": round(nbytes / (med * 1e-3) / 1e9, 1) if nbytes else None,
+                      "env": {k: v for k, v in os.environ.items() if k.startswith("SPECVLM_")}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--case", default=None, help="run one call only (small case for profiling / sweeps)")
+    ap.add_argument("--layers", type=int, default=0)
+    ap.add_argument("--frames", type=int, default=0)
+    ap.add_argument("--workload", type=int, default=2)
+    ap.add_argument("--gamma", type=int, default=None)
+    ap.add_argument("--iters", type=int, default=10)
+    ap.add_argument("--flush", action="store_true", help="write a 512 MB buffer before each launch")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
@@ -498,6 +557,9 @@ def main():
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
+    if args.case:
+        run_case(args)
+        return
     if args.impl == "reference":
         run_reference(args, rank)
         return

@@ -12,6 +12,30 @@
 
 namespace specvlm {
 
+// Issues the bulk tensor copies of tile `tg` (64 tokens of K and of V) of sequence b into one
+// pipeline stage; completion is counted on `full`.
+template <int D>
+__device__ __forceinline__ void issue_kv_tile(const CUtensorMap* tm_k, const CUtensorMap* tm_v,
+                                              const AttnParams& p, int b, int g, int layer, int tg,
+                                              uint32_t dst, uint32_t full, uint64_t policy) {
+  constexpr int TILE_BYTES = kTileTokens * D * 2;
+  int blk, tok;
+  if (p.block_table) {
+    const int tiles_per_block = p.block_tokens / kTileTokens;
+    blk = p.block_table[(size_t)b * p.max_blocks + tg / tiles_per_block];
+    tok = (tg % tiles_per_block) * kTileTokens;
+  } else {
+    blk = b;
+    tok = tg * kTileTokens;
+  }
+  mbar_arrive_expect_tx(full, 2 * TILE_BYTES);
+#pragma unroll
+  for (int h = 0; h < D / 64; ++h) {
+    tma_load_5d(dst + h * (kTileTokens * 128), tm_k, full, h * 64, tok, g, blk, layer, policy);
+    tma_load_5d(dst + TILE_BYTES + h * (kTileTokens * 128), tm_v, full, h * 64, tok, g, blk, layer, policy);
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Kernel A: up to 16 query rows per KV head (decode: the group's heads; small verify windows).
 // 4 consumer warps each own 16 of a tile's 64 tokens and keep private running (max, sum, O);
@@ -294,7 +318,7 @@ attn_rows16_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 // from shared memory once per group.  The last warp is the TMA producer.
 // ---------------------------------------------------------------------------------------------
 template <int D, int MT, int NG, int STAGES, int MINB>
-__global__ void __launch_bounds__(32 * (4 * NG + 1), MINB)
+__global__ void __launch_bounds__(NG == 1 ? 128 : 32 * (4 * NG + 1), MINB)
 attn_rowsN_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                   const AttnParams p) {
   constexpr int TILE_BYTES = kTileTokens * D * 2;
@@ -336,37 +360,36 @@ attn_rowsN_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   }
   __syncthreads();
 
-  if (warp == 4 * NG) {
+  // NG == 1: no producer warp (4 warps per CTA keep the full register budget at 2 CTAs per SM);
+  // thread 0 refills a stage right after the first group barrier of the next tile, by which
+  // time every warp has finished reading it.  NG == 2: a dedicated producer warp and empty
+  // barriers, because the two groups only synchronise within themselves.
+  constexpr bool kInline = NG == 1;
+  uint64_t policy = 0;
+  if (kInline) {
+    if (tid == 0 && n_my > 0) {
+      tma_prefetch_desc(&tm_k);
+      tma_prefetch_desc(&tm_v);
+      policy = l2_policy_evict_first();
+      const int pre = n_my < STAGES ? n_my : STAGES;
+      for (int i = 0; i < pre; ++i)
+        issue_kv_tile<D>(&tm_k, &tm_v, p, b, g, layer, tile_begin + i, base + i * STAGE_BYTES,
+                         bar_full + 8 * i, policy);
+    }
+  } else if (warp == 4 * NG) {
     // ------------------------------------------------------------------ producer
     if (lane == 0 && n_my > 0) {
       tma_prefetch_desc(&tm_k);
       tma_prefetch_desc(&tm_v);
-      const uint64_t policy = l2_policy_evict_first();
-      const int tiles_per_block = p.block_tokens / kTileTokens;
+      policy = l2_policy_evict_first();
       int issued = 0;
       bool ok = true;
       for (int i = 0; i < n_my && ok; ++i) {
         const int s = i % STAGES;
         if (i >= STAGES) ok = mbar_wait(bar_empty + 8 * s, ((i / STAGES) - 1) & 1, abort_flag);
         if (!ok) break;
-        const int tg = tile_begin + i;
-        int blk, tok;
-        if (p.block_table) {
-          blk = p.block_table[(size_t)b * p.max_blocks + tg / tiles_per_block];
-          tok = (tg % tiles_per_block) * kTileTokens;
-        } else {
-          blk = b;
-          tok = tg * kTileTokens;
-        }
-        const uint32_t full = bar_full + 8 * s;
-        mbar_arrive_expect_tx(full, STAGE_BYTES);
-        const uint32_t dst = base + s * STAGE_BYTES;
-#pragma unroll
-        for (int h = 0; h < D / 64; ++h) {
-          tma_load_5d(dst + h * (kTileTokens * 128), &tm_k, full, h * 64, tok, g, blk, layer, policy);
-          tma_load_5d(dst + TILE_BYTES + h * (kTileTokens * 128), &tm_v, full, h * 64, tok, g, blk,
-                      layer, policy);
-        }
+        issue_kv_tile<D>(&tm_k, &tm_v, p, b, g, layer, tile_begin + i, base + s * STAGE_BYTES,
+                         bar_full + 8 * s, policy);
         issued = i + 1;
       }
       if (!ok) {
@@ -487,6 +510,12 @@ attn_rowsN_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
       }
     }
     asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+    if (kInline && tid == 0 && alive && i >= 1 && i - 1 + STAGES < n_my) {
+      // every warp is past its last read of the previous tile's stage: refill it
+      const int nxt = i - 1 + STAGES;
+      issue_kv_tile<D>(&tm_k, &tm_v, p, b, g, layer, tile_begin + nxt, base + ((i - 1) % STAGES) * STAGE_BYTES,
+                       bar_full + 8 * ((i - 1) % STAGES), policy);
+    }
     // tile maxima, probabilities -> shared memory (bf16), rescale the accumulators
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
@@ -536,7 +565,7 @@ attn_rowsN_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
       }
     }
     __syncwarp();
-    if (lane == 0 && alive) mbar_arrive(bar_empty + 8 * s);
+    if (!kInline && lane == 0 && alive) mbar_arrive(bar_empty + 8 * s);
   }
 
   // ------------------------------------------------------------ row sums across the group's warps
@@ -553,6 +582,14 @@ attn_rowsN_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
   if (!alive || *abort_flag) {
     if (p.d_status && (tid & 127) == 0) *p.d_status = SPECVLM_ERR_TIMEOUT;
+    if (kInline && tid == 0) {
+      // stay until the copies this thread issued have landed (bounded)
+      const uint64_t t0 = global_timer_ns();
+      for (int i = n_my > STAGES ? n_my - STAGES : 0; i < n_my; ++i)
+        while (!mbar_try_wait(bar_full + 8 * (i % STAGES), (i / STAGES) & 1) &&
+               global_timer_ns() - t0 < kWaitLimitNs) {
+        }
+    }
     return;
   }
   const int item = lb * p.n_kv_heads + g;
@@ -632,29 +669,38 @@ static int env_int(const char* name, int dflt) {
   return s && *s ? atoi(s) : dflt;
 }
 
-// How many CTAs share one (layer, sequence, KV head): enough to fill the GPU a few times over,
-// never less than 4 tiles per CTA, at most 64.
-static int choose_splits(int max_seq_len, int64_t items) {
-  const int forced = env_int("SPECVLM_ATTN_SPLITS", 0);
+// How many CTAs share one (layer, sequence, KV head).  All CTAs of a launch stream the same number
+// of tiles, so the launch takes ceil(CTAs / resident slots) rounds of (tiles per CTA + a fixed
+// start-up/epilogue cost of about two tiles); pick the split count that minimises that product.
+static int choose_splits(int max_seq_len, int64_t items, int rows) {
   const int n_tiles = (max_seq_len + kTileTokens - 1) / kTileTokens;
-  int s;
+  const int forced = env_int("SPECVLM_ATTN_SPLITS", 0);
+  int best = 1;
   if (forced > 0) {
-    s = forced;
+    best = forced;
   } else {
-    const int64_t target_ctas = (int64_t)sm_count() * 2 * 4;
-    s = (int)((target_ctas + items - 1) / items);
-    const int by_len = (n_tiles + 3) / 4;
-    if (s > by_len) s = by_len;
+    const int64_t slots = (int64_t)sm_count() * (rows > 48 ? 1 : 2);
+    double best_cost = 1e300;
+    for (int s = 1; s <= 64 && s <= n_tiles; ++s) {
+      const int per = (n_tiles + s - 1) / s;
+      if ((s - 1) * per >= n_tiles) continue;            // would leave an empty split
+      const double rounds = (double)((items * s + slots - 1) / slots);
+      const double cost = rounds * (per + 2.0) + (s > 1 ? 0.5 : 0.0);
+      if (cost < best_cost - 1e-9) {
+        best_cost = cost;
+        best = s;
+      }
+    }
   }
-  if (s > 64) s = 64;
-  if (s > n_tiles) s = n_tiles;
-  if (s < 1) s = 1;
-  return s;
+  if (best > 64) best = 64;
+  if (best > n_tiles) best = n_tiles;
+  if (best < 1) best = 1;
+  return best;
 }
 
 static size_t attn_ws_bytes(const specvlm_kv_t* kv, int32_t batch, int rows) {
   const int64_t items = (int64_t)kv->n_layers * batch * kv->n_kv_heads;
-  const int splits = choose_splits(kv->max_seq_len, items);
+  const int splits = choose_splits(kv->max_seq_len, items, rows);
   if (splits == 1) return 256;
   const size_t o = round_up((size_t)items * splits * rows * kv->head_dim * sizeof(float), 256);
   const size_t l = round_up((size_t)items * splits * rows * sizeof(float), 256);
@@ -683,7 +729,7 @@ static int32_t launch_rowsN(const CUtensorMap& tk, const CUtensorMap& tv, const 
   auto kern = attn_rowsN_kernel<D, MT, NG, STAGES, MINB>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
     return SPECVLM_ERR_CUDA;
-  kern<<<grid, 32 * (4 * NG + 1), SMEM, st>>>(tk, tv, p);
+  kern<<<grid, NG == 1 ? 128 : 32 * (4 * NG + 1), SMEM, st>>>(tk, tv, p);
   return launch_status();
 }
 
@@ -713,7 +759,7 @@ static int32_t attn_common(const specvlm_kv_t* kv, const void* q, int32_t batch,
   if (lb64 > 65535 * 64 || kv->n_kv_heads > 65535) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
 
   const int64_t items = lb64 * kv->n_kv_heads;
-  const int splits = choose_splits(kv->max_seq_len, items);
+  const int splits = choose_splits(kv->max_seq_len, items, rows);
   const size_t need = attn_ws_bytes(kv, batch, rows);
   if (splits > 1) {
     if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) return SPECVLM_ERR_INVALID_ARG;
