@@ -460,6 +460,223 @@ scores_colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Pass 2 on the 5th-generation tensor cores.  CTA = (block of 128 video keys, layer), looping over
+// the layer's KV heads and the sequence's row tiles as above, but
+//   D[key][row] = K_block (A: 128 keys x d, K-major) * Q_tile^T (B: 128 rows x d, K-major)
+// is one chain of tcgen05.mma instructions (M = N = 128, K = 16 each) issued by a single thread,
+// with both operands read straight from the 128-byte-swizzled tiles the TMA wrote and the fp32
+// accumulator in tensor memory (two 128-column buffers, so the next tile's MMAs overlap this
+// tile's epilogue).  With the keys on the TMEM lanes, an epilogue thread owns one key: it reads
+// its 128 row values with tcgen05.ld and adds up 2^(s - lse_row) in a single register for the
+// whole layer -- the column sum needs no cross-thread reduction at all.
+// Warps: 0 = TMA producer, 1 = TMEM allocation + MMA issue, 2..5 = epilogue (one TMEM lane
+// quadrant each).
+// ---------------------------------------------------------------------------------------------
+template <int D, int STAGES>
+__global__ void __launch_bounds__(192, 1)
+scores_colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
+                        const __grid_constant__ ScoreParams p) {
+  constexpr int TILE_BYTES = kKeyTile * D * 2;
+  constexpr int KSTEPS = D / 16;
+  constexpr uint32_t kTmemCols = 256;
+  constexpr uint32_t kIdesc = umma_idesc_bf16(128, 128, false, false);
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t base = (raw_addr + 1023u) & ~1023u;
+  uint8_t* const smem = smem_raw + (base - raw_addr);
+  const uint32_t k_sm = base;                                    // 2 K-block buffers
+  const uint32_t q_sm = base + 2 * TILE_BYTES;                   // Q ring
+  constexpr int kTail = (2 + STAGES) * TILE_BYTES;
+  const uint32_t bar_qfull = base + kTail;
+  const uint32_t bar_qempty = bar_qfull + 8 * STAGES;
+  const uint32_t bar_kfull = bar_qempty + 8 * STAGES;            // [2]
+  const uint32_t bar_kempty = bar_kfull + 16;                    // [2]
+  const uint32_t bar_tfull = bar_kempty + 16;                    // [2]
+  const uint32_t bar_tempty = bar_tfull + 16;                    // [2]
+  uint8_t* const tail = smem + kTail + 16 * STAGES + 64;
+  volatile int* const abort_flag = reinterpret_cast<volatile int*>(tail);
+  volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(tail + 8);
+  float* const lse_sm = reinterpret_cast<float*>(tail + 16);     // [2][128], log2 units
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int b = find_seq(p, blockIdx.x);
+  const ScoreSeq sq = p.seq[b];
+  const int kblock = blockIdx.x - sq.tile_off;
+  const int layer = blockIdx.y;
+  const int key0 = (sq.video_start / 64) * 64 + kblock * kKeyTile;
+  const int n_qt = (sq.n_text + p.qt - 1) / p.qt;
+  const int n_units = p.n_kv_heads;
+  const int n_tiles = n_units * n_qt;
+
+  if (tid == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(bar_qfull + 8 * s, 1);
+      mbar_init(bar_qempty + 8 * s, 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar_kfull + 8 * i, 1);
+      mbar_init(bar_kempty + 8 * i, 1);
+      mbar_init(bar_tfull + 8 * i, 1);
+      mbar_init(bar_tempty + 8 * i, 4);
+    }
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      tma_prefetch_desc(&tm_k);
+      tma_prefetch_desc(&tm_q);
+      const uint64_t pol_k = l2_policy_evict_first();
+      const uint64_t pol_q = l2_policy_evict_last();             // Q is re-read by every key block
+      const uint32_t q_tx = (D / 64) * p.qt * p.group * 128;     // bytes of one Q box set
+      bool ok = true;
+      int qi = 0;
+      for (int u = 0; u < n_units && ok; ++u) {
+        const int kb = u & 1;
+        if (u >= 2) ok = mbar_wait(bar_kempty + 8 * kb, ((u >> 1) - 1) & 1, abort_flag);
+        if (!ok) break;
+        mbar_arrive_expect_tx(bar_kfull + 8 * kb, TILE_BYTES);
+        load_key_tile<D>(&tm_k, p, b, u, layer, key0, k_sm + kb * TILE_BYTES, bar_kfull + 8 * kb, pol_k);
+        for (int t = 0; t < n_qt && ok; ++t, ++qi) {
+          const int s = qi % STAGES;
+          if (qi >= STAGES) ok = mbar_wait(bar_qempty + 8 * s, ((qi / STAGES) - 1) & 1, abort_flag);
+          if (!ok) break;
+          mbar_arrive_expect_tx(bar_qfull + 8 * s, q_tx);
+#pragma unroll
+          for (int h = 0; h < D / 64; ++h)
+            tma_load_5d(q_sm + s * TILE_BYTES + h * (kKeyTile * 128), &tm_q, bar_qfull + 8 * s, h * 64, 0, u,
+                        sq.text_off + t * p.qt, layer, pol_q);
+        }
+      }
+      if (!ok) {
+        if (p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
+        const uint64_t t0 = global_timer_ns();
+        for (int i = qi > STAGES ? qi - STAGES : 0; i < qi; ++i)
+          while (!mbar_try_wait(bar_qfull + 8 * (i % STAGES), (i / STAGES) & 1) &&
+                 global_timer_ns() - t0 < kWaitLimitNs) {
+          }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issue (one thread)
+    if (lane == 0) {
+      bool ok = true;
+      int it = 0;
+      for (int u = 0; u < n_units && ok; ++u) {
+        const int kb = u & 1;
+        ok = mbar_wait(bar_kfull + 8 * kb, (u >> 1) & 1, abort_flag);
+        for (int t = 0; t < n_qt && ok; ++t, ++it) {
+          const int s = it % STAGES, buf = it & 1;
+          ok = mbar_wait(bar_qfull + 8 * s, (it / STAGES) & 1, abort_flag);
+          if (ok && it >= 2) ok = mbar_wait(bar_tempty + 8 * buf, ((it >> 1) - 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const uint32_t a0 = k_sm + kb * TILE_BYTES, b0 = q_sm + s * TILE_BYTES;
+#pragma unroll
+          for (int ks = 0; ks < KSTEPS; ++ks) {
+            // 16 channels per step: 32 bytes along the swizzled 128-byte row; channels 64.. live
+            // in the second half-tile
+            const uint32_t off = (ks >> 2) * (kKeyTile * 128) + (ks & 3) * 32;
+            umma_bf16_ss(tmem_base + buf * 128, umma_desc_sw128(a0 + off, 16, 1024),
+                         umma_desc_sw128(b0 + off, 16, 1024), kIdesc, ks > 0 ? 1u : 0u);
+          }
+          umma_commit(bar_qempty + 8 * s);      // the Q stage is free once these MMAs have read it
+          umma_commit(bar_tfull + 8 * buf);     // and the accumulator buffer is complete
+        }
+        if (ok) umma_commit(bar_kempty + 8 * kb);
+      }
+      if (!ok && p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue: 4 warps, 128 keys
+    const int quad = warp & 3;                  // TMEM lanes [32 * quad, 32 * quad + 32)
+    const int key_l = quad * 32 + lane;         // this thread's key inside the block
+    const int et = (warp - 2) * 32 + lane;      // 0..127: used to stage the row LSEs
+    float acc = 0.f;
+    bool alive = true;
+    int it = 0;
+    for (int u = 0; u < n_units; ++u) {
+      const float* lse_u = p.lse + ((size_t)layer * p.sum_text + sq.text_off) * p.n_q_heads + u * p.group;
+      for (int t = 0; t < n_qt; ++t, ++it) {
+        const int buf = it & 1;
+        const int rows_valid = min(p.qt, sq.n_text - t * p.qt) * p.group;
+        {
+          float v = 0.f;
+          if (et < rows_valid) {
+            const int il = et / p.group, hg = et - il * p.group;
+            v = __ldg(lse_u + (size_t)(t * p.qt + il) * p.n_q_heads + hg) * kLog2e;
+          }
+          lse_sm[buf * 128 + et] = v;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (alive && !mbar_wait(bar_tfull + 8 * buf, (it >> 1) & 1, abort_flag)) alive = false;
+        alive = __all_sync(0xffffffffu, alive); // warp-uniform: the TMEM loads below are warp-collective
+        if (!alive) continue;                   // keep taking part in the barrier above
+        tc_fence_after_sync();
+        const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * 128;
+        uint32_t v0[32], v1[32], v2[32], v3[32];
+        tmem_ld_x32(taddr, v0);
+        tmem_ld_x32(taddr + 32, v1);
+        tmem_ld_x32(taddr + 64, v2);
+        tmem_ld_x32(taddr + 96, v3);
+        tmem_ld_wait();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);   // buffer free for the MMAs of tile it+2
+        const float* ls = lse_sm + buf * 128;
+        if (rows_valid == 128) {
+          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;    // four chains for instruction-level parallelism
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            const float4 l0 = *reinterpret_cast<const float4*>(ls + j);
+            const float4 l1 = *reinterpret_cast<const float4*>(ls + 32 + j);
+            const float4 l2 = *reinterpret_cast<const float4*>(ls + 64 + j);
+            const float4 l3 = *reinterpret_cast<const float4*>(ls + 96 + j);
+            a0 += fast_exp2(__uint_as_float(v0[j]) * p.scale_log2 - l0.x) + fast_exp2(__uint_as_float(v0[j + 1]) * p.scale_log2 - l0.y) +
+                  fast_exp2(__uint_as_float(v0[j + 2]) * p.scale_log2 - l0.z) + fast_exp2(__uint_as_float(v0[j + 3]) * p.scale_log2 - l0.w);
+            a1 += fast_exp2(__uint_as_float(v1[j]) * p.scale_log2 - l1.x) + fast_exp2(__uint_as_float(v1[j + 1]) * p.scale_log2 - l1.y) +
+                  fast_exp2(__uint_as_float(v1[j + 2]) * p.scale_log2 - l1.z) + fast_exp2(__uint_as_float(v1[j + 3]) * p.scale_log2 - l1.w);
+            a2 += fast_exp2(__uint_as_float(v2[j]) * p.scale_log2 - l2.x) + fast_exp2(__uint_as_float(v2[j + 1]) * p.scale_log2 - l2.y) +
+                  fast_exp2(__uint_as_float(v2[j + 2]) * p.scale_log2 - l2.z) + fast_exp2(__uint_as_float(v2[j + 3]) * p.scale_log2 - l2.w);
+            a3 += fast_exp2(__uint_as_float(v3[j]) * p.scale_log2 - l3.x) + fast_exp2(__uint_as_float(v3[j + 1]) * p.scale_log2 - l3.y) +
+                  fast_exp2(__uint_as_float(v3[j + 2]) * p.scale_log2 - l3.z) + fast_exp2(__uint_as_float(v3[j + 3]) * p.scale_log2 - l3.w);
+          }
+          acc += (a0 + a1) + (a2 + a3);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            if (j < rows_valid) acc += fast_exp2(__uint_as_float(v0[j]) * p.scale_log2 - ls[j]);
+            if (32 + j < rows_valid) acc += fast_exp2(__uint_as_float(v1[j]) * p.scale_log2 - ls[32 + j]);
+            if (64 + j < rows_valid) acc += fast_exp2(__uint_as_float(v2[j]) * p.scale_log2 - ls[64 + j]);
+            if (96 + j < rows_valid) acc += fast_exp2(__uint_as_float(v3[j]) * p.scale_log2 - ls[96 + j]);
+          }
+        }
+      }
+    }
+    if (alive && !*abort_flag) {
+      const int j = key0 + key_l - sq.video_start;           // video token index of this key
+      if (j >= 0 && j < sq.n_video) p.partial[(size_t)layer * p.sum_video + sq.score_off + j] = acc;
+    } else if (p.d_status && et == 0) {
+      *p.d_status = SPECVLM_ERR_TIMEOUT;
+    }
+  }
+  // every role ends here; the allocating warp returns the tensor memory
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
 // scores[j] = (sum over layers, in order, of partial[l][j]) / (L * Hq * n_text of j's sequence)
 __global__ void scores_finish_kernel(const __grid_constant__ ScoreParams p, float* __restrict__ scores) {
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
@@ -586,13 +803,26 @@ static int32_t launch_lse(ScoreSetup& su, cudaStream_t st) {
 
 template <int D>
 static int32_t launch_colsum(ScoreSetup& su, float* scores, cudaStream_t st) {
-  constexpr int STAGES = 3;
-  constexpr int SMEM = (STAGES + 1) * kKeyTile * D * 2 + 1024 + 16 * STAGES + 16 + 16 + 128 * 4;
-  auto k = scores_colsum_kernel<D, STAGES>;
-  if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
-    return SPECVLM_ERR_CUDA;
-  k<<<dim3((unsigned)su.n_key_blocks, (unsigned)su.kv.n_layers), 288, SMEM, st>>>(su.tk, su.tq, su.p2);
-  int32_t rc = launch_status();
+  const char* impl = getenv("SPECVLM_SCORES_IMPL");
+  const bool legacy = impl && impl[0] == 'm';      // "mma": the mma.sync kernel
+  int32_t rc;
+  if (legacy) {
+    constexpr int STAGES = 3;
+    constexpr int SMEM = (STAGES + 1) * kKeyTile * D * 2 + 1024 + 16 * STAGES + 16 + 16 + 128 * 4;
+    auto k = scores_colsum_kernel<D, STAGES>;
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
+      return SPECVLM_ERR_CUDA;
+    k<<<dim3((unsigned)su.n_key_blocks, (unsigned)su.kv.n_layers), 288, SMEM, st>>>(su.tk, su.tq, su.p2);
+    rc = launch_status();
+  } else {
+    constexpr int STAGES = 4;
+    constexpr int SMEM = (2 + STAGES) * kKeyTile * D * 2 + 1024 + 16 * STAGES + 64 + 16 + 2 * 128 * 4;
+    auto k = scores_colsum_tc_kernel<D, STAGES>;
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
+      return SPECVLM_ERR_CUDA;
+    k<<<dim3((unsigned)su.n_key_blocks, (unsigned)su.kv.n_layers), 192, SMEM, st>>>(su.tk, su.tq, su.p2);
+    rc = launch_status();
+  }
   if (rc != SPECVLM_OK) return rc;
   scores_finish_kernel<<<(unsigned)((su.p2.sum_video + 255) / 256), 256, 0, st>>>(su.p2, scores);
   return launch_status();
