@@ -8,6 +8,7 @@
 // fp32 with base-2 exponentials.  Long sequences are split across CTAs; a second kernel merges
 // the split partials by their log-sum-exp.
 #include "attn.cuh"
+#include "attn_sched.h"
 #include "host_util.h"
 
 namespace specvlm {
@@ -743,6 +744,17 @@ static int32_t launch_any(const CUtensorMap& tk, const CUtensorMap& tv, const At
   return launch_rowsN<D, 3, 2>(tk, tv, p, grid, st);
 }
 
+// tcgen05 path (attn_tc.cu)
+size_t attn_tc_ws_bytes(const specvlm_kv_t* kv, int32_t batch, int rows);
+int32_t attn_tc_launch(const specvlm_kv_t* kv, const void* q, int32_t batch, int32_t n_q_heads, int32_t n_q,
+                       float sm_scale, void* out, float* lse, void* ws, size_t ws_bytes, int32_t* d_status,
+                       cudaStream_t st);
+
+static bool use_legacy_mma() {
+  const char* s = getenv("SPECVLM_ATTN_IMPL");
+  return s && s[0] == 'm';             // "mma": the mma.sync kernels
+}
+
 static int32_t attn_common(const specvlm_kv_t* kv, const void* q, int32_t batch, int32_t n_q_heads,
                            int32_t n_q, float sm_scale, void* out, float* lse, void* ws,
                            size_t ws_bytes, int32_t* d_status, void* stream) {
@@ -754,6 +766,9 @@ static int32_t attn_common(const specvlm_kv_t* kv, const void* q, int32_t batch,
   const int group = n_q_heads / kv->n_kv_heads;
   if (group > 16 || n_q > 9) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   const int rows = group * n_q;
+  if (!use_legacy_mma())
+    return attn_tc_launch(kv, q, batch, n_q_heads, n_q, sm_scale, out, lse, ws, ws_bytes, d_status,
+                          static_cast<cudaStream_t>(stream));
   if (rows > 96) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   const int64_t lb64 = (int64_t)kv->n_layers * batch;
   if (lb64 > 65535 * 64 || kv->n_kv_heads > 65535) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
@@ -823,7 +838,9 @@ extern "C" size_t specvlm_attn_workspace_bytes(const specvlm_kv_t* kv, int32_t b
   if (!kv || batch < 1 || n_q_heads < 1 || gamma < 0 || kv->n_kv_heads < 1 ||
       n_q_heads % kv->n_kv_heads != 0 || kv->n_layers < 1 || kv->max_seq_len < 1)
     return 0;
-  return attn_ws_bytes(kv, batch, (n_q_heads / kv->n_kv_heads) * (gamma + 1));
+  const int rows = (n_q_heads / kv->n_kv_heads) * (gamma + 1);
+  if (!use_legacy_mma()) return rows <= 128 && batch <= kSchedMaxBatch ? attn_tc_ws_bytes(kv, batch, rows) : 0;
+  return attn_ws_bytes(kv, batch, rows);
 }
 
 extern "C" int32_t specvlm_draft_decode_attn(const specvlm_kv_t* kv, const void* q, int32_t batch,

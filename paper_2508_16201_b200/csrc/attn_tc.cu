@@ -1,0 +1,721 @@
+// Streaming softmax attention over a bf16 K/V cache on the 5th-generation tensor cores of sm_100a:
+// draft decode attention (1 query token) and (gamma+1)-query verification attention.
+//
+// One persistent CTA per SM streams a contiguous slice of the flat (layer, sequence, KV head, tile)
+// list (attn_sched.h), so the cache is read exactly once, every SM moves the same number of bytes
+// and only two partial results per CTA ever touch scratch memory.
+//
+// Roles inside a CTA (7 warps):
+//   warp 0   TMA producer: 64-token K and V tiles, HBM -> shared memory ring (128-byte swizzle)
+//   warp 1   MMA issuer (one thread): S = Q K^T and O += P V as tcgen05.mma, accumulators in TMEM
+//   warps 2-5 softmax: S from TMEM, running max / sum, P (bf16) to shared memory, final O from TMEM
+//   warp 6   query loader: the item's query rows -> the swizzled A-operand tile, one item ahead
+// The GQA group's heads times the query tokens are the M rows of the tiles.  Row r of an item lives
+// in TMEM lane 32*((r/16)%4) + 16*(r/64) + r%16, which spreads 16-row chunks over the four softmax
+// warps (a warp can only read its own 32 lanes).
+//
+// The running maximum is only raised when a tile's maximum exceeds it by more than 2^8; O is then
+// rescaled in place in TMEM.  Probabilities stay below 2^8, well inside bf16 / fp32 range, and the
+// common tile needs no pass over O at all.
+#include "attn.cuh"
+#include "attn_sched.h"
+#include "host_util.h"
+
+namespace specvlm {
+
+struct AttnTcParams {
+  const __nv_bfloat16* q;     // [L][B][n_q][Hq][D]
+  __nv_bfloat16* out;         // same shape
+  float* lse;                 // [L][B][n_q][Hq] or null
+  float* ws_o;                // partial results: [2 * grid][rows][D], normalised
+  float* ws_lse;              // [2 * grid][rows], log2 units
+  int32_t* ws_cnt;            // [items] arrival counters, zero at launch
+  const int32_t* block_table; // [B][max_blocks] or null
+  const int32_t* seq_lens;    // [B]
+  int32_t* d_status;
+  int32_t batch, n_layers, n_q, n_q_heads, n_kv_heads, group, rows;
+  int32_t max_blocks, block_tokens, max_seq_len;
+  float scale_log2;           // sm_scale * log2(e)
+};
+
+constexpr float kRescaleThreshold = 8.f;   // log2 units
+
+__device__ __forceinline__ int row_to_lane(int r) {
+  const int chunk = r >> 4;
+  return ((chunk & 3) << 5) + ((chunk >> 2) << 4) + (r & 15);
+}
+
+// 16 TMEM lanes x 64 fp32 columns -> 32 registers per thread: registers 4j, 4j+1 hold lane
+// (base + tid/4), columns 8j + 2(tid%4) + {0,1}; registers 4j+2, 4j+3 the same columns of lane
+// (base + 8 + tid/4).
+__device__ __forceinline__ void tmem_ld_16x256b_x8(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_16x256b_x8(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.16x256b.x8.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ uint4 ldg_nc_v4(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ float ldg_cg_f32(const float* p) {
+  float v;
+  asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ float4 ldg_cg_f32x4(const float* p) {
+  float4 v;
+  asm volatile("ld.global.cg.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+  return v;
+}
+
+// Walks a CTA's slice segment by segment.
+struct SliceCursor {
+  int64_t f, end;
+  Segment sg;
+  int j;          // tile inside the current segment
+  int seg_idx;    // segments entered so far - 1
+  __device__ __forceinline__ void start(int64_t begin, int64_t end_, const int* prefix, int batch, int hkv) {
+    f = begin;
+    end = end_;
+    j = 0;
+    seg_idx = 0;
+    if (f < end) sg = segment_at(f, end, prefix, batch, hkv);
+  }
+  __device__ __forceinline__ bool first_of_segment() const { return j == 0; }
+  __device__ __forceinline__ bool last_of_segment() const { return j == sg.n_tiles - 1; }
+  __device__ __forceinline__ void next_tile(const int* prefix, int batch, int hkv) {
+    ++f;
+    if (++j == sg.n_tiles) {
+      j = 0;
+      ++seg_idx;
+      if (f < end) sg = segment_at(f, end, prefix, batch, hkv);
+    }
+  }
+};
+
+template <int D, int STAGES>
+struct TcLayout {
+  static constexpr int KT_BYTES = kTileTokens * D * 2;          // one K (or V) tile
+  static constexpr int STAGE_BYTES = 2 * KT_BYTES;
+  static constexpr int Q_BYTES = 128 * D * 2;                   // A operand of S = Q K^T
+  static constexpr int P_BYTES = 128 * kTileTokens * 2;         // A operand of O += P V
+  static constexpr int OFF_Q = STAGES * STAGE_BYTES;
+  static constexpr int OFF_P = OFF_Q + 2 * Q_BYTES;
+  static constexpr int OFF_BAR = OFF_P + 2 * P_BYTES;
+  static constexpr int N_BARS = 2 * STAGES + 16;
+  static constexpr int OFF_MISC = OFF_BAR + 8 * N_BARS;         // abort flag, tmem slot, last-arriver flag
+  static constexpr int OFF_PREFIX = OFF_MISC + 32;
+  static constexpr int TOTAL = OFF_PREFIX + (kSchedMaxBatch + 1) * 4 + 1024;   // + alignment slack
+};
+
+template <int D, int STAGES>
+__global__ void __launch_bounds__(224, 1)
+attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+               const __grid_constant__ AttnTcParams p) {
+  using L = TcLayout<D, STAGES>;
+  constexpr int KT_BYTES = L::KT_BYTES, STAGE_BYTES = L::STAGE_BYTES, Q_BYTES = L::Q_BYTES, P_BYTES = L::P_BYTES;
+  constexpr uint32_t kTmemCols = 256;                 // S buffers at columns 0 and 64, O at 128
+  constexpr uint32_t kIdescQK = umma_idesc_bf16(128, kTileTokens, false, false);
+  constexpr uint32_t kIdescPV = umma_idesc_bf16(128, D, false, true);   // V tile: channels run along the row
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t base = (raw_addr + 1023u) & ~1023u;
+  uint8_t* const smem = smem_raw + (base - raw_addr);
+  const uint32_t kv_sm = base, q_sm = base + L::OFF_Q, p_sm = base + L::OFF_P;
+  const uint32_t bar0 = base + L::OFF_BAR;
+  const uint32_t bar_kv_full = bar0, bar_kv_empty = bar0 + 8 * STAGES;
+  const uint32_t bar_q_full = bar0 + 16 * STAGES;      // [2]
+  const uint32_t bar_q_empty = bar_q_full + 16;        // [2]
+  const uint32_t bar_s_full = bar_q_empty + 16;        // [2]
+  const uint32_t bar_s_empty = bar_s_full + 16;        // [2]
+  const uint32_t bar_p_full = bar_s_empty + 16;        // [2]
+  const uint32_t bar_p_empty = bar_p_full + 16;        // [2]
+  const uint32_t bar_o_full = bar_p_empty + 16;
+  const uint32_t bar_o_empty = bar_o_full + 8;
+  const uint32_t bar_ep_done = bar_o_empty + 8;        // softmax threads: partial result written
+  const uint32_t bar_ep_flag = bar_ep_done + 8;        // ... and the arrival counter has been read
+  volatile int* const abort_flag = reinterpret_cast<volatile int*>(smem + L::OFF_MISC);
+  volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_MISC + 8);
+  volatile int* const last_flag = reinterpret_cast<volatile int*>(smem + L::OFF_MISC + 16);
+  volatile int* const any_empty = reinterpret_cast<volatile int*>(smem + L::OFF_MISC + 20);
+  int* const prefix = reinterpret_cast<int*>(smem + L::OFF_PREFIX);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  // ------------------------------------------------------------------ set-up
+  if (tid == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(bar_kv_full + 8 * s, 1);
+      mbar_init(bar_kv_empty + 8 * s, 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar_q_full + 8 * i, 1);
+      mbar_init(bar_q_empty + 8 * i, 1);
+      mbar_init(bar_s_full + 8 * i, 1);
+      mbar_init(bar_s_empty + 8 * i, 4);
+      mbar_init(bar_p_full + 8 * i, 4);
+      mbar_init(bar_p_empty + 8 * i, 1);
+    }
+    mbar_init(bar_o_full, 1);
+    mbar_init(bar_o_empty, 4);
+    mbar_init(bar_ep_done, 4);
+    mbar_init(bar_ep_flag, 1);
+    *abort_flag = 0;
+    *any_empty = 0;
+    prefix[0] = 0;
+    mbar_fence_init();
+  }
+  __syncthreads();
+  if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+  // tiles per sequence, then their running sum
+  for (int b = tid; b < p.batch; b += blockDim.x) {
+    int n = p.seq_lens[b];
+    n = n < 0 ? 0 : (n > p.max_seq_len ? p.max_seq_len : n);
+    prefix[b + 1] = (n + kTileTokens - 1) / kTileTokens;
+    if (n == 0) *any_empty = 1;
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) {
+    int carry = 0;
+    for (int b0 = 0; b0 < p.batch; b0 += 32) {
+      const int b = b0 + lane;
+      int v = b < p.batch ? prefix[b + 1] : 0;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int o = __shfl_up_sync(0xffffffffu, v, off);
+        if (lane >= off) v += o;
+      }
+      if (b < p.batch) prefix[b + 1] = v + carry;
+      carry += __shfl_sync(0xffffffffu, v, 31);
+    }
+  }
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  const int hkv = p.n_kv_heads;
+  const int64_t total = (int64_t)p.n_layers * hkv * prefix[p.batch];
+  const int n_active = sched_active_ctas(total, (int)gridDim.x);
+  const int cta = blockIdx.x;
+  const int64_t T0 = (total > 0 && cta < n_active) ? slice_begin(cta, n_active, total) : 0;
+  const int64_t T1 = (total > 0 && cta < n_active) ? slice_begin(cta + 1, n_active, total) : 0;
+  const int n_items = p.n_layers * p.batch * hkv;
+
+  if (warp == 0) {
+    // ================================================================ TMA producer
+    if (lane == 0 && T1 > T0) {
+      tma_prefetch_desc(&tm_k);
+      tma_prefetch_desc(&tm_v);
+      const uint64_t policy = l2_policy_evict_first();
+      const int tiles_per_block = p.block_table ? p.block_tokens / kTileTokens : 1;
+      SliceCursor c;
+      c.start(T0, T1, prefix, p.batch, hkv);
+      bool ok = true;
+      int i = 0;
+      auto block_of = [&](const SliceCursor& cc) -> int {
+        if (!p.block_table) return cc.sg.b;
+        return __ldg(p.block_table + (size_t)cc.sg.b * p.max_blocks + (cc.sg.tile0 + cc.j) / tiles_per_block);
+      };
+      int blk = block_of(c);
+      for (; c.f < T1; ++i) {
+        const int s = i % STAGES;
+        const int layer = c.sg.layer, g = c.sg.g, tile = c.sg.tile0 + c.j;
+        const int tok = p.block_table ? (tile % tiles_per_block) * kTileTokens : tile * kTileTokens;
+        const int blk_now = blk;
+        c.next_tile(prefix, p.batch, hkv);
+        if (c.f < T1) blk = block_of(c);              // table entry of the next tile, one tile ahead
+        if (i >= STAGES) ok = mbar_wait(bar_kv_empty + 8 * s, ((i / STAGES) - 1) & 1, abort_flag);
+        if (!ok) break;
+        const uint32_t full = bar_kv_full + 8 * s;
+        const uint32_t dst = kv_sm + s * STAGE_BYTES;
+        mbar_arrive_expect_tx(full, STAGE_BYTES);
+#pragma unroll
+        for (int h = 0; h < D / 64; ++h) {
+          tma_load_5d(dst + h * (kTileTokens * 128), &tm_k, full, h * 64, tok, g, blk_now, layer, policy);
+          tma_load_5d(dst + KT_BYTES + h * (kTileTokens * 128), &tm_v, full, h * 64, tok, g, blk_now, layer, policy);
+        }
+      }
+      if (!ok) {
+        // a wait expired: report, then stay until this CTA's copies in flight have landed (bounded)
+        if (p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
+        const uint64_t t0 = global_timer_ns();
+        for (int k = i > STAGES ? i - STAGES : 0; k < i; ++k)
+          while (!mbar_try_wait(bar_kv_full + 8 * (k % STAGES), (k / STAGES) & 1) &&
+                 global_timer_ns() - t0 < kWaitLimitNs) {
+          }
+      }
+    }
+  } else if (warp == 1) {
+    // ================================================================ MMA issuer
+    if (lane == 0 && T1 > T0) {
+      SliceCursor cq, cp;            // S = Q K^T runs one tile ahead of O += P V
+      cq.start(T0, T1, prefix, p.batch, hkv);
+      cp.start(T0, T1, prefix, p.batch, hkv);
+      const int n = (int)(T1 - T0);
+      bool ok = true;
+      auto issue_qk = [&](int i) {
+        const int st = i % STAGES, buf = i & 1, qb = cq.seg_idx & 1;
+        ok = mbar_wait(bar_kv_full + 8 * st, (i / STAGES) & 1, abort_flag);
+        if (ok && cq.first_of_segment()) ok = mbar_wait(bar_q_full + 8 * qb, (cq.seg_idx >> 1) & 1, abort_flag);
+        if (ok && i >= 2) ok = mbar_wait(bar_s_empty + 8 * buf, ((i >> 1) - 1) & 1, abort_flag);
+        if (!ok) return;
+        tc_fence_after_sync();
+        const uint32_t a0 = q_sm + qb * Q_BYTES, b0 = kv_sm + st * STAGE_BYTES;
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+          // 16 channels per step = 32 bytes along the swizzled 128-byte row; channels 64.. are the
+          // second 64-channel block of the tile
+          const uint32_t offa = (ks >> 2) * (128 * 128) + (ks & 3) * 32;
+          const uint32_t offb = (ks >> 2) * (kTileTokens * 128) + (ks & 3) * 32;
+          umma_bf16_ss(tmem_base + buf * kTileTokens, umma_desc_sw128(a0 + offa, 16, 1024),
+                       umma_desc_sw128(b0 + offb, 16, 1024), kIdescQK, ks > 0 ? 1u : 0u);
+        }
+        umma_commit(bar_s_full + 8 * buf);
+        if (cq.last_of_segment()) umma_commit(bar_q_empty + 8 * qb);
+        cq.next_tile(prefix, p.batch, hkv);
+      };
+      auto issue_pv = [&](int i) {
+        const int st = i % STAGES, buf = i & 1;
+        ok = mbar_wait(bar_p_full + 8 * buf, (i >> 1) & 1, abort_flag);
+        if (ok && cp.first_of_segment() && cp.seg_idx >= 1)
+          ok = mbar_wait(bar_o_empty, (cp.seg_idx - 1) & 1, abort_flag);
+        if (!ok) return;
+        tc_fence_after_sync();
+        const uint32_t a0 = p_sm + buf * P_BYTES, b0 = kv_sm + st * STAGE_BYTES + KT_BYTES;
+#pragma unroll
+        for (int kt = 0; kt < kTileTokens / 16; ++kt) {
+          // 16 tokens per step: 32 bytes along P's row; 16 rows of 128 bytes down the V tile, whose
+          // 64-channel blocks are kTileTokens * 128 bytes apart
+          umma_bf16_ss(tmem_base + 128, umma_desc_sw128(a0 + kt * 32, 16, 1024),
+                       umma_desc_sw128(b0 + kt * 2048, kTileTokens * 128, 1024), kIdescPV,
+                       (!cp.first_of_segment() || kt > 0) ? 1u : 0u);
+        }
+        umma_commit(bar_kv_empty + 8 * st);
+        umma_commit(bar_p_empty + 8 * buf);
+        if (cp.last_of_segment()) umma_commit(bar_o_full);
+        cp.next_tile(prefix, p.batch, hkv);
+      };
+      issue_qk(0);
+      for (int i = 0; i < n && ok; ++i) {
+        if (i + 1 < n) issue_qk(i + 1);
+        if (ok) issue_pv(i);
+      }
+      if (!ok && p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
+    }
+  } else if (warp == 6) {
+    // ================================================================ query loader
+    if (T1 > T0) {
+      for (int idx = lane; idx < 2 * Q_BYTES / 16; idx += 32)      // rows no item uses stay zero
+        *reinterpret_cast<uint4*>(smem + L::OFF_Q + idx * 16) = make_uint4(0, 0, 0, 0);
+      __syncwarp();
+      SliceCursor c;
+      c.start(T0, T1, prefix, p.batch, hkv);
+      bool ok = true;
+      while (c.f < T1 && ok) {
+        const int qb = c.seg_idx & 1;
+        if (c.seg_idx >= 2)
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_q_empty + 8 * qb, ((c.seg_idx >> 1) - 1) & 1, abort_flag));
+        if (!ok) break;
+        const int lb = c.sg.layer * p.batch + c.sg.b;
+        uint8_t* const qbuf = smem + L::OFF_Q + qb * Q_BYTES;
+        constexpr int CPR = D / 8;                                   // 16-byte chunks per row
+        for (int ci = lane; ci < p.rows * CPR; ci += 32) {
+          const int r = ci / CPR, c16 = ci - r * CPR;
+          const int t = r / p.group, hh = r - t * p.group;
+          const uint4 val = ldg_nc_v4(p.q + (((size_t)lb * p.n_q + t) * p.n_q_heads + c.sg.g * p.group + hh) * D + c16 * 8);
+          const int m = row_to_lane(r);
+          *reinterpret_cast<uint4*>(qbuf + (c16 >> 3) * (128 * 128) + m * 128 + (((c16 & 7) ^ (m & 7)) << 4)) = val;
+        }
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_q_full + 8 * qb);
+        // on to the next segment
+        const int64_t nf = c.f + c.sg.n_tiles;
+        const int si = c.seg_idx + 1;
+        c.start(nf, T1, prefix, p.batch, hkv);
+        c.seg_idx = si;
+      }
+    }
+  } else {
+    // ================================================================ softmax / epilogue (warps 2..5)
+    const int quarter = warp & 3;                 // TMEM lanes [32 * quarter, +32)
+    const int st = (warp - 2) * 32 + lane;        // 0..127
+    const int nh = (p.rows > 16 * quarter ? 1 : 0) + (p.rows > 16 * (quarter + 4) ? 1 : 0);
+    const int lr = lane >> 2, lc = (lane & 3) * 2;   // row inside a 16-lane half (and +8), first column of a pair
+
+    // sequences without any token: their outputs are zero, their LSE -inf
+    if (*any_empty) {
+      for (int item = cta; item < n_items; item += gridDim.x) {
+        const int lb = item / hkv, g = item - lb * hkv, b = lb % p.batch;
+        if (prefix[b + 1] != prefix[b]) continue;
+        for (int idx = st; idx < p.rows * (D / 8); idx += 128) {
+          const int r = idx / (D / 8), c8 = idx - r * (D / 8);
+          const int t = r / p.group, h = g * p.group + (r - t * p.group);
+          const size_t orow = ((size_t)lb * p.n_q + t) * p.n_q_heads + h;
+          *reinterpret_cast<uint4*>(p.out + orow * D + c8 * 8) = make_uint4(0, 0, 0, 0);
+          if (p.lse && c8 == 0) p.lse[orow] = -INFINITY;
+        }
+      }
+    }
+
+    SliceCursor c;
+    c.start(T0, T1, prefix, p.batch, hkv);
+    bool ok = true;
+    int i = 0;            // tiles processed by this CTA
+    int n_partial = 0;    // partial epilogues so far
+#define SM_WAIT(bar, parity)                                                        \
+  do {                                                                              \
+    ok = __all_sync(0xffffffffu, mbar_wait((bar), (parity), abort_flag));           \
+    if (!ok) goto softmax_done;                                                     \
+  } while (0)
+
+    while (c.f < T1) {
+      const Segment sg = c.sg;
+      const int seg_idx = c.seg_idx;
+      int kv_len = p.seq_lens[sg.b];
+      kv_len = kv_len < 0 ? 0 : (kv_len > p.max_seq_len ? p.max_seq_len : kv_len);
+      // rows of this thread: half h, 16-lane chunk quarter + 4h, rows 16*chunk + lr and + 8
+      int lim[2][2];
+      float m_used[2][2], l_sum[2][2];
+#pragma unroll
+      for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int r = 16 * (quarter + 4 * h) + lr + 8 * e;
+          lim[h][e] = r < p.rows ? kv_len - p.n_q + r / p.group + 1 : 0;
+          m_used[h][e] = -INFINITY;
+          l_sum[h][e] = 0.f;
+        }
+
+      for (int j = 0; j < sg.n_tiles; ++j, ++i) {
+        const int buf = i & 1;
+        const int tile_tok0 = (sg.tile0 + j) * kTileTokens;
+        const bool need_mask = tile_tok0 + kTileTokens > kv_len - p.n_q + 1;
+        SM_WAIT(bar_s_full + 8 * buf, (i >> 1) & 1);
+        tc_fence_after_sync();
+        uint32_t v[2][32];
+        if (nh > 0) tmem_ld_16x256b_x8(tmem_base + ((uint32_t)(32 * quarter) << 16) + buf * kTileTokens, v[0]);
+        if (nh > 1) tmem_ld_16x256b_x8(tmem_base + ((uint32_t)(32 * quarter + 16) << 16) + buf * kTileTokens, v[1]);
+        tmem_ld_wait();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_s_empty + 8 * buf);
+        if (i >= 2) SM_WAIT(bar_p_empty + 8 * buf, ((i >> 1) - 1) & 1);      // P buffer free again
+
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if (h >= nh) break;
+          float s[32];
+          float mx0 = -INFINITY, mx1 = -INFINITY;
+          if (need_mask) {
+#pragma unroll
+            for (int k = 0; k < 32; ++k) {
+              const int tok = tile_tok0 + (k >> 2) * 8 + lc + (k & 1);
+              const int e = (k >> 1) & 1;
+              const float x = tok < lim[h][e] ? __uint_as_float(v[h][k]) * p.scale_log2 : -INFINITY;
+              s[k] = x;
+              if (e == 0) mx0 = fmaxf(mx0, x); else mx1 = fmaxf(mx1, x);
+            }
+          } else {
+#pragma unroll
+            for (int k = 0; k < 32; ++k) {
+              const float x = __uint_as_float(v[h][k]) * p.scale_log2;
+              s[k] = x;
+              if (((k >> 1) & 1) == 0) mx0 = fmaxf(mx0, x); else mx1 = fmaxf(mx1, x);
+            }
+          }
+          mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+          mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+          mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+          mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+          if (j == 0) {
+            // first tile of the segment: O is overwritten by this tile's product
+            m_used[h][0] = mx0;
+            m_used[h][1] = mx1;
+          } else {
+            const bool up0 = mx0 > m_used[h][0] + kRescaleThreshold, up1 = mx1 > m_used[h][1] + kRescaleThreshold;
+            if (__any_sync(0xffffffffu, up0 || up1)) {
+              // raise the reference maximum of those rows and rescale their O rows in TMEM
+              const float a0 = up0 ? fast_exp2(m_used[h][0] - mx0) : 1.f;
+              const float a1 = up1 ? fast_exp2(m_used[h][1] - mx1) : 1.f;
+              if (up0) m_used[h][0] = mx0;
+              if (up1) m_used[h][1] = mx1;
+              l_sum[h][0] *= a0;
+              l_sum[h][1] *= a1;
+              SM_WAIT(bar_p_empty + 8 * (buf ^ 1), ((i - 1) >> 1) & 1);    // O += P V of the previous tile is complete
+              tc_fence_after_sync();
+#pragma unroll
+              for (int cc = 0; cc < D / 64; ++cc) {
+                uint32_t o[32];
+                const uint32_t oaddr = tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + 128 + cc * 64;
+                tmem_ld_16x256b_x8(oaddr, o);
+                tmem_ld_wait();
+#pragma unroll
+                for (int k = 0; k < 32; ++k)
+                  o[k] = __float_as_uint(__uint_as_float(o[k]) * (((k >> 1) & 1) ? a1 : a0));
+                tmem_st_16x256b_x8(oaddr, o);
+              }
+              tmem_st_wait();
+              tc_fence_before_sync();
+            }
+          }
+          const float mu0 = m_used[h][0] == -INFINITY ? 0.f : m_used[h][0];
+          const float mu1 = m_used[h][1] == -INFINITY ? 0.f : m_used[h][1];
+          float ps0 = 0.f, ps1 = 0.f;
+          const int m0 = 32 * quarter + 16 * h + lr, m1 = m0 + 8;       // A-operand rows = TMEM lanes
+          const uint32_t prow0 = p_sm + buf * P_BYTES + m0 * 128 + lc * 2;
+          const uint32_t prow1 = p_sm + buf * P_BYTES + m1 * 128 + lc * 2;
+#pragma unroll
+          for (int jj = 0; jj < 8; ++jj) {
+            const float p0 = fast_exp2(s[4 * jj] - mu0), p1 = fast_exp2(s[4 * jj + 1] - mu0);
+            const float p2 = fast_exp2(s[4 * jj + 2] - mu1), p3 = fast_exp2(s[4 * jj + 3] - mu1);
+            ps0 += p0 + p1;
+            ps1 += p2 + p3;
+            asm volatile("st.shared.b32 [%0], %1;" ::"r"(prow0 + ((jj ^ (m0 & 7)) << 4)), "r"(pack_bf16x2(p0, p1)) : "memory");
+            asm volatile("st.shared.b32 [%0], %1;" ::"r"(prow1 + ((jj ^ (m1 & 7)) << 4)), "r"(pack_bf16x2(p2, p3)) : "memory");
+          }
+          l_sum[h][0] += ps0;
+          l_sum[h][1] += ps1;
+        }
+        if (tile_tok0 + kTileTokens > kv_len) {
+          // last, ragged tile: the V rows past the end of the sequence hold whatever the page held;
+          // clear them so that a zero probability times a stale non-finite value cannot reach O
+          SM_WAIT(bar_kv_full + 8 * (i % STAGES), (i / STAGES) & 1);
+          uint8_t* vt = smem + (i % STAGES) * STAGE_BYTES + KT_BYTES;
+          const int first = kv_len - tile_tok0;
+          for (int idx = st; idx < (kTileTokens - first) * (D / 8); idx += 128) {
+            const int t = first + idx / (D / 8), c16 = idx % (D / 8);
+            *reinterpret_cast<uint4*>(vt + (c16 >> 3) * (kTileTokens * 128) + t * 128 + (c16 & 7) * 16) =
+                make_uint4(0, 0, 0, 0);
+          }
+        }
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_p_full + 8 * buf);
+      }
+
+      // ---------------------------------------------------------------- end of the segment: O -> out
+      const bool complete = sg.tile0 == 0 && sg.n_tiles == sg.item_tiles;
+      const int lb = sg.layer * p.batch + sg.b;
+      const int slot = partial_slot(cta, T0, sg.item_begin);
+      SM_WAIT(bar_o_full, seg_idx & 1);
+      tc_fence_after_sync();
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        if (h >= nh) break;
+        float inv[2], lse2[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          float lt = l_sum[h][e];
+          lt += __shfl_xor_sync(0xffffffffu, lt, 1);
+          lt += __shfl_xor_sync(0xffffffffu, lt, 2);
+          inv[e] = lt > 0.f ? 1.f / lt : 0.f;
+          lse2[e] = lt > 0.f ? m_used[h][e] + log2f(lt) : -INFINITY;
+        }
+#pragma unroll
+        for (int cc = 0; cc < D / 64; ++cc) {
+          uint32_t o[32];
+          tmem_ld_16x256b_x8(tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + 128 + cc * 64, o);
+          tmem_ld_wait();
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int r = 16 * (quarter + 4 * h) + lr + 8 * e;
+            if (r >= p.rows) continue;
+            if (complete) {
+              const int t = r / p.group, hq = sg.g * p.group + (r - t * p.group);
+              const size_t orow = ((size_t)lb * p.n_q + t) * p.n_q_heads + hq;
+              __nv_bfloat16* dst = p.out + orow * D + cc * 64 + lc;
+#pragma unroll
+              for (int jj = 0; jj < 8; ++jj)
+                *reinterpret_cast<uint32_t*>(dst + jj * 8) =
+                    pack_bf16x2(__uint_as_float(o[4 * jj + 2 * e]) * inv[e], __uint_as_float(o[4 * jj + 2 * e + 1]) * inv[e]);
+              if (p.lse && cc == 0 && (lane & 3) == 0) p.lse[orow] = lse2[e] * kLn2;
+            } else {
+              float* dst = p.ws_o + ((size_t)slot * p.rows + r) * D + cc * 64 + lc;
+#pragma unroll
+              for (int jj = 0; jj < 8; ++jj)
+                *reinterpret_cast<float2*>(dst + jj * 8) =
+                    make_float2(__uint_as_float(o[4 * jj + 2 * e]) * inv[e], __uint_as_float(o[4 * jj + 2 * e + 1]) * inv[e]);
+              if (cc == 0 && (lane & 3) == 0) p.ws_lse[(size_t)slot * p.rows + r] = lse2[e];
+            }
+          }
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_o_empty);
+
+      if (!complete) {
+        // the CTA that brings an item's last partial result merges all of them, in slice order
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_ep_done);
+        const int64_t item_end = sg.item_begin + sg.item_tiles;
+        const int c_first = slice_owner(sg.item_begin, n_active, total);
+        const int c_last = slice_owner(item_end - 1, n_active, total);
+        if (st == 0) {
+          if (mbar_wait(bar_ep_done, n_partial & 1, abort_flag)) {
+            const int old = atomicAdd(p.ws_cnt + sg.item, 1);
+            __threadfence();
+            *last_flag = (old == c_last - c_first) ? 1 : 0;
+          } else {
+            *last_flag = 0;
+          }
+          mbar_arrive(bar_ep_flag);
+        }
+        SM_WAIT(bar_ep_flag, n_partial & 1);
+        ++n_partial;
+        if (*last_flag) {
+          __threadfence();
+          const int np = c_last - c_first + 1;
+          for (int idx = st; idx < p.rows * (D / 4); idx += 128) {
+            const int r = idx / (D / 4), c4 = idx - r * (D / 4);
+            float M = -INFINITY;
+            for (int cpart = c_first; cpart <= c_last; ++cpart) {
+              const int sl = partial_slot(cpart, slice_begin(cpart, n_active, total), sg.item_begin);
+              M = fmaxf(M, ldg_cg_f32(p.ws_lse + (size_t)sl * p.rows + r));
+            }
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            float den = 0.f;
+            if (M != -INFINITY) {
+              for (int cpart = c_first; cpart <= c_last; ++cpart) {
+                const int sl = partial_slot(cpart, slice_begin(cpart, n_active, total), sg.item_begin);
+                const float w = fast_exp2(ldg_cg_f32(p.ws_lse + (size_t)sl * p.rows + r) - M);
+                const float4 x = ldg_cg_f32x4(p.ws_o + ((size_t)sl * p.rows + r) * D + c4 * 4);
+                acc.x += w * x.x;
+                acc.y += w * x.y;
+                acc.z += w * x.z;
+                acc.w += w * x.w;
+                den += w;
+              }
+            }
+            (void)np;
+            const float invd = den > 0.f ? 1.f / den : 0.f;
+            const int t = r / p.group, hq = sg.g * p.group + (r - t * p.group);
+            const size_t orow = ((size_t)lb * p.n_q + t) * p.n_q_heads + hq;
+            uint2 packed;
+            packed.x = pack_bf16x2(acc.x * invd, acc.y * invd);
+            packed.y = pack_bf16x2(acc.z * invd, acc.w * invd);
+            *reinterpret_cast<uint2*>(p.out + orow * D + c4 * 4) = packed;
+            if (p.lse && c4 == 0) p.lse[orow] = den > 0.f ? (M + log2f(den)) * kLn2 : -INFINITY;
+          }
+        }
+      }
+      // next segment
+      {
+        const int64_t nf = sg.item_begin + sg.tile0 + sg.n_tiles;
+        c.start(nf, T1, prefix, p.batch, hkv);
+        c.seg_idx = seg_idx + 1;
+      }
+    }
+  softmax_done:
+    if (!ok && p.d_status && st == 0) *p.d_status = SPECVLM_ERR_TIMEOUT;
+#undef SM_WAIT
+  }
+
+  // every role ends here; the allocating warp returns the tensor memory
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------
+static int tc_grid(const specvlm_kv_t* kv, int32_t batch) {
+  const int64_t tiles_max = (int64_t)kv->n_layers * batch * kv->n_kv_heads *
+                            ((kv->max_seq_len + kTileTokens - 1) / kTileTokens);
+  return sched_active_ctas(tiles_max, sm_count());
+}
+
+size_t attn_tc_ws_bytes(const specvlm_kv_t* kv, int32_t batch, int rows) {
+  const int grid = tc_grid(kv, batch);
+  const size_t items = (size_t)kv->n_layers * batch * kv->n_kv_heads;
+  return round_up((size_t)2 * grid * rows * kv->head_dim * sizeof(float), 256) +
+         round_up((size_t)2 * grid * rows * sizeof(float), 256) + round_up(items * sizeof(int32_t), 256);
+}
+
+template <int D, int STAGES>
+static int32_t launch_tc(const CUtensorMap& tk, const CUtensorMap& tv, const AttnTcParams& p, int grid,
+                         cudaStream_t st) {
+  using L = TcLayout<D, STAGES>;
+  auto kern = attn_tc_kernel<D, STAGES>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL) != cudaSuccess)
+    return SPECVLM_ERR_CUDA;
+  kern<<<grid, 224, L::TOTAL, st>>>(tk, tv, p);
+  return launch_status();
+}
+
+int32_t attn_tc_launch(const specvlm_kv_t* kv, const void* q, int32_t batch, int32_t n_q_heads, int32_t n_q,
+                       float sm_scale, void* out, float* lse, void* ws, size_t ws_bytes, int32_t* d_status,
+                       cudaStream_t st) {
+  const int group = n_q_heads / kv->n_kv_heads;
+  const int rows = group * n_q;
+  if (rows > 128 || batch > kSchedMaxBatch) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  const int64_t items = (int64_t)kv->n_layers * batch * kv->n_kv_heads;
+  if (items > 0x3fffffff) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) return SPECVLM_ERR_INVALID_ARG;
+  if (ws_bytes < attn_tc_ws_bytes(kv, batch, rows)) return SPECVLM_ERR_WORKSPACE_TOO_SMALL;
+  const int grid = tc_grid(kv, batch);
+
+  CUtensorMap tk, tv;
+  int32_t rc = encode_kv_map(&tk, kv, kv->k, kTileTokens);
+  if (rc != SPECVLM_OK) return rc;
+  rc = encode_kv_map(&tv, kv, kv->v, kTileTokens);
+  if (rc != SPECVLM_OK) return rc;
+
+  AttnTcParams p;
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.lse = lse;
+  uint8_t* w = static_cast<uint8_t*>(ws);
+  p.ws_o = reinterpret_cast<float*>(w);
+  w += round_up((size_t)2 * grid * rows * kv->head_dim * sizeof(float), 256);
+  p.ws_lse = reinterpret_cast<float*>(w);
+  w += round_up((size_t)2 * grid * rows * sizeof(float), 256);
+  p.ws_cnt = reinterpret_cast<int32_t*>(w);
+  p.block_table = kv->block_table;
+  p.seq_lens = kv->seq_lens;
+  p.d_status = d_status;
+  p.batch = batch;
+  p.n_layers = kv->n_layers;
+  p.n_q = n_q;
+  p.n_q_heads = n_q_heads;
+  p.n_kv_heads = kv->n_kv_heads;
+  p.group = group;
+  p.rows = rows;
+  p.max_blocks = kv->max_blocks;
+  p.block_tokens = kv->block_tokens;
+  p.max_seq_len = kv->max_seq_len;
+  p.scale_log2 = sm_scale * kLog2e;
+
+  if (cudaMemsetAsync(p.ws_cnt, 0, (size_t)items * sizeof(int32_t), st) != cudaSuccess) return SPECVLM_ERR_CUDA;
+  return kv->head_dim == 128 ? launch_tc<128, 4>(tk, tv, p, grid, st) : launch_tc<64, 8>(tk, tv, p, grid, st);
+}
+
+}  // namespace specvlm
