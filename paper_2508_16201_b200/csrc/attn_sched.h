@@ -18,7 +18,7 @@
 
 namespace specvlm {
 
-constexpr int kSchedMaxBatch = 255;     // sequences per call (their tile counts live in shared memory)
+constexpr int kSchedMaxBatch = 127;     // sequences per call (their tile counts live in shared memory)
 constexpr int kSchedMinTilesPerCta = 4;   // below this a slice is not worth a CTA of its own
 
 // Number of CTAs that get a non-empty slice.

@@ -5,18 +5,25 @@
 // list (attn_sched.h), so the cache is read exactly once, every SM moves the same number of bytes
 // and only two partial results per CTA ever touch scratch memory.
 //
-// Roles inside a CTA (7 warps):
-//   warp 0   TMA producer: 64-token K and V tiles, HBM -> shared memory ring (128-byte swizzle)
-//   warp 1   MMA issuer (one thread): S = Q K^T and O += P V as tcgen05.mma, accumulators in TMEM
-//   warps 2-5 softmax: S from TMEM, running max / sum, P (bf16) to shared memory, final O from TMEM
-//   warp 6   query loader: the item's query rows -> the swizzled A-operand tile, one item ahead
-// The GQA group's heads times the query tokens are the M rows of the tiles.  Row r of an item lives
-// in TMEM lane 32*((r/16)%4) + 16*(r/64) + r%16, which spreads 16-row chunks over the four softmax
-// warps (a warp can only read its own 32 lanes).
+// Roles inside a CTA (12 warps = 3 warpgroups; the first gives registers to the other two):
+//   warp 0     TMA producer: 64-token K tiles and V tiles, HBM -> two shared-memory rings (128-byte
+//              swizzle).  K and V have rings of their own because a K tile is free again as soon
+//              as S = Q K^T has been computed, long before its V tile.
+//   warp 1     issues S = Q K^T (one thread, tcgen05.mma, accumulator in TMEM)
+//   warp 2     issues O += P V (one thread); two issuers, because one thread cannot issue both
+//              chains and poll their barriers within a tile's memory time
+//   warp 3     query loader: the item's query rows -> the swizzled A-operand tile, one item ahead
+//   warps 4-7  softmax group 0: the even tiles of the slice
+//   warps 8-11 softmax group 1: the odd tiles.  Each group has its own S buffer, P buffer, running
+//              (max, sum) and its own O accumulator; the two are merged once per item.
+// The GQA group's heads times the query tokens are the M rows of the tiles: M = 64 when they fit
+// (rows 16c..16c+15 live in TMEM lanes 32c..32c+15), else M = 128 (row r in lane
+// 32*((r/16)%4) + 16*(r/64) + r%16); either way 16-row chunks are spread over the four warps of a
+// group, since a warp can only read its own 32 lanes.
 //
-// The running maximum is only raised when a tile's maximum exceeds it by more than 2^8; O is then
-// rescaled in place in TMEM.  Probabilities stay below 2^8, well inside bf16 / fp32 range, and the
-// common tile needs no pass over O at all.
+// The running maximum of a row is only raised when a tile's maximum exceeds it by more than 2^8; O
+// is then rescaled in place in TMEM.  Probabilities stay below 2^8, well inside bf16 / fp32 range,
+// and the common tile needs no pass over O at all.
 #include "attn.cuh"
 #include "attn_sched.h"
 #include "host_util.h"
@@ -39,10 +46,14 @@ struct AttnTcParams {
 };
 
 constexpr float kRescaleThreshold = 8.f;   // log2 units
+constexpr int kTcThreads = 384;
+constexpr int kRegsLight = 96, kRegsSoftmax = 200;   // 128 * 96 + 256 * 200 <= 64 K registers
 
-__device__ __forceinline__ int row_to_lane(int r) {
-  const int chunk = r >> 4;
-  return ((chunk & 3) << 5) + ((chunk >> 2) << 4) + (r & 15);
+template <int N> __device__ __forceinline__ void setmaxnreg_dec() {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N> __device__ __forceinline__ void setmaxnreg_inc() {
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
 }
 
 // 16 TMEM lanes x 64 fp32 columns -> 32 registers per thread: registers 4j, 4j+1 hold lane
@@ -102,73 +113,102 @@ struct SliceCursor {
     seg_idx = 0;
     if (f < end) sg = segment_at(f, end, prefix, batch, hkv);
   }
-  __device__ __forceinline__ bool first_of_segment() const { return j == 0; }
   __device__ __forceinline__ bool last_of_segment() const { return j == sg.n_tiles - 1; }
   __device__ __forceinline__ void next_tile(const int* prefix, int batch, int hkv) {
     ++f;
-    if (++j == sg.n_tiles) {
-      j = 0;
-      ++seg_idx;
-      if (f < end) sg = segment_at(f, end, prefix, batch, hkv);
-    }
+    if (++j == sg.n_tiles) next_segment(prefix, batch, hkv);
+  }
+  __device__ __forceinline__ void next_segment(const int* prefix, int batch, int hkv) {
+    f = sg.item_begin + sg.tile0 + sg.n_tiles;
+    j = 0;
+    ++seg_idx;
+    if (f < end) sg = segment_at(f, end, prefix, batch, hkv);
   }
 };
 
-template <int D, int STAGES>
-struct TcLayout {
+// Shared-memory plan.  A small region (barriers, flags, per-sequence tile counts, the softmax
+// groups' row statistics) sits at the start of the dynamic shared memory; the tile rings and the
+// operand tiles follow at the next 1024-byte boundary.
+template <int D, int M>
+struct TcCfg {
   static constexpr int KT_BYTES = kTileTokens * D * 2;          // one K (or V) tile
-  static constexpr int STAGE_BYTES = 2 * KT_BYTES;
-  static constexpr int Q_BYTES = 128 * D * 2;                   // A operand of S = Q K^T
-  static constexpr int P_BYTES = 128 * kTileTokens * 2;         // A operand of O += P V
-  static constexpr int OFF_Q = STAGES * STAGE_BYTES;
+  static constexpr int NK = D == 128 ? (M == 64 ? 5 : 3) : 8;   // K ring stages
+  static constexpr int NV = D == 128 ? (M == 64 ? 6 : 4) : 8;   // V ring stages
+  static constexpr int Q_BYTES = M * D * 2;                     // A operand of S = Q K^T
+  static constexpr int P_BYTES = M * kTileTokens * 2;           // A operand of O += P V
+  static constexpr int OFF_K = 0;
+  static constexpr int OFF_V = OFF_K + NK * KT_BYTES;
+  static constexpr int OFF_Q = OFF_V + NV * KT_BYTES;
   static constexpr int OFF_P = OFF_Q + 2 * Q_BYTES;
-  static constexpr int OFF_BAR = OFF_P + 2 * P_BYTES;
-  static constexpr int N_BARS = 2 * STAGES + 16;
-  static constexpr int OFF_MISC = OFF_BAR + 8 * N_BARS;         // abort flag, tmem slot, last-arriver flag
-  static constexpr int OFF_PREFIX = OFF_MISC + 32;
-  static constexpr int TOTAL = OFF_PREFIX + (kSchedMaxBatch + 1) * 4 + 1024;   // + alignment slack
+  static constexpr int BIG = OFF_P + 2 * P_BYTES;
+  static constexpr int N_BARS = 2 * NK + 2 * NV + 17;
+  static constexpr int SM_BAR = 0;
+  static constexpr int SM_MISC = SM_BAR + 8 * N_BARS;
+  static constexpr int SM_PREFIX = SM_MISC + 32;
+  static constexpr int SM_STATS = SM_PREFIX + (kSchedMaxBatch + 1) * 4;     // [2 segments][2 groups][M rows] float2
+  static constexpr int SMALL_USED = SM_STATS + 2 * 2 * M * 8;
+  static constexpr int SMALL = (SMALL_USED + 1023) / 1024 * 1024;
+  static constexpr int kMaxSmem = 232448;                       // 227 KB
+  // a spare KB for a base that is not 1024-byte aligned, where there is room for it
+  static constexpr int TOTAL = SMALL + BIG + (SMALL + BIG + 1024 <= kMaxSmem ? 1024 : 0);
+  static constexpr uint32_t TMEM_COLS = 128 + 2 * D <= 256 ? 256 : 512;   // S0 | S1 | O0 | O1
+  static_assert(SMALL + BIG <= kMaxSmem, "shared-memory plan does not fit");
 };
 
-template <int D, int STAGES>
-__global__ void __launch_bounds__(224, 1)
+template <int D, int M>
+__global__ void __launch_bounds__(kTcThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                const __grid_constant__ AttnTcParams p) {
-  using L = TcLayout<D, STAGES>;
-  constexpr int KT_BYTES = L::KT_BYTES, STAGE_BYTES = L::STAGE_BYTES, Q_BYTES = L::Q_BYTES, P_BYTES = L::P_BYTES;
-  constexpr uint32_t kTmemCols = 256;                 // S buffers at columns 0 and 64, O at 128
-  constexpr uint32_t kIdescQK = umma_idesc_bf16(128, kTileTokens, false, false);
-  constexpr uint32_t kIdescPV = umma_idesc_bf16(128, D, false, true);   // V tile: channels run along the row
+  using C = TcCfg<D, M>;
+  constexpr int KT_BYTES = C::KT_BYTES, NK = C::NK, NV = C::NV, Q_BYTES = C::Q_BYTES, P_BYTES = C::P_BYTES;
+  constexpr int NH = M / 64;                          // 16-lane halves a softmax warp may own
+  constexpr uint32_t kColS = 0, kColO = 128;          // TMEM columns: S of group g at 64 g, O at 128 + D g
+  constexpr uint32_t kIdescQK = umma_idesc_bf16(M, kTileTokens, false, false);
+  constexpr uint32_t kIdescPV = umma_idesc_bf16(M, D, false, true);   // V tile: channels run along the row
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
-  const uint32_t base = (raw_addr + 1023u) & ~1023u;
-  uint8_t* const smem = smem_raw + (base - raw_addr);
-  const uint32_t kv_sm = base, q_sm = base + L::OFF_Q, p_sm = base + L::OFF_P;
-  const uint32_t bar0 = base + L::OFF_BAR;
-  const uint32_t bar_kv_full = bar0, bar_kv_empty = bar0 + 8 * STAGES;
-  const uint32_t bar_q_full = bar0 + 16 * STAGES;      // [2]
+  const uint32_t big = (raw_addr + C::SMALL_USED + 1023u) & ~1023u;
+  uint8_t* const big_ptr = smem_raw + (big - raw_addr);
+  const uint32_t k_sm = big + C::OFF_K, v_sm = big + C::OFF_V, q_sm = big + C::OFF_Q, p_sm = big + C::OFF_P;
+  const uint32_t bar0 = raw_addr + C::SM_BAR;
+  const uint32_t bar_k_full = bar0, bar_k_empty = bar_k_full + 8 * NK;
+  const uint32_t bar_v_full = bar_k_empty + 8 * NK, bar_v_empty = bar_v_full + 8 * NV;
+  const uint32_t bar_q_full = bar_v_empty + 8 * NV;    // [2]
   const uint32_t bar_q_empty = bar_q_full + 16;        // [2]
-  const uint32_t bar_s_full = bar_q_empty + 16;        // [2]
+  const uint32_t bar_s_full = bar_q_empty + 16;        // [2]: one per softmax group
   const uint32_t bar_s_empty = bar_s_full + 16;        // [2]
   const uint32_t bar_p_full = bar_s_empty + 16;        // [2]
   const uint32_t bar_p_empty = bar_p_full + 16;        // [2]
   const uint32_t bar_o_full = bar_p_empty + 16;
   const uint32_t bar_o_empty = bar_o_full + 8;
-  const uint32_t bar_ep_done = bar_o_empty + 8;        // softmax threads: partial result written
+  const uint32_t bar_ep_stats = bar_o_empty + 8;       // both groups' row statistics are in shared memory
+  const uint32_t bar_ep_done = bar_ep_stats + 8;       // a partial result has been written
   const uint32_t bar_ep_flag = bar_ep_done + 8;        // ... and the arrival counter has been read
-  volatile int* const abort_flag = reinterpret_cast<volatile int*>(smem + L::OFF_MISC);
-  volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_MISC + 8);
-  volatile int* const last_flag = reinterpret_cast<volatile int*>(smem + L::OFF_MISC + 16);
-  volatile int* const any_empty = reinterpret_cast<volatile int*>(smem + L::OFF_MISC + 20);
-  int* const prefix = reinterpret_cast<int*>(smem + L::OFF_PREFIX);
+  volatile int* const abort_flag = reinterpret_cast<volatile int*>(smem_raw + C::SM_MISC);
+  volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_raw + C::SM_MISC + 8);
+  volatile int* const last_flag = reinterpret_cast<volatile int*>(smem_raw + C::SM_MISC + 16);
+  volatile int* const any_empty = reinterpret_cast<volatile int*>(smem_raw + C::SM_MISC + 20);
+  int* const prefix = reinterpret_cast<int*>(smem_raw + C::SM_PREFIX);
+  float2* const stats = reinterpret_cast<float2*>(smem_raw + C::SM_STATS);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
+  // the plan needs the tiles inside the allocation (true whenever the base is 1024-byte aligned)
+  if (big + C::BIG > raw_addr + C::TOTAL) {
+    if (tid == 0 && p.d_status) *p.d_status = SPECVLM_ERR_CUDA;
+    return;
+  }
+
   // ------------------------------------------------------------------ set-up
   if (tid == 0) {
-    for (int s = 0; s < STAGES; ++s) {
-      mbar_init(bar_kv_full + 8 * s, 1);
-      mbar_init(bar_kv_empty + 8 * s, 1);
+    for (int s = 0; s < NK; ++s) {
+      mbar_init(bar_k_full + 8 * s, 1);
+      mbar_init(bar_k_empty + 8 * s, 1);
+    }
+    for (int s = 0; s < NV; ++s) {
+      mbar_init(bar_v_full + 8 * s, 1);
+      mbar_init(bar_v_empty + 8 * s, 1);
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_q_full + 8 * i, 1);
@@ -179,8 +219,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       mbar_init(bar_p_empty + 8 * i, 1);
     }
     mbar_init(bar_o_full, 1);
-    mbar_init(bar_o_empty, 4);
-    mbar_init(bar_ep_done, 4);
+    mbar_init(bar_o_empty, 8);
+    mbar_init(bar_ep_stats, 8);
+    mbar_init(bar_ep_done, 8);
     mbar_init(bar_ep_flag, 1);
     *abort_flag = 0;
     *any_empty = 0;
@@ -188,7 +229,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     mbar_fence_init();
   }
   __syncthreads();
-  if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+  if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), C::TMEM_COLS);
   // tiles per sequence, then their running sum
   for (int b = tid; b < p.batch; b += blockDim.x) {
     int n = p.seq_lens[b];
@@ -219,13 +260,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   const int64_t total = (int64_t)p.n_layers * hkv * prefix[p.batch];
   const int n_active = sched_active_ctas(total, (int)gridDim.x);
   const int cta = blockIdx.x;
-  const int64_t T0 = (total > 0 && cta < n_active) ? slice_begin(cta, n_active, total) : 0;
-  const int64_t T1 = (total > 0 && cta < n_active) ? slice_begin(cta + 1, n_active, total) : 0;
+  const bool active = total > 0 && cta < n_active;
+  const int64_t T0 = active ? slice_begin(cta, n_active, total) : 0;
+  const int64_t T1 = active ? slice_begin(cta + 1, n_active, total) : 0;
   const int n_items = p.n_layers * p.batch * hkv;
 
   if (warp == 0) {
     // ================================================================ TMA producer
-    if (lane == 0 && T1 > T0) {
+    setmaxnreg_dec<kRegsLight>();
+    if (lane == 0 && active) {
       tma_prefetch_desc(&tm_k);
       tma_prefetch_desc(&tm_v);
       const uint64_t policy = l2_policy_evict_first();
@@ -233,136 +276,167 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       SliceCursor c;
       c.start(T0, T1, prefix, p.batch, hkv);
       bool ok = true;
-      int i = 0;
-      auto block_of = [&](const SliceCursor& cc) -> int {
-        if (!p.block_table) return cc.sg.b;
-        return __ldg(p.block_table + (size_t)cc.sg.b * p.max_blocks + (cc.sg.tile0 + cc.j) / tiles_per_block);
-      };
-      int blk = block_of(c);
-      for (; c.f < T1; ++i) {
-        const int s = i % STAGES;
-        const int layer = c.sg.layer, g = c.sg.g, tile = c.sg.tile0 + c.j;
-        const int tok = p.block_table ? (tile % tiles_per_block) * kTileTokens : tile * kTileTokens;
-        const int blk_now = blk;
-        c.next_tile(prefix, p.batch, hkv);
-        if (c.f < T1) blk = block_of(c);              // table entry of the next tile, one tile ahead
-        if (i >= STAGES) ok = mbar_wait(bar_kv_empty + 8 * s, ((i / STAGES) - 1) & 1, abort_flag);
-        if (!ok) break;
-        const uint32_t full = bar_kv_full + 8 * s;
-        const uint32_t dst = kv_sm + s * STAGE_BYTES;
-        mbar_arrive_expect_tx(full, STAGE_BYTES);
+      int i = 0, k_issued = 0, v_issued = 0;
+      while (c.f < T1 && ok) {
+        const Segment sg = c.sg;
+        const int32_t* table = p.block_table ? p.block_table + (size_t)sg.b * p.max_blocks : nullptr;
+        int blk_next = table ? __ldg(table + sg.tile0 / tiles_per_block) : sg.b;
+        for (int j = 0; j < sg.n_tiles; ++j, ++i) {
+          const int tile = sg.tile0 + j;
+          const int blk = blk_next;
+          if (table && j + 1 < sg.n_tiles) blk_next = __ldg(table + (tile + 1) / tiles_per_block);   // one tile ahead
+          const int tok = table ? (tile % tiles_per_block) * kTileTokens : tile * kTileTokens;
+          const int ks = i % NK, vs = i % NV;
+          if (i >= NK) ok = mbar_wait(bar_k_empty + 8 * ks, ((i / NK) - 1) & 1, abort_flag);
+          if (!ok) break;
+          mbar_arrive_expect_tx(bar_k_full + 8 * ks, KT_BYTES);
 #pragma unroll
-        for (int h = 0; h < D / 64; ++h) {
-          tma_load_5d(dst + h * (kTileTokens * 128), &tm_k, full, h * 64, tok, g, blk_now, layer, policy);
-          tma_load_5d(dst + KT_BYTES + h * (kTileTokens * 128), &tm_v, full, h * 64, tok, g, blk_now, layer, policy);
+          for (int h = 0; h < D / 64; ++h)
+            tma_load_5d(k_sm + ks * KT_BYTES + h * (kTileTokens * 128), &tm_k, bar_k_full + 8 * ks, h * 64, tok, sg.g,
+                        blk, sg.layer, policy);
+          k_issued = i + 1;
+          if (i >= NV) ok = mbar_wait(bar_v_empty + 8 * vs, ((i / NV) - 1) & 1, abort_flag);
+          if (!ok) break;
+          mbar_arrive_expect_tx(bar_v_full + 8 * vs, KT_BYTES);
+#pragma unroll
+          for (int h = 0; h < D / 64; ++h)
+            tma_load_5d(v_sm + vs * KT_BYTES + h * (kTileTokens * 128), &tm_v, bar_v_full + 8 * vs, h * 64, tok, sg.g,
+                        blk, sg.layer, policy);
+          v_issued = i + 1;
         }
+        c.next_segment(prefix, p.batch, hkv);
       }
       if (!ok) {
         // a wait expired: report, then stay until this CTA's copies in flight have landed (bounded)
         if (p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
         const uint64_t t0 = global_timer_ns();
-        for (int k = i > STAGES ? i - STAGES : 0; k < i; ++k)
-          while (!mbar_try_wait(bar_kv_full + 8 * (k % STAGES), (k / STAGES) & 1) &&
-                 global_timer_ns() - t0 < kWaitLimitNs) {
+        for (int k = k_issued > NK ? k_issued - NK : 0; k < k_issued; ++k)
+          while (!mbar_test_wait(bar_k_full + 8 * (k % NK), (k / NK) & 1) && global_timer_ns() - t0 < kWaitLimitNs) {
+          }
+        for (int k = v_issued > NV ? v_issued - NV : 0; k < v_issued; ++k)
+          while (!mbar_test_wait(bar_v_full + 8 * (k % NV), (k / NV) & 1) && global_timer_ns() - t0 < kWaitLimitNs) {
           }
       }
     }
   } else if (warp == 1) {
-    // ================================================================ MMA issuer
-    if (lane == 0 && T1 > T0) {
-      SliceCursor cq, cp;            // S = Q K^T runs one tile ahead of O += P V
-      cq.start(T0, T1, prefix, p.batch, hkv);
-      cp.start(T0, T1, prefix, p.batch, hkv);
+    // ================================================================ S = Q K^T issuer
+    setmaxnreg_dec<kRegsLight>();
+    if (lane == 0 && active) {
+      SliceCursor c;
+      c.start(T0, T1, prefix, p.batch, hkv);
       const int n = (int)(T1 - T0);
+      const uint64_t dq0 = umma_desc_sw128(q_sm, 16, 1024), dk0 = umma_desc_sw128(k_sm, 16, 1024);
       bool ok = true;
-      auto issue_qk = [&](int i) {
-        const int st = i % STAGES, buf = i & 1, qb = cq.seg_idx & 1;
-        ok = mbar_wait(bar_kv_full + 8 * st, (i / STAGES) & 1, abort_flag);
-        if (ok && cq.first_of_segment()) ok = mbar_wait(bar_q_full + 8 * qb, (cq.seg_idx >> 1) & 1, abort_flag);
-        if (ok && i >= 2) ok = mbar_wait(bar_s_empty + 8 * buf, ((i >> 1) - 1) & 1, abort_flag);
-        if (!ok) return;
+      for (int i = 0; i < n; ++i) {
+        const int g = i & 1, ks = i % NK, qb = c.seg_idx & 1;
+        ok = mbar_wait(bar_k_full + 8 * ks, (i / NK) & 1, abort_flag);
+        if (ok && c.j == 0) ok = mbar_wait(bar_q_full + 8 * qb, (c.seg_idx >> 1) & 1, abort_flag);
+        if (ok && i >= 2) ok = mbar_wait(bar_s_empty + 8 * g, ((i >> 1) - 1) & 1, abort_flag);
+        if (!ok) break;
         tc_fence_after_sync();
-        const uint32_t a0 = q_sm + qb * Q_BYTES, b0 = kv_sm + st * STAGE_BYTES;
+        const uint64_t da = umma_desc_advance(dq0, qb * Q_BYTES), db = umma_desc_advance(dk0, ks * KT_BYTES);
+        const uint32_t d_tmem = tmem_base + kColS + g * kTileTokens;
 #pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) {
+        for (int s = 0; s < D / 16; ++s)
           // 16 channels per step = 32 bytes along the swizzled 128-byte row; channels 64.. are the
-          // second 64-channel block of the tile
-          const uint32_t offa = (ks >> 2) * (128 * 128) + (ks & 3) * 32;
-          const uint32_t offb = (ks >> 2) * (kTileTokens * 128) + (ks & 3) * 32;
-          umma_bf16_ss(tmem_base + buf * kTileTokens, umma_desc_sw128(a0 + offa, 16, 1024),
-                       umma_desc_sw128(b0 + offb, 16, 1024), kIdescQK, ks > 0 ? 1u : 0u);
-        }
-        umma_commit(bar_s_full + 8 * buf);
-        if (cq.last_of_segment()) umma_commit(bar_q_empty + 8 * qb);
-        cq.next_tile(prefix, p.batch, hkv);
-      };
-      auto issue_pv = [&](int i) {
-        const int st = i % STAGES, buf = i & 1;
-        ok = mbar_wait(bar_p_full + 8 * buf, (i >> 1) & 1, abort_flag);
-        if (ok && cp.first_of_segment() && cp.seg_idx >= 1)
-          ok = mbar_wait(bar_o_empty, (cp.seg_idx - 1) & 1, abort_flag);
-        if (!ok) return;
-        tc_fence_after_sync();
-        const uint32_t a0 = p_sm + buf * P_BYTES, b0 = kv_sm + st * STAGE_BYTES + KT_BYTES;
-#pragma unroll
-        for (int kt = 0; kt < kTileTokens / 16; ++kt) {
-          // 16 tokens per step: 32 bytes along P's row; 16 rows of 128 bytes down the V tile, whose
-          // 64-channel blocks are kTileTokens * 128 bytes apart
-          umma_bf16_ss(tmem_base + 128, umma_desc_sw128(a0 + kt * 32, 16, 1024),
-                       umma_desc_sw128(b0 + kt * 2048, kTileTokens * 128, 1024), kIdescPV,
-                       (!cp.first_of_segment() || kt > 0) ? 1u : 0u);
-        }
-        umma_commit(bar_kv_empty + 8 * st);
-        umma_commit(bar_p_empty + 8 * buf);
-        if (cp.last_of_segment()) umma_commit(bar_o_full);
-        cp.next_tile(prefix, p.batch, hkv);
-      };
-      issue_qk(0);
-      for (int i = 0; i < n && ok; ++i) {
-        if (i + 1 < n) issue_qk(i + 1);
-        if (ok) issue_pv(i);
+          // second 64-channel block of each tile
+          umma_bf16_ss(d_tmem, umma_desc_advance(da, (s >> 2) * (M * 128) + (s & 3) * 32),
+                       umma_desc_advance(db, (s >> 2) * (kTileTokens * 128) + (s & 3) * 32), kIdescQK, s > 0 ? 1u : 0u);
+        umma_commit(bar_s_full + 8 * g);
+        umma_commit(bar_k_empty + 8 * ks);
+        if (c.last_of_segment()) umma_commit(bar_q_empty + 8 * qb);
+        c.next_tile(prefix, p.batch, hkv);
       }
       if (!ok && p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
     }
-  } else if (warp == 6) {
+  } else if (warp == 2) {
+    // ================================================================ O += P V issuer
+    setmaxnreg_dec<kRegsLight>();
+    if (lane == 0 && active) {
+      SliceCursor c;
+      c.start(T0, T1, prefix, p.batch, hkv);
+      const int n = (int)(T1 - T0);
+      const uint64_t dp0 = umma_desc_sw128(p_sm, 16, 1024);
+      const uint64_t dv0 = umma_desc_sw128(v_sm, kTileTokens * 128, 1024);   // 64-channel blocks 8 KB apart
+      bool ok = true;
+      for (int i = 0; i < n; ++i) {
+        const int g = i & 1, vs = i % NV;
+        ok = mbar_wait(bar_v_full + 8 * vs, (i / NV) & 1, abort_flag);
+        // the first product of each group overwrites that group's O: the previous item must be out
+        if (ok && c.j < 2 && c.seg_idx >= 1) ok = mbar_wait(bar_o_empty, (c.seg_idx - 1) & 1, abort_flag);
+        if (ok) ok = mbar_wait(bar_p_full + 8 * g, (i >> 1) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint64_t da = umma_desc_advance(dp0, g * P_BYTES), db = umma_desc_advance(dv0, vs * KT_BYTES);
+        const uint32_t d_tmem = tmem_base + kColO + g * D;
+        const uint32_t acc0 = c.j >= 2 ? 1u : 0u;
+#pragma unroll
+        for (int kt = 0; kt < kTileTokens / 16; ++kt)
+          // 16 tokens per step: 32 bytes along P's row, 16 rows of 128 bytes down the V tile
+          umma_bf16_ss(d_tmem, umma_desc_advance(da, kt * 32), umma_desc_advance(db, kt * 2048), kIdescPV,
+                       kt > 0 ? 1u : acc0);
+        umma_commit(bar_p_empty + 8 * g);
+        umma_commit(bar_v_empty + 8 * vs);
+        if (c.last_of_segment()) umma_commit(bar_o_full);
+        c.next_tile(prefix, p.batch, hkv);
+      }
+      if (!ok && p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
+    }
+  } else if (warp == 3) {
     // ================================================================ query loader
-    if (T1 > T0) {
+    setmaxnreg_dec<kRegsLight>();
+    if (active) {
       for (int idx = lane; idx < 2 * Q_BYTES / 16; idx += 32)      // rows no item uses stay zero
-        *reinterpret_cast<uint4*>(smem + L::OFF_Q + idx * 16) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(big_ptr + C::OFF_Q + idx * 16) = make_uint4(0, 0, 0, 0);
       __syncwarp();
       SliceCursor c;
       c.start(T0, T1, prefix, p.batch, hkv);
       bool ok = true;
+      constexpr int CPR = D / 8;                                   // 16-byte chunks per row
+      const int n_chunks = p.rows * CPR;
       while (c.f < T1 && ok) {
         const int qb = c.seg_idx & 1;
         if (c.seg_idx >= 2)
           ok = __all_sync(0xffffffffu, mbar_wait(bar_q_empty + 8 * qb, ((c.seg_idx >> 1) - 1) & 1, abort_flag));
         if (!ok) break;
         const int lb = c.sg.layer * p.batch + c.sg.b;
-        uint8_t* const qbuf = smem + L::OFF_Q + qb * Q_BYTES;
-        constexpr int CPR = D / 8;                                   // 16-byte chunks per row
-        for (int ci = lane; ci < p.rows * CPR; ci += 32) {
-          const int r = ci / CPR, c16 = ci - r * CPR;
-          const int t = r / p.group, hh = r - t * p.group;
-          const uint4 val = ldg_nc_v4(p.q + (((size_t)lb * p.n_q + t) * p.n_q_heads + c.sg.g * p.group + hh) * D + c16 * 8);
-          const int m = row_to_lane(r);
-          *reinterpret_cast<uint4*>(qbuf + (c16 >> 3) * (128 * 128) + m * 128 + (((c16 & 7) ^ (m & 7)) << 4)) = val;
+        uint8_t* const qbuf = big_ptr + C::OFF_Q + qb * Q_BYTES;
+        for (int c0 = 0; c0 < n_chunks; c0 += 32 * 8) {
+          uint4 val[8];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {                            // all loads of a batch in flight together
+            const int ci = c0 + u * 32 + lane;
+            if (ci < n_chunks) {
+              const int r = ci / CPR, c16 = ci - r * CPR;
+              const int t = r / p.group, hh = r - t * p.group;
+              val[u] = ldg_nc_v4(p.q + (((size_t)lb * p.n_q + t) * p.n_q_heads + c.sg.g * p.group + hh) * D + c16 * 8);
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const int ci = c0 + u * 32 + lane;
+            if (ci < n_chunks) {
+              const int r = ci / CPR, c16 = ci - r * CPR;
+              // row of the A operand: r itself for M = 64, the row's TMEM lane for M = 128
+              const int m = M == 64 ? r : ((((r >> 4) & 3) << 5) + ((r >> 6) << 4) + (r & 15));
+              *reinterpret_cast<uint4*>(qbuf + (c16 >> 3) * (M * 128) + m * 128 + (((c16 & 7) ^ (m & 7)) << 4)) = val[u];
+            }
+          }
         }
         fence_proxy_async();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_q_full + 8 * qb);
-        // on to the next segment
-        const int64_t nf = c.f + c.sg.n_tiles;
-        const int si = c.seg_idx + 1;
-        c.start(nf, T1, prefix, p.batch, hkv);
-        c.seg_idx = si;
+        c.next_segment(prefix, p.batch, hkv);
       }
     }
   } else {
-    // ================================================================ softmax / epilogue (warps 2..5)
+    // ================================================================ softmax / epilogue (warps 4..11)
+    setmaxnreg_inc<kRegsSoftmax>();
+    const int grp = (warp - 4) >> 2;              // tiles with (index & 1) == grp
     const int quarter = warp & 3;                 // TMEM lanes [32 * quarter, +32)
-    const int st = (warp - 2) * 32 + lane;        // 0..127
-    const int nh = (p.rows > 16 * quarter ? 1 : 0) + (p.rows > 16 * (quarter + 4) ? 1 : 0);
+    const int gt = (warp & 3) * 32 + lane;        // 0..127 inside the group
+    const int st = grp * 128 + gt;                // 0..255 over both groups
+    const int nh = (p.rows > 16 * quarter ? 1 : 0) + (NH > 1 && p.rows > 16 * (quarter + 4) ? 1 : 0);
     const int lr = lane >> 2, lc = (lane & 3) * 2;   // row inside a 16-lane half (and +8), first column of a pair
 
     // sequences without any token: their outputs are zero, their LSE -inf
@@ -370,7 +444,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       for (int item = cta; item < n_items; item += gridDim.x) {
         const int lb = item / hkv, g = item - lb * hkv, b = lb % p.batch;
         if (prefix[b + 1] != prefix[b]) continue;
-        for (int idx = st; idx < p.rows * (D / 8); idx += 128) {
+        for (int idx = st; idx < p.rows * (D / 8); idx += 256) {
           const int r = idx / (D / 8), c8 = idx - r * (D / 8);
           const int t = r / p.group, h = g * p.group + (r - t * p.group);
           const size_t orow = ((size_t)lb * p.n_q + t) * p.n_q_heads + h;
@@ -383,7 +457,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     SliceCursor c;
     c.start(T0, T1, prefix, p.batch, hkv);
     bool ok = true;
-    int i = 0;            // tiles processed by this CTA
+    int i0 = 0;           // index (inside the slice) of the current segment's first tile
     int n_partial = 0;    // partial epilogues so far
 #define SM_WAIT(bar, parity)                                                        \
   do {                                                                              \
@@ -396,11 +470,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       const int seg_idx = c.seg_idx;
       int kv_len = p.seq_lens[sg.b];
       kv_len = kv_len < 0 ? 0 : (kv_len > p.max_seq_len ? p.max_seq_len : kv_len);
-      // rows of this thread: half h, 16-lane chunk quarter + 4h, rows 16*chunk + lr and + 8
-      int lim[2][2];
-      float m_used[2][2], l_sum[2][2];
+      // rows of this thread: half h is the 16-row chunk quarter + 4h, rows 16 * chunk + lr and + 8
+      int lim[NH][2];
+      float m_used[NH][2], l_sum[NH][2];
 #pragma unroll
-      for (int h = 0; h < 2; ++h)
+      for (int h = 0; h < NH; ++h)
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
           const int r = 16 * (quarter + 4 * h) + lr + 8 * e;
@@ -409,49 +483,51 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           l_sum[h][e] = 0.f;
         }
 
-      for (int j = 0; j < sg.n_tiles; ++j, ++i) {
-        const int buf = i & 1;
+      for (int j = (i0 + grp) & 1; j < sg.n_tiles; j += 2) {
+        const int i = i0 + j;
         const int tile_tok0 = (sg.tile0 + j) * kTileTokens;
         const bool need_mask = tile_tok0 + kTileTokens > kv_len - p.n_q + 1;
-        SM_WAIT(bar_s_full + 8 * buf, (i >> 1) & 1);
+        SM_WAIT(bar_s_full + 8 * grp, (i >> 1) & 1);
         tc_fence_after_sync();
-        uint32_t v[2][32];
-        if (nh > 0) tmem_ld_16x256b_x8(tmem_base + ((uint32_t)(32 * quarter) << 16) + buf * kTileTokens, v[0]);
-        if (nh > 1) tmem_ld_16x256b_x8(tmem_base + ((uint32_t)(32 * quarter + 16) << 16) + buf * kTileTokens, v[1]);
+        uint32_t v[NH][32];
+#pragma unroll
+        for (int h = 0; h < NH; ++h)
+          if (h < nh) tmem_ld_16x256b_x8(tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + kColS + grp * kTileTokens, v[h]);
         tmem_ld_wait();
         tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) mbar_arrive(bar_s_empty + 8 * buf);
-        if (i >= 2) SM_WAIT(bar_p_empty + 8 * buf, ((i >> 1) - 1) & 1);      // P buffer free again
+        if (lane == 0) mbar_arrive(bar_s_empty + 8 * grp);
+        // the group's previous product has completed: P may be overwritten, O may be rescaled
+        if (i >= 2) SM_WAIT(bar_p_empty + 8 * grp, ((i >> 1) - 1) & 1);
 
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
+        for (int h = 0; h < NH; ++h) {
           if (h >= nh) break;
           float s[32];
-          float mx0 = -INFINITY, mx1 = -INFINITY;
+          float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
           if (need_mask) {
 #pragma unroll
             for (int k = 0; k < 32; ++k) {
               const int tok = tile_tok0 + (k >> 2) * 8 + lc + (k & 1);
-              const int e = (k >> 1) & 1;
-              const float x = tok < lim[h][e] ? __uint_as_float(v[h][k]) * p.scale_log2 : -INFINITY;
+              const float x = tok < lim[h][(k >> 1) & 1] ? __uint_as_float(v[h][k]) * p.scale_log2 : -INFINITY;
               s[k] = x;
-              if (e == 0) mx0 = fmaxf(mx0, x); else mx1 = fmaxf(mx1, x);
+              mx[k & 3] = fmaxf(mx[k & 3], x);
             }
           } else {
 #pragma unroll
             for (int k = 0; k < 32; ++k) {
               const float x = __uint_as_float(v[h][k]) * p.scale_log2;
               s[k] = x;
-              if (((k >> 1) & 1) == 0) mx0 = fmaxf(mx0, x); else mx1 = fmaxf(mx1, x);
+              mx[k & 3] = fmaxf(mx[k & 3], x);
             }
           }
+          float mx0 = fmaxf(mx[0], mx[1]), mx1 = fmaxf(mx[2], mx[3]);
           mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-          mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
           mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+          mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
           mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-          if (j == 0) {
-            // first tile of the segment: O is overwritten by this tile's product
+          if (j < 2) {
+            // the group's first tile of the item: O is overwritten by this tile's product
             m_used[h][0] = mx0;
             m_used[h][1] = mx1;
           } else {
@@ -464,12 +540,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               if (up1) m_used[h][1] = mx1;
               l_sum[h][0] *= a0;
               l_sum[h][1] *= a1;
-              SM_WAIT(bar_p_empty + 8 * (buf ^ 1), ((i - 1) >> 1) & 1);    // O += P V of the previous tile is complete
               tc_fence_after_sync();
 #pragma unroll
               for (int cc = 0; cc < D / 64; ++cc) {
                 uint32_t o[32];
-                const uint32_t oaddr = tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + 128 + cc * 64;
+                const uint32_t oaddr = tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + kColO + grp * D + cc * 64;
                 tmem_ld_16x256b_x8(oaddr, o);
                 tmem_ld_wait();
 #pragma unroll
@@ -483,29 +558,30 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           }
           const float mu0 = m_used[h][0] == -INFINITY ? 0.f : m_used[h][0];
           const float mu1 = m_used[h][1] == -INFINITY ? 0.f : m_used[h][1];
-          float ps0 = 0.f, ps1 = 0.f;
-          const int m0 = 32 * quarter + 16 * h + lr, m1 = m0 + 8;       // A-operand rows = TMEM lanes
-          const uint32_t prow0 = p_sm + buf * P_BYTES + m0 * 128 + lc * 2;
-          const uint32_t prow1 = p_sm + buf * P_BYTES + m1 * 128 + lc * 2;
+          float ps[4] = {0.f, 0.f, 0.f, 0.f};
+          // rows of the A operand of O += P V: the item's row for M = 64, the TMEM lane for M = 128
+          const int m0 = (M == 64 ? 16 * quarter : 32 * quarter + 16 * h) + lr, m1 = m0 + 8;
+          const uint32_t prow0 = p_sm + grp * P_BYTES + m0 * 128 + lc * 2;
+          const uint32_t prow1 = p_sm + grp * P_BYTES + m1 * 128 + lc * 2;
 #pragma unroll
           for (int jj = 0; jj < 8; ++jj) {
             const float p0 = fast_exp2(s[4 * jj] - mu0), p1 = fast_exp2(s[4 * jj + 1] - mu0);
             const float p2 = fast_exp2(s[4 * jj + 2] - mu1), p3 = fast_exp2(s[4 * jj + 3] - mu1);
-            ps0 += p0 + p1;
-            ps1 += p2 + p3;
+            ps[jj & 1] += p0 + p1;
+            ps[2 + (jj & 1)] += p2 + p3;
             asm volatile("st.shared.b32 [%0], %1;" ::"r"(prow0 + ((jj ^ (m0 & 7)) << 4)), "r"(pack_bf16x2(p0, p1)) : "memory");
             asm volatile("st.shared.b32 [%0], %1;" ::"r"(prow1 + ((jj ^ (m1 & 7)) << 4)), "r"(pack_bf16x2(p2, p3)) : "memory");
           }
-          l_sum[h][0] += ps0;
-          l_sum[h][1] += ps1;
+          l_sum[h][0] += ps[0] + ps[1];
+          l_sum[h][1] += ps[2] + ps[3];
         }
         if (tile_tok0 + kTileTokens > kv_len) {
           // last, ragged tile: the V rows past the end of the sequence hold whatever the page held;
           // clear them so that a zero probability times a stale non-finite value cannot reach O
-          SM_WAIT(bar_kv_full + 8 * (i % STAGES), (i / STAGES) & 1);
-          uint8_t* vt = smem + (i % STAGES) * STAGE_BYTES + KT_BYTES;
+          SM_WAIT(bar_v_full + 8 * (i % NV), (i / NV) & 1);
+          uint8_t* vt = big_ptr + C::OFF_V + (i % NV) * KT_BYTES;
           const int first = kv_len - tile_tok0;
-          for (int idx = st; idx < (kTileTokens - first) * (D / 8); idx += 128) {
+          for (int idx = gt; idx < (kTileTokens - first) * (D / 8); idx += 128) {
             const int t = first + idx / (D / 8), c16 = idx % (D / 8);
             *reinterpret_cast<uint4*>(vt + (c16 >> 3) * (kTileTokens * 128) + t * 128 + (c16 & 7) * 16) =
                 make_uint4(0, 0, 0, 0);
@@ -513,51 +589,92 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         }
         fence_proxy_async();
         __syncwarp();
-        if (lane == 0) mbar_arrive(bar_p_full + 8 * buf);
+        if (lane == 0) mbar_arrive(bar_p_full + 8 * grp);
       }
 
-      // ---------------------------------------------------------------- end of the segment: O -> out
+      // ---------------------------------------------------------------- end of the item's segment
+      // publish this group's row statistics, then merge the two groups' accumulators:
+      //   O = (w0 O0 + w1 O1) / (w0 l0 + w1 l1),  w_g = 2^(m_g - max(m0, m1))
       const bool complete = sg.tile0 == 0 && sg.n_tiles == sg.item_tiles;
       const int lb = sg.layer * p.batch + sg.b;
       const int slot = partial_slot(cta, T0, sg.item_begin);
-      SM_WAIT(bar_o_full, seg_idx & 1);
-      tc_fence_after_sync();
+      // statistics slots alternate between segments: a group may reach its next write while the
+      // other one still reads this segment's values
+      float2* const seg_stats = stats + (seg_idx & 1) * 2 * M;
+      auto srow = [&](int h) { return (M == 64 ? 16 * quarter : 32 * quarter + 16 * h) + lr; };
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
+      for (int h = 0; h < NH; ++h) {
         if (h >= nh) break;
-        float inv[2], lse2[2];
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
           float lt = l_sum[h][e];
           lt += __shfl_xor_sync(0xffffffffu, lt, 1);
           lt += __shfl_xor_sync(0xffffffffu, lt, 2);
-          inv[e] = lt > 0.f ? 1.f / lt : 0.f;
-          lse2[e] = lt > 0.f ? m_used[h][e] + log2f(lt) : -INFINITY;
+          if ((lane & 3) == 0) seg_stats[grp * M + srow(h) + 8 * e] = make_float2(m_used[h][e], lt);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_ep_stats);
+      SM_WAIT(bar_ep_stats, seg_idx & 1);
+      SM_WAIT(bar_o_full, seg_idx & 1);
+      tc_fence_after_sync();
+      // a group without a tile in this segment (one-tile segments) has nothing in its accumulator
+      const bool has0 = sg.n_tiles >= 2 || (i0 & 1) == 0, has1 = sg.n_tiles >= 2 || (i0 & 1) == 1;
+#pragma unroll
+      for (int h = 0; h < NH; ++h) {
+        if (h >= nh) break;
+        float w0[2], w1[2], lse2[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int ln = srow(h) + 8 * e;
+          const float2 s0 = seg_stats[ln], s1 = seg_stats[M + ln];
+          const float l0 = has0 ? s0.y : 0.f, l1 = has1 ? s1.y : 0.f;
+          const float ma = l0 > 0.f ? s0.x : -INFINITY, mb = l1 > 0.f ? s1.x : -INFINITY;
+          const float mm = fmaxf(ma, mb);
+          const float a = l0 > 0.f ? fast_exp2(ma - mm) : 0.f, b = l1 > 0.f ? fast_exp2(mb - mm) : 0.f;
+          const float den = a * l0 + b * l1;
+          const float inv = den > 0.f ? 1.f / den : 0.f;
+          w0[e] = a * inv;
+          w1[e] = b * inv;
+          lse2[e] = den > 0.f ? mm + log2f(den) : -INFINITY;
         }
 #pragma unroll
         for (int cc = 0; cc < D / 64; ++cc) {
-          uint32_t o[32];
-          tmem_ld_16x256b_x8(tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + 128 + cc * 64, o);
+          if ((cc & 1) != (D == 128 ? grp : 0)) continue;       // the groups share the column chunks
+          if (D == 64 && grp == 1) continue;
+          uint32_t oa[32], ob[32];
+          const uint32_t oaddr = tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + kColO + cc * 64;
+          if (has0) tmem_ld_16x256b_x8(oaddr, oa);
+          if (has1) tmem_ld_16x256b_x8(oaddr + D, ob);
           tmem_ld_wait();
 #pragma unroll
           for (int e = 0; e < 2; ++e) {
             const int r = 16 * (quarter + 4 * h) + lr + 8 * e;
             if (r >= p.rows) continue;
+            float res[16];
+#pragma unroll
+            for (int jj = 0; jj < 8; ++jj)
+#pragma unroll
+              for (int x = 0; x < 2; ++x) {
+                const int k = 4 * jj + 2 * e + x;
+                float acc = 0.f;
+                if (has0) acc = __uint_as_float(oa[k]) * w0[e];
+                if (has1) acc += __uint_as_float(ob[k]) * w1[e];
+                res[2 * jj + x] = acc;
+              }
             if (complete) {
               const int t = r / p.group, hq = sg.g * p.group + (r - t * p.group);
               const size_t orow = ((size_t)lb * p.n_q + t) * p.n_q_heads + hq;
               __nv_bfloat16* dst = p.out + orow * D + cc * 64 + lc;
 #pragma unroll
               for (int jj = 0; jj < 8; ++jj)
-                *reinterpret_cast<uint32_t*>(dst + jj * 8) =
-                    pack_bf16x2(__uint_as_float(o[4 * jj + 2 * e]) * inv[e], __uint_as_float(o[4 * jj + 2 * e + 1]) * inv[e]);
+                *reinterpret_cast<uint32_t*>(dst + jj * 8) = pack_bf16x2(res[2 * jj], res[2 * jj + 1]);
               if (p.lse && cc == 0 && (lane & 3) == 0) p.lse[orow] = lse2[e] * kLn2;
             } else {
               float* dst = p.ws_o + ((size_t)slot * p.rows + r) * D + cc * 64 + lc;
 #pragma unroll
               for (int jj = 0; jj < 8; ++jj)
-                *reinterpret_cast<float2*>(dst + jj * 8) =
-                    make_float2(__uint_as_float(o[4 * jj + 2 * e]) * inv[e], __uint_as_float(o[4 * jj + 2 * e + 1]) * inv[e]);
+                *reinterpret_cast<float2*>(dst + jj * 8) = make_float2(res[2 * jj], res[2 * jj + 1]);
               if (cc == 0 && (lane & 3) == 0) p.ws_lse[(size_t)slot * p.rows + r] = lse2[e];
             }
           }
@@ -589,20 +706,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         ++n_partial;
         if (*last_flag) {
           __threadfence();
-          const int np = c_last - c_first + 1;
-          for (int idx = st; idx < p.rows * (D / 4); idx += 128) {
+          for (int idx = st; idx < p.rows * (D / 4); idx += 256) {
             const int r = idx / (D / 4), c4 = idx - r * (D / 4);
-            float M = -INFINITY;
+            float mm = -INFINITY;
             for (int cpart = c_first; cpart <= c_last; ++cpart) {
               const int sl = partial_slot(cpart, slice_begin(cpart, n_active, total), sg.item_begin);
-              M = fmaxf(M, ldg_cg_f32(p.ws_lse + (size_t)sl * p.rows + r));
+              mm = fmaxf(mm, ldg_cg_f32(p.ws_lse + (size_t)sl * p.rows + r));
             }
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             float den = 0.f;
-            if (M != -INFINITY) {
+            if (mm != -INFINITY) {
               for (int cpart = c_first; cpart <= c_last; ++cpart) {
                 const int sl = partial_slot(cpart, slice_begin(cpart, n_active, total), sg.item_begin);
-                const float w = fast_exp2(ldg_cg_f32(p.ws_lse + (size_t)sl * p.rows + r) - M);
+                const float w = fast_exp2(ldg_cg_f32(p.ws_lse + (size_t)sl * p.rows + r) - mm);
                 const float4 x = ldg_cg_f32x4(p.ws_o + ((size_t)sl * p.rows + r) * D + c4 * 4);
                 acc.x += w * x.x;
                 acc.y += w * x.y;
@@ -611,7 +727,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                 den += w;
               }
             }
-            (void)np;
             const float invd = den > 0.f ? 1.f / den : 0.f;
             const int t = r / p.group, hq = sg.g * p.group + (r - t * p.group);
             const size_t orow = ((size_t)lb * p.n_q + t) * p.n_q_heads + hq;
@@ -619,19 +734,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             packed.x = pack_bf16x2(acc.x * invd, acc.y * invd);
             packed.y = pack_bf16x2(acc.z * invd, acc.w * invd);
             *reinterpret_cast<uint2*>(p.out + orow * D + c4 * 4) = packed;
-            if (p.lse && c4 == 0) p.lse[orow] = den > 0.f ? (M + log2f(den)) * kLn2 : -INFINITY;
+            if (p.lse && c4 == 0) p.lse[orow] = den > 0.f ? (mm + log2f(den)) * kLn2 : -INFINITY;
           }
         }
       }
-      // next segment
-      {
-        const int64_t nf = sg.item_begin + sg.tile0 + sg.n_tiles;
-        c.start(nf, T1, prefix, p.batch, hkv);
-        c.seg_idx = seg_idx + 1;
-      }
+      i0 += sg.n_tiles;
+      c.next_segment(prefix, p.batch, hkv);
     }
   softmax_done:
-    if (!ok && p.d_status && st == 0) *p.d_status = SPECVLM_ERR_TIMEOUT;
+    if (!ok && p.d_status && gt == 0) *p.d_status = SPECVLM_ERR_TIMEOUT;
 #undef SM_WAIT
   }
 
@@ -640,7 +751,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   __syncthreads();
   if (warp == 1) {
     tc_fence_after_sync();
-    tmem_dealloc(tmem_base, kTmemCols);
+    tmem_dealloc(tmem_base, C::TMEM_COLS);
   }
 }
 
@@ -660,14 +771,14 @@ size_t attn_tc_ws_bytes(const specvlm_kv_t* kv, int32_t batch, int rows) {
          round_up((size_t)2 * grid * rows * sizeof(float), 256) + round_up(items * sizeof(int32_t), 256);
 }
 
-template <int D, int STAGES>
+template <int D, int M>
 static int32_t launch_tc(const CUtensorMap& tk, const CUtensorMap& tv, const AttnTcParams& p, int grid,
                          cudaStream_t st) {
-  using L = TcLayout<D, STAGES>;
-  auto kern = attn_tc_kernel<D, STAGES>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL) != cudaSuccess)
+  using C = TcCfg<D, M>;
+  auto kern = attn_tc_kernel<D, M>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::TOTAL) != cudaSuccess)
     return SPECVLM_ERR_CUDA;
-  kern<<<grid, 224, L::TOTAL, st>>>(tk, tv, p);
+  kern<<<grid, kTcThreads, C::TOTAL, st>>>(tk, tv, p);
   return launch_status();
 }
 
@@ -715,7 +826,9 @@ int32_t attn_tc_launch(const specvlm_kv_t* kv, const void* q, int32_t batch, int
   p.scale_log2 = sm_scale * kLog2e;
 
   if (cudaMemsetAsync(p.ws_cnt, 0, (size_t)items * sizeof(int32_t), st) != cudaSuccess) return SPECVLM_ERR_CUDA;
-  return kv->head_dim == 128 ? launch_tc<128, 4>(tk, tv, p, grid, st) : launch_tc<64, 8>(tk, tv, p, grid, st);
+  if (kv->head_dim == 128)
+    return rows <= 64 ? launch_tc<128, 64>(tk, tv, p, grid, st) : launch_tc<128, 128>(tk, tv, p, grid, st);
+  return rows <= 64 ? launch_tc<64, 64>(tk, tv, p, grid, st) : launch_tc<64, 128>(tk, tv, p, grid, st);
 }
 
 }  // namespace specvlm
