@@ -3,23 +3,24 @@
 //
 // One persistent CTA per SM streams a contiguous slice of the flat (layer, sequence, KV head, tile)
 // list (attn_sched.h), so the cache is read exactly once, every SM moves the same number of bytes
-// and only two partial results per CTA ever touch scratch memory.
+// and only two partial results per CTA ever touch scratch memory.  A tile is 128 tokens: two
+// 64-token sub-tiles (one cache page each) as the TMA moves them.
 //
 // Roles inside a CTA (12 warps = 3 warpgroups; the first gives registers to the other two):
-//   warp 0     TMA producer: 64-token K tiles and V tiles, HBM -> two shared-memory rings (128-byte
-//              swizzle).  K and V have rings of their own because a K tile is free again as soon
-//              as S = Q K^T has been computed, long before its V tile.
+//   warp 0     TMA producer: the item's query rows, 64-token K sub-tiles into pair slots (a K tile
+//              must be 128 contiguous rows for the N = 128 product), V sub-tiles into a ring of
+//              single slots.  K and V have rings of their own because a K tile is free again as
+//              soon as S = Q K^T has been computed, long before its V tiles.
 //   warp 1     issues S = Q K^T (one thread, tcgen05.mma, accumulator in TMEM)
-//   warp 2     issues O += P V (one thread); two issuers, because one thread cannot issue both
-//              chains and poll their barriers within a tile's memory time
-//   warp 3     query loader: the item's query rows -> the swizzled A-operand tile, one item ahead
+//   warp 2     issues O += P V (one thread)
 //   warps 4-7  softmax group 0: the even tiles of the slice
 //   warps 8-11 softmax group 1: the odd tiles.  Each group has its own S buffer, P buffer, running
 //              (max, sum) and its own O accumulator; the two are merged once per item.
+// 128-token tiles keep the two issuing threads, whose per-tile cost in barrier round trips is
+// fixed, below the time HBM needs to deliver a tile.
 // The GQA group's heads times the query tokens are the M rows of the tiles: M = 64 when they fit
-// (rows 16c..16c+15 live in TMEM lanes 32c..32c+15), else M = 128 (row r in lane
-// 32*((r/16)%4) + 16*(r/64) + r%16); either way 16-row chunks are spread over the four warps of a
-// group, since a warp can only read its own 32 lanes.
+// (row r lives in TMEM lane 32 (r / 16) + r % 16), else M = 128 (row r in lane r); a softmax warp
+// owns the rows of its 32 TMEM lanes.
 //
 // The running maximum of a row is only raised when a tile's maximum exceeds it by more than 2^8; O
 // is then rescaled in place in TMEM.  Probabilities stay below 2^8, well inside bf16 / fp32 range,
@@ -31,8 +32,7 @@
 namespace specvlm {
 
 struct AttnTcParams {
-  const __nv_bfloat16* q;     // [L][B][n_q][Hq][D]
-  __nv_bfloat16* out;         // same shape
+  __nv_bfloat16* out;         // [L][B][n_q][Hq][D]
   float* lse;                 // [L][B][n_q][Hq] or null
   float* ws_o;                // partial results: [2 * grid][rows][D], normalised
   float* ws_lse;              // [2 * grid][rows], log2 units
@@ -46,6 +46,7 @@ struct AttnTcParams {
 };
 
 constexpr float kRescaleThreshold = 8.f;   // log2 units
+constexpr int kBigTokens = 2 * kTileTokens;          // tokens per MMA tile
 constexpr int kTcThreads = 384;
 constexpr int kRegsLight = 96, kRegsSoftmax = 200;   // 128 * 96 + 256 * 200 <= 64 K registers
 
@@ -84,11 +85,6 @@ __device__ __forceinline__ void tmem_st_16x256b_x8(uint32_t taddr, const uint32_
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-__device__ __forceinline__ uint4 ldg_nc_v4(const void* p) {
-  uint4 v;
-  asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-  return v;
-}
 __device__ __forceinline__ float ldg_cg_f32(const float* p) {
   float v;
   asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p));
@@ -126,22 +122,25 @@ struct SliceCursor {
   }
 };
 
+__device__ __forceinline__ int clamp_len(int n, int max_len) { return n < 0 ? 0 : (n > max_len ? max_len : n); }
+
 // Shared-memory plan.  A small region (barriers, flags, per-sequence tile counts, the softmax
 // groups' row statistics) sits at the start of the dynamic shared memory; the tile rings and the
 // operand tiles follow at the next 1024-byte boundary.
 template <int D, int M>
 struct TcCfg {
-  static constexpr int KT_BYTES = kTileTokens * D * 2;          // one K (or V) tile
-  static constexpr int NK = D == 128 ? (M == 64 ? 5 : 3) : 8;   // K ring stages
-  static constexpr int NV = D == 128 ? (M == 64 ? 6 : 4) : 8;   // V ring stages
+  static constexpr int SUB_BYTES = kTileTokens * D * 2;         // one 64-token K (or V) sub-tile
+  static constexpr int NKP = D == 128 ? 2 : 3;                  // K ring: pair slots (128 tokens)
+  static constexpr int NVS = D == 128 ? (M == 64 ? 6 : 3) : 6;  // V ring: single slots (64 tokens)
+  static constexpr int NQ = (D == 128 && M == 128) ? 1 : 2;     // query buffers
   static constexpr int Q_BYTES = M * D * 2;                     // A operand of S = Q K^T
-  static constexpr int P_BYTES = M * kTileTokens * 2;           // A operand of O += P V
+  static constexpr int P_BYTES = M * kBigTokens * 2;            // A operand of O += P V
   static constexpr int OFF_K = 0;
-  static constexpr int OFF_V = OFF_K + NK * KT_BYTES;
-  static constexpr int OFF_Q = OFF_V + NV * KT_BYTES;
-  static constexpr int OFF_P = OFF_Q + 2 * Q_BYTES;
+  static constexpr int OFF_V = OFF_K + NKP * 2 * SUB_BYTES;
+  static constexpr int OFF_Q = OFF_V + NVS * SUB_BYTES;
+  static constexpr int OFF_P = OFF_Q + NQ * Q_BYTES;
   static constexpr int BIG = OFF_P + 2 * P_BYTES;
-  static constexpr int N_BARS = 2 * NK + 2 * NV + 17;
+  static constexpr int N_BARS = 2 * NKP + 2 * NVS + 17;
   static constexpr int SM_BAR = 0;
   static constexpr int SM_MISC = SM_BAR + 8 * N_BARS;
   static constexpr int SM_PREFIX = SM_MISC + 32;
@@ -151,19 +150,20 @@ struct TcCfg {
   static constexpr int kMaxSmem = 232448;                       // 227 KB
   // a spare KB for a base that is not 1024-byte aligned, where there is room for it
   static constexpr int TOTAL = SMALL + BIG + (SMALL + BIG + 1024 <= kMaxSmem ? 1024 : 0);
-  static constexpr uint32_t TMEM_COLS = 128 + 2 * D <= 256 ? 256 : 512;   // S0 | S1 | O0 | O1
+  static constexpr uint32_t COL_S = 0, COL_O = 2 * kBigTokens;  // TMEM: S of group g at 128 g, O at 256 + D g
+  static constexpr uint32_t TMEM_COLS = 512;
   static_assert(SMALL + BIG <= kMaxSmem, "shared-memory plan does not fit");
 };
 
 template <int D, int M>
 __global__ void __launch_bounds__(kTcThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
-               const __grid_constant__ AttnTcParams p) {
+               const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ AttnTcParams p) {
   using C = TcCfg<D, M>;
-  constexpr int KT_BYTES = C::KT_BYTES, NK = C::NK, NV = C::NV, Q_BYTES = C::Q_BYTES, P_BYTES = C::P_BYTES;
+  constexpr int SUB_BYTES = C::SUB_BYTES, NKP = C::NKP, NVS = C::NVS, NQ = C::NQ;
+  constexpr int Q_BYTES = C::Q_BYTES, P_BYTES = C::P_BYTES;
   constexpr int NH = M / 64;                          // 16-lane halves a softmax warp may own
-  constexpr uint32_t kColS = 0, kColO = 128;          // TMEM columns: S of group g at 64 g, O at 128 + D g
-  constexpr uint32_t kIdescQK = umma_idesc_bf16(M, kTileTokens, false, false);
+  constexpr uint32_t kIdescQK = umma_idesc_bf16(M, kBigTokens, false, false);
   constexpr uint32_t kIdescPV = umma_idesc_bf16(M, D, false, true);   // V tile: channels run along the row
 
   extern __shared__ uint8_t smem_raw[];
@@ -172,9 +172,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   uint8_t* const big_ptr = smem_raw + (big - raw_addr);
   const uint32_t k_sm = big + C::OFF_K, v_sm = big + C::OFF_V, q_sm = big + C::OFF_Q, p_sm = big + C::OFF_P;
   const uint32_t bar0 = raw_addr + C::SM_BAR;
-  const uint32_t bar_k_full = bar0, bar_k_empty = bar_k_full + 8 * NK;
-  const uint32_t bar_v_full = bar_k_empty + 8 * NK, bar_v_empty = bar_v_full + 8 * NV;
-  const uint32_t bar_q_full = bar_v_empty + 8 * NV;    // [2]
+  const uint32_t bar_k_full = bar0, bar_k_empty = bar_k_full + 8 * NKP;
+  const uint32_t bar_v_full = bar_k_empty + 8 * NKP, bar_v_empty = bar_v_full + 8 * NVS;
+  const uint32_t bar_q_full = bar_v_empty + 8 * NVS;   // [2]
   const uint32_t bar_q_empty = bar_q_full + 16;        // [2]
   const uint32_t bar_s_full = bar_q_empty + 16;        // [2]: one per softmax group
   const uint32_t bar_s_empty = bar_s_full + 16;        // [2]
@@ -202,11 +202,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 
   // ------------------------------------------------------------------ set-up
   if (tid == 0) {
-    for (int s = 0; s < NK; ++s) {
+    for (int s = 0; s < NKP; ++s) {
       mbar_init(bar_k_full + 8 * s, 1);
       mbar_init(bar_k_empty + 8 * s, 1);
     }
-    for (int s = 0; s < NV; ++s) {
+    for (int s = 0; s < NVS; ++s) {
       mbar_init(bar_v_full + 8 * s, 1);
       mbar_init(bar_v_empty + 8 * s, 1);
     }
@@ -232,11 +232,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), C::TMEM_COLS);
   // tiles per sequence, then their running sum
   for (int b = tid; b < p.batch; b += blockDim.x) {
-    int n = p.seq_lens[b];
-    n = n < 0 ? 0 : (n > p.max_seq_len ? p.max_seq_len : n);
-    prefix[b + 1] = (n + kTileTokens - 1) / kTileTokens;
+    const int n = clamp_len(p.seq_lens[b], p.max_seq_len);
+    prefix[b + 1] = (n + kBigTokens - 1) / kBigTokens;
     if (n == 0) *any_empty = 1;
   }
+  // query rows that no item uses stay zero (the TMA only ever writes the first `rows` rows)
+  for (int idx = tid; idx < NQ * Q_BYTES / 16; idx += blockDim.x)
+    *reinterpret_cast<uint4*>(big_ptr + C::OFF_Q + idx * 16) = make_uint4(0, 0, 0, 0);
+  fence_proxy_async();
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 0) {
@@ -264,6 +267,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   const int64_t T0 = active ? slice_begin(cta, n_active, total) : 0;
   const int64_t T1 = active ? slice_begin(cta + 1, n_active, total) : 0;
   const int n_items = p.n_layers * p.batch * hkv;
+  const int n_my = (int)(T1 - T0);
 
   if (warp == 0) {
     // ================================================================ TMA producer
@@ -271,38 +275,67 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     if (lane == 0 && active) {
       tma_prefetch_desc(&tm_k);
       tma_prefetch_desc(&tm_v);
+      tma_prefetch_desc(&tm_q);
       const uint64_t policy = l2_policy_evict_first();
-      const int tiles_per_block = p.block_table ? p.block_tokens / kTileTokens : 1;
+      const uint64_t policy_q = l2_policy_evict_last();
+      const int subs_per_block = p.block_table ? p.block_tokens / kTileTokens : 1;
       SliceCursor c;
       c.start(T0, T1, prefix, p.batch, hkv);
       bool ok = true;
-      int i = 0, k_issued = 0, v_issued = 0;
+      int i = 0, vc = 0, k_issued = 0;      // tiles, V sub-tiles, K tiles issued so far
       while (c.f < T1 && ok) {
         const Segment sg = c.sg;
+        // the item's query rows: a box of (64 channels) x (group heads) x (n_q tokens) per 64-channel block
+        {
+          const int qb = c.seg_idx % NQ;
+          if (c.seg_idx >= NQ) ok = mbar_wait(bar_q_empty + 8 * qb, ((c.seg_idx / NQ) - 1) & 1, abort_flag);
+          if (!ok) break;
+          mbar_arrive_expect_tx(bar_q_full + 8 * qb, (uint32_t)p.rows * 128u * (D / 64));
+#pragma unroll
+          for (int h = 0; h < D / 64; ++h)
+            tma_load_5d(q_sm + qb * Q_BYTES + h * (M * 128), &tm_q, bar_q_full + 8 * qb, h * 64, 0, 0, sg.g,
+                        sg.layer * p.batch + sg.b, policy_q);
+        }
+        const int n_sub_seq = (clamp_len(p.seq_lens[sg.b], p.max_seq_len) + kTileTokens - 1) / kTileTokens;
         const int32_t* table = p.block_table ? p.block_table + (size_t)sg.b * p.max_blocks : nullptr;
-        int blk_next = table ? __ldg(table + sg.tile0 / tiles_per_block) : sg.b;
-        for (int j = 0; j < sg.n_tiles; ++j, ++i) {
-          const int tile = sg.tile0 + j;
-          const int blk = blk_next;
-          if (table && j + 1 < sg.n_tiles) blk_next = __ldg(table + (tile + 1) / tiles_per_block);   // one tile ahead
-          const int tok = table ? (tile % tiles_per_block) * kTileTokens : tile * kTileTokens;
-          const int ks = i % NK, vs = i % NV;
-          if (i >= NK) ok = mbar_wait(bar_k_empty + 8 * ks, ((i / NK) - 1) & 1, abort_flag);
+        int blk[2], blk_next[2] = {sg.b, sg.b};
+        if (table) {
+          const int s0 = 2 * sg.tile0;
+          blk_next[0] = __ldg(table + s0 / subs_per_block);
+          blk_next[1] = s0 + 1 < n_sub_seq ? __ldg(table + (s0 + 1) / subs_per_block) : 0;
+        }
+        for (int j = 0; j < sg.n_tiles && ok; ++j, ++i) {
+          const int s0 = 2 * (sg.tile0 + j);                    // first sub-tile of this tile
+          const int n_sub = n_sub_seq - s0 < 2 ? n_sub_seq - s0 : 2;
+          blk[0] = blk_next[0];
+          blk[1] = blk_next[1];
+          if (table && j + 1 < sg.n_tiles) {                    // table entries of the next tile, one tile ahead
+            blk_next[0] = __ldg(table + (s0 + 2) / subs_per_block);
+            blk_next[1] = s0 + 3 < n_sub_seq ? __ldg(table + (s0 + 3) / subs_per_block) : 0;
+          }
+          const int kp = i % NKP;
+          if (i >= NKP) ok = mbar_wait(bar_k_empty + 8 * kp, ((i / NKP) - 1) & 1, abort_flag);
           if (!ok) break;
-          mbar_arrive_expect_tx(bar_k_full + 8 * ks, KT_BYTES);
+          mbar_arrive_expect_tx(bar_k_full + 8 * kp, n_sub * SUB_BYTES);
+          for (int u = 0; u < n_sub; ++u) {
+            const int tok = table ? ((s0 + u) % subs_per_block) * kTileTokens : (s0 + u) * kTileTokens;
 #pragma unroll
-          for (int h = 0; h < D / 64; ++h)
-            tma_load_5d(k_sm + ks * KT_BYTES + h * (kTileTokens * 128), &tm_k, bar_k_full + 8 * ks, h * 64, tok, sg.g,
-                        blk, sg.layer, policy);
+            for (int h = 0; h < D / 64; ++h)      // K tile: [64-channel block][128 tokens][128 B]
+              tma_load_5d(k_sm + kp * 2 * SUB_BYTES + h * (kBigTokens * 128) + u * (kTileTokens * 128), &tm_k,
+                          bar_k_full + 8 * kp, h * 64, tok, sg.g, blk[u], sg.layer, policy);
+          }
           k_issued = i + 1;
-          if (i >= NV) ok = mbar_wait(bar_v_empty + 8 * vs, ((i / NV) - 1) & 1, abort_flag);
-          if (!ok) break;
-          mbar_arrive_expect_tx(bar_v_full + 8 * vs, KT_BYTES);
+          for (int u = 0; u < n_sub && ok; ++u, ++vc) {
+            const int vs = vc % NVS;
+            if (vc >= NVS) ok = mbar_wait(bar_v_empty + 8 * vs, ((vc / NVS) - 1) & 1, abort_flag);
+            if (!ok) break;
+            const int tok = table ? ((s0 + u) % subs_per_block) * kTileTokens : (s0 + u) * kTileTokens;
+            mbar_arrive_expect_tx(bar_v_full + 8 * vs, SUB_BYTES);
 #pragma unroll
-          for (int h = 0; h < D / 64; ++h)
-            tma_load_5d(v_sm + vs * KT_BYTES + h * (kTileTokens * 128), &tm_v, bar_v_full + 8 * vs, h * 64, tok, sg.g,
-                        blk, sg.layer, policy);
-          v_issued = i + 1;
+            for (int h = 0; h < D / 64; ++h)      // V sub-tile: [64-channel block][64 tokens][128 B]
+              tma_load_5d(v_sm + vs * SUB_BYTES + h * (kTileTokens * 128), &tm_v, bar_v_full + 8 * vs, h * 64, tok,
+                          sg.g, blk[u], sg.layer, policy);
+          }
         }
         c.next_segment(prefix, p.batch, hkv);
       }
@@ -310,11 +343,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         // a wait expired: report, then stay until this CTA's copies in flight have landed (bounded)
         if (p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
         const uint64_t t0 = global_timer_ns();
-        for (int k = k_issued > NK ? k_issued - NK : 0; k < k_issued; ++k)
-          while (!mbar_test_wait(bar_k_full + 8 * (k % NK), (k / NK) & 1) && global_timer_ns() - t0 < kWaitLimitNs) {
+        for (int k = k_issued > NKP ? k_issued - NKP : 0; k < k_issued; ++k)
+          while (!mbar_test_wait(bar_k_full + 8 * (k % NKP), (k / NKP) & 1) && global_timer_ns() - t0 < kWaitLimitNs) {
           }
-        for (int k = v_issued > NV ? v_issued - NV : 0; k < v_issued; ++k)
-          while (!mbar_test_wait(bar_v_full + 8 * (k % NV), (k / NV) & 1) && global_timer_ns() - t0 < kWaitLimitNs) {
+        for (int k = vc > NVS ? vc - NVS : 0; k < vc; ++k)
+          while (!mbar_test_wait(bar_v_full + 8 * (k % NVS), (k / NVS) & 1) && global_timer_ns() - t0 < kWaitLimitNs) {
           }
       }
     }
@@ -324,26 +357,25 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     if (lane == 0 && active) {
       SliceCursor c;
       c.start(T0, T1, prefix, p.batch, hkv);
-      const int n = (int)(T1 - T0);
       const uint64_t dq0 = umma_desc_sw128(q_sm, 16, 1024), dk0 = umma_desc_sw128(k_sm, 16, 1024);
       bool ok = true;
-      for (int i = 0; i < n; ++i) {
-        const int g = i & 1, ks = i % NK, qb = c.seg_idx & 1;
-        ok = mbar_wait(bar_k_full + 8 * ks, (i / NK) & 1, abort_flag);
-        if (ok && c.j == 0) ok = mbar_wait(bar_q_full + 8 * qb, (c.seg_idx >> 1) & 1, abort_flag);
+      for (int i = 0; i < n_my; ++i) {
+        const int g = i & 1, kp = i % NKP, qb = c.seg_idx % NQ;
+        ok = mbar_wait(bar_k_full + 8 * kp, (i / NKP) & 1, abort_flag);
+        if (ok && c.j == 0) ok = mbar_wait(bar_q_full + 8 * qb, (c.seg_idx / NQ) & 1, abort_flag);
         if (ok && i >= 2) ok = mbar_wait(bar_s_empty + 8 * g, ((i >> 1) - 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
-        const uint64_t da = umma_desc_advance(dq0, qb * Q_BYTES), db = umma_desc_advance(dk0, ks * KT_BYTES);
-        const uint32_t d_tmem = tmem_base + kColS + g * kTileTokens;
+        const uint64_t da = umma_desc_advance(dq0, qb * Q_BYTES), db = umma_desc_advance(dk0, kp * 2 * SUB_BYTES);
+        const uint32_t d_tmem = tmem_base + C::COL_S + g * kBigTokens;
 #pragma unroll
         for (int s = 0; s < D / 16; ++s)
           // 16 channels per step = 32 bytes along the swizzled 128-byte row; channels 64.. are the
-          // second 64-channel block of each tile
+          // second 64-channel block of each operand
           umma_bf16_ss(d_tmem, umma_desc_advance(da, (s >> 2) * (M * 128) + (s & 3) * 32),
-                       umma_desc_advance(db, (s >> 2) * (kTileTokens * 128) + (s & 3) * 32), kIdescQK, s > 0 ? 1u : 0u);
+                       umma_desc_advance(db, (s >> 2) * (kBigTokens * 128) + (s & 3) * 32), kIdescQK, s > 0 ? 1u : 0u);
         umma_commit(bar_s_full + 8 * g);
-        umma_commit(bar_k_empty + 8 * ks);
+        umma_commit(bar_k_empty + 8 * kp);
         if (c.last_of_segment()) umma_commit(bar_q_empty + 8 * qb);
         c.next_tile(prefix, p.batch, hkv);
       }
@@ -355,80 +387,44 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     if (lane == 0 && active) {
       SliceCursor c;
       c.start(T0, T1, prefix, p.batch, hkv);
-      const int n = (int)(T1 - T0);
       const uint64_t dp0 = umma_desc_sw128(p_sm, 16, 1024);
       const uint64_t dv0 = umma_desc_sw128(v_sm, kTileTokens * 128, 1024);   // 64-channel blocks 8 KB apart
       bool ok = true;
-      for (int i = 0; i < n; ++i) {
-        const int g = i & 1, vs = i % NV;
-        ok = mbar_wait(bar_v_full + 8 * vs, (i / NV) & 1, abort_flag);
+      int vc = 0, n_sub_seq = 0;
+      for (int i = 0; i < n_my; ++i) {
+        const int g = i & 1;
+        if (c.j == 0) n_sub_seq = (clamp_len(p.seq_lens[c.sg.b], p.max_seq_len) + kTileTokens - 1) / kTileTokens;
+        const int s0 = 2 * (c.sg.tile0 + c.j);
+        const int n_sub = n_sub_seq - s0 < 2 ? n_sub_seq - s0 : 2;
         // the first product of each group overwrites that group's O: the previous item must be out
-        if (ok && c.j < 2 && c.seg_idx >= 1) ok = mbar_wait(bar_o_empty, (c.seg_idx - 1) & 1, abort_flag);
+        if (c.j < 2 && c.seg_idx >= 1) ok = mbar_wait(bar_o_empty, (c.seg_idx - 1) & 1, abort_flag);
         if (ok) ok = mbar_wait(bar_p_full + 8 * g, (i >> 1) & 1, abort_flag);
         if (!ok) break;
-        tc_fence_after_sync();
-        const uint64_t da = umma_desc_advance(dp0, g * P_BYTES), db = umma_desc_advance(dv0, vs * KT_BYTES);
-        const uint32_t d_tmem = tmem_base + kColO + g * D;
-        const uint32_t acc0 = c.j >= 2 ? 1u : 0u;
+        const uint64_t da = umma_desc_advance(dp0, g * P_BYTES);
+        const uint32_t d_tmem = tmem_base + C::COL_O + g * D;
+        for (int u = 0; u < n_sub && ok; ++u, ++vc) {
+          const int vs = vc % NVS;
+          ok = mbar_wait(bar_v_full + 8 * vs, (vc / NVS) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const uint64_t dau = umma_desc_advance(da, u * (M * 128)), db = umma_desc_advance(dv0, vs * SUB_BYTES);
+          const uint32_t acc0 = (c.j >= 2 || u > 0) ? 1u : 0u;
 #pragma unroll
-        for (int kt = 0; kt < kTileTokens / 16; ++kt)
-          // 16 tokens per step: 32 bytes along P's row, 16 rows of 128 bytes down the V tile
-          umma_bf16_ss(d_tmem, umma_desc_advance(da, kt * 32), umma_desc_advance(db, kt * 2048), kIdescPV,
-                       kt > 0 ? 1u : acc0);
+          for (int kt = 0; kt < kTileTokens / 16; ++kt)
+            // 16 tokens per step: 32 bytes along P's row, 16 rows of 128 bytes down the V sub-tile
+            umma_bf16_ss(d_tmem, umma_desc_advance(dau, kt * 32), umma_desc_advance(db, kt * 2048), kIdescPV,
+                         kt > 0 ? 1u : acc0);
+          umma_commit(bar_v_empty + 8 * vs);
+        }
+        if (!ok) break;
         umma_commit(bar_p_empty + 8 * g);
-        umma_commit(bar_v_empty + 8 * vs);
         if (c.last_of_segment()) umma_commit(bar_o_full);
         c.next_tile(prefix, p.batch, hkv);
       }
       if (!ok && p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
     }
   } else if (warp == 3) {
-    // ================================================================ query loader
     setmaxnreg_dec<kRegsLight>();
-    if (active) {
-      for (int idx = lane; idx < 2 * Q_BYTES / 16; idx += 32)      // rows no item uses stay zero
-        *reinterpret_cast<uint4*>(big_ptr + C::OFF_Q + idx * 16) = make_uint4(0, 0, 0, 0);
-      __syncwarp();
-      SliceCursor c;
-      c.start(T0, T1, prefix, p.batch, hkv);
-      bool ok = true;
-      constexpr int CPR = D / 8;                                   // 16-byte chunks per row
-      const int n_chunks = p.rows * CPR;
-      while (c.f < T1 && ok) {
-        const int qb = c.seg_idx & 1;
-        if (c.seg_idx >= 2)
-          ok = __all_sync(0xffffffffu, mbar_wait(bar_q_empty + 8 * qb, ((c.seg_idx >> 1) - 1) & 1, abort_flag));
-        if (!ok) break;
-        const int lb = c.sg.layer * p.batch + c.sg.b;
-        uint8_t* const qbuf = big_ptr + C::OFF_Q + qb * Q_BYTES;
-        for (int c0 = 0; c0 < n_chunks; c0 += 32 * 8) {
-          uint4 val[8];
-#pragma unroll
-          for (int u = 0; u < 8; ++u) {                            // all loads of a batch in flight together
-            const int ci = c0 + u * 32 + lane;
-            if (ci < n_chunks) {
-              const int r = ci / CPR, c16 = ci - r * CPR;
-              const int t = r / p.group, hh = r - t * p.group;
-              val[u] = ldg_nc_v4(p.q + (((size_t)lb * p.n_q + t) * p.n_q_heads + c.sg.g * p.group + hh) * D + c16 * 8);
-            }
-          }
-#pragma unroll
-          for (int u = 0; u < 8; ++u) {
-            const int ci = c0 + u * 32 + lane;
-            if (ci < n_chunks) {
-              const int r = ci / CPR, c16 = ci - r * CPR;
-              // row of the A operand: r itself for M = 64, the row's TMEM lane for M = 128
-              const int m = M == 64 ? r : ((((r >> 4) & 3) << 5) + ((r >> 6) << 4) + (r & 15));
-              *reinterpret_cast<uint4*>(qbuf + (c16 >> 3) * (M * 128) + m * 128 + (((c16 & 7) ^ (m & 7)) << 4)) = val[u];
-            }
-          }
-        }
-        fence_proxy_async();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_q_full + 8 * qb);
-        c.next_segment(prefix, p.batch, hkv);
-      }
-    }
   } else {
     // ================================================================ softmax / epilogue (warps 4..11)
     setmaxnreg_inc<kRegsSoftmax>();
@@ -436,8 +432,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     const int quarter = warp & 3;                 // TMEM lanes [32 * quarter, +32)
     const int gt = (warp & 3) * 32 + lane;        // 0..127 inside the group
     const int st = grp * 128 + gt;                // 0..255 over both groups
-    const int nh = (p.rows > 16 * quarter ? 1 : 0) + (NH > 1 && p.rows > 16 * (quarter + 4) ? 1 : 0);
     const int lr = lane >> 2, lc = (lane & 3) * 2;   // row inside a 16-lane half (and +8), first column of a pair
+    // rows of this warp: half h covers item rows row0(h) + [0, 16), held in TMEM lanes 32 * quarter + 16 h + [0, 16)
+    auto row0 = [&](int h) { return M == 64 ? 16 * quarter : 32 * quarter + 16 * h; };
+    const int nh = (p.rows > row0(0) ? 1 : 0) + (NH > 1 && p.rows > row0(1) ? 1 : 0);
 
     // sequences without any token: their outputs are zero, their LSE -inf
     if (*any_empty) {
@@ -458,6 +456,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     c.start(T0, T1, prefix, p.batch, hkv);
     bool ok = true;
     int i0 = 0;           // index (inside the slice) of the current segment's first tile
+    int vc0 = 0;          // V sub-tiles of the slice before the current segment
     int n_partial = 0;    // partial epilogues so far
 #define SM_WAIT(bar, parity)                                                        \
   do {                                                                              \
@@ -468,16 +467,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     while (c.f < T1) {
       const Segment sg = c.sg;
       const int seg_idx = c.seg_idx;
-      int kv_len = p.seq_lens[sg.b];
-      kv_len = kv_len < 0 ? 0 : (kv_len > p.max_seq_len ? p.max_seq_len : kv_len);
-      // rows of this thread: half h is the 16-row chunk quarter + 4h, rows 16 * chunk + lr and + 8
+      const int kv_len = clamp_len(p.seq_lens[sg.b], p.max_seq_len);
+      const int n_sub_seq = (kv_len + kTileTokens - 1) / kTileTokens;
       int lim[NH][2];
       float m_used[NH][2], l_sum[NH][2];
 #pragma unroll
       for (int h = 0; h < NH; ++h)
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
-          const int r = 16 * (quarter + 4 * h) + lr + 8 * e;
+          const int r = row0(h) + lr + 8 * e;
           lim[h][e] = r < p.rows ? kv_len - p.n_q + r / p.group + 1 : 0;
           m_used[h][e] = -INFINITY;
           l_sum[h][e] = 0.f;
@@ -485,40 +483,50 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 
       for (int j = (i0 + grp) & 1; j < sg.n_tiles; j += 2) {
         const int i = i0 + j;
-        const int tile_tok0 = (sg.tile0 + j) * kTileTokens;
-        const bool need_mask = tile_tok0 + kTileTokens > kv_len - p.n_q + 1;
+        const int tile_tok0 = (sg.tile0 + j) * kBigTokens;
+        const bool need_mask = tile_tok0 + kBigTokens > kv_len - p.n_q + 1;
         SM_WAIT(bar_s_full + 8 * grp, (i >> 1) & 1);
         tc_fence_after_sync();
-        uint32_t v[NH][32];
-#pragma unroll
-        for (int h = 0; h < NH; ++h)
-          if (h < nh) tmem_ld_16x256b_x8(tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + kColS + grp * kTileTokens, v[h]);
-        tmem_ld_wait();
-        tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_s_empty + 8 * grp);
-        // the group's previous product has completed: P may be overwritten, O may be rescaled
-        if (i >= 2) SM_WAIT(bar_p_empty + 8 * grp, ((i >> 1) - 1) & 1);
-
+        if (nh == 0) {
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_s_empty + 8 * grp);
+        }
 #pragma unroll
         for (int h = 0; h < NH; ++h) {
           if (h >= nh) break;
-          float s[32];
+          // S rows of this half: 128 columns = two loads of 64
+          uint32_t v0[32], v1[32];
+          const uint32_t saddr = tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + C::COL_S + grp * kBigTokens;
+          tmem_ld_16x256b_x8(saddr, v0);
+          tmem_ld_16x256b_x8(saddr + 64, v1);
+          tmem_ld_wait();
+          if (h == nh - 1) {
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_s_empty + 8 * grp);
+          }
+          // the group's previous product has completed: P may be overwritten, O may be rescaled
+          if (h == 0 && i >= 2) SM_WAIT(bar_p_empty + 8 * grp, ((i >> 1) - 1) & 1);
+
           float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
           if (need_mask) {
 #pragma unroll
             for (int k = 0; k < 32; ++k) {
               const int tok = tile_tok0 + (k >> 2) * 8 + lc + (k & 1);
-              const float x = tok < lim[h][(k >> 1) & 1] ? __uint_as_float(v[h][k]) * p.scale_log2 : -INFINITY;
-              s[k] = x;
-              mx[k & 3] = fmaxf(mx[k & 3], x);
+              const int lm = lim[h][(k >> 1) & 1];
+              const float x0 = tok < lm ? __uint_as_float(v0[k]) * p.scale_log2 : -INFINITY;
+              const float x1 = tok + kTileTokens < lm ? __uint_as_float(v1[k]) * p.scale_log2 : -INFINITY;
+              v0[k] = __float_as_uint(x0);
+              v1[k] = __float_as_uint(x1);
+              mx[k & 3] = fmaxf(mx[k & 3], fmaxf(x0, x1));
             }
           } else {
 #pragma unroll
             for (int k = 0; k < 32; ++k) {
-              const float x = __uint_as_float(v[h][k]) * p.scale_log2;
-              s[k] = x;
-              mx[k & 3] = fmaxf(mx[k & 3], x);
+              const float x0 = __uint_as_float(v0[k]) * p.scale_log2, x1 = __uint_as_float(v1[k]) * p.scale_log2;
+              v0[k] = __float_as_uint(x0);
+              v1[k] = __float_as_uint(x1);
+              mx[k & 3] = fmaxf(mx[k & 3], fmaxf(x0, x1));
             }
           }
           float mx0 = fmaxf(mx[0], mx[1]), mx1 = fmaxf(mx[2], mx[3]);
@@ -544,7 +552,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 #pragma unroll
               for (int cc = 0; cc < D / 64; ++cc) {
                 uint32_t o[32];
-                const uint32_t oaddr = tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + kColO + grp * D + cc * 64;
+                const uint32_t oaddr = tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + C::COL_O + grp * D + cc * 64;
                 tmem_ld_16x256b_x8(oaddr, o);
                 tmem_ld_wait();
 #pragma unroll
@@ -559,28 +567,37 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           const float mu0 = m_used[h][0] == -INFINITY ? 0.f : m_used[h][0];
           const float mu1 = m_used[h][1] == -INFINITY ? 0.f : m_used[h][1];
           float ps[4] = {0.f, 0.f, 0.f, 0.f};
-          // rows of the A operand of O += P V: the item's row for M = 64, the TMEM lane for M = 128
-          const int m0 = (M == 64 ? 16 * quarter : 32 * quarter + 16 * h) + lr, m1 = m0 + 8;
+          // rows of the A operand of O += P V: the item's rows
+          const int m0 = row0(h) + lr, m1 = m0 + 8;
           const uint32_t prow0 = p_sm + grp * P_BYTES + m0 * 128 + lc * 2;
           const uint32_t prow1 = p_sm + grp * P_BYTES + m1 * 128 + lc * 2;
 #pragma unroll
-          for (int jj = 0; jj < 8; ++jj) {
-            const float p0 = fast_exp2(s[4 * jj] - mu0), p1 = fast_exp2(s[4 * jj + 1] - mu0);
-            const float p2 = fast_exp2(s[4 * jj + 2] - mu1), p3 = fast_exp2(s[4 * jj + 3] - mu1);
-            ps[jj & 1] += p0 + p1;
-            ps[2 + (jj & 1)] += p2 + p3;
-            asm volatile("st.shared.b32 [%0], %1;" ::"r"(prow0 + ((jj ^ (m0 & 7)) << 4)), "r"(pack_bf16x2(p0, p1)) : "memory");
-            asm volatile("st.shared.b32 [%0], %1;" ::"r"(prow1 + ((jj ^ (m1 & 7)) << 4)), "r"(pack_bf16x2(p2, p3)) : "memory");
+          for (int half = 0; half < 2; ++half) {          // the tile's two 64-token blocks
+#pragma unroll
+            for (int jj = 0; jj < 8; ++jj) {
+              const uint32_t* vv = half ? v1 : v0;
+              const float p0 = fast_exp2(__uint_as_float(vv[4 * jj]) - mu0), p1 = fast_exp2(__uint_as_float(vv[4 * jj + 1]) - mu0);
+              const float p2 = fast_exp2(__uint_as_float(vv[4 * jj + 2]) - mu1), p3 = fast_exp2(__uint_as_float(vv[4 * jj + 3]) - mu1);
+              ps[jj & 1] += p0 + p1;
+              ps[2 + (jj & 1)] += p2 + p3;
+              asm volatile("st.shared.b32 [%0], %1;" ::"r"(prow0 + half * (M * 128) + ((jj ^ (m0 & 7)) << 4)),
+                           "r"(pack_bf16x2(p0, p1)) : "memory");
+              asm volatile("st.shared.b32 [%0], %1;" ::"r"(prow1 + half * (M * 128) + ((jj ^ (m1 & 7)) << 4)),
+                           "r"(pack_bf16x2(p2, p3)) : "memory");
+            }
           }
           l_sum[h][0] += ps[0] + ps[1];
           l_sum[h][1] += ps[2] + ps[3];
         }
-        if (tile_tok0 + kTileTokens > kv_len) {
-          // last, ragged tile: the V rows past the end of the sequence hold whatever the page held;
+        if (nh == 0 && i >= 2) SM_WAIT(bar_p_empty + 8 * grp, ((i >> 1) - 1) & 1);
+        if (tile_tok0 + kBigTokens > kv_len && (kv_len & (kTileTokens - 1)) != 0) {
+          // the sequence ends inside a sub-tile: the V rows past its end hold whatever the page held;
           // clear them so that a zero probability times a stale non-finite value cannot reach O
-          SM_WAIT(bar_v_full + 8 * (i % NV), (i / NV) & 1);
-          uint8_t* vt = big_ptr + C::OFF_V + (i % NV) * KT_BYTES;
-          const int first = kv_len - tile_tok0;
+          const int last_sub = n_sub_seq - 1;
+          const int vcl = vc0 + 2 * j + (last_sub - 2 * (sg.tile0 + j));   // that sub-tile's place in the V ring
+          SM_WAIT(bar_v_full + 8 * (vcl % NVS), (vcl / NVS) & 1);
+          uint8_t* vt = big_ptr + C::OFF_V + (vcl % NVS) * SUB_BYTES;
+          const int first = kv_len - last_sub * kTileTokens;
           for (int idx = gt; idx < (kTileTokens - first) * (D / 8); idx += 128) {
             const int t = first + idx / (D / 8), c16 = idx % (D / 8);
             *reinterpret_cast<uint4*>(vt + (c16 >> 3) * (kTileTokens * 128) + t * 128 + (c16 & 7) * 16) =
@@ -601,7 +618,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       // statistics slots alternate between segments: a group may reach its next write while the
       // other one still reads this segment's values
       float2* const seg_stats = stats + (seg_idx & 1) * 2 * M;
-      auto srow = [&](int h) { return (M == 64 ? 16 * quarter : 32 * quarter + 16 * h) + lr; };
 #pragma unroll
       for (int h = 0; h < NH; ++h) {
         if (h >= nh) break;
@@ -610,7 +626,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           float lt = l_sum[h][e];
           lt += __shfl_xor_sync(0xffffffffu, lt, 1);
           lt += __shfl_xor_sync(0xffffffffu, lt, 2);
-          if ((lane & 3) == 0) seg_stats[grp * M + srow(h) + 8 * e] = make_float2(m_used[h][e], lt);
+          if ((lane & 3) == 0) seg_stats[grp * M + row0(h) + lr + 8 * e] = make_float2(m_used[h][e], lt);
         }
       }
       __syncwarp();
@@ -626,7 +642,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         float w0[2], w1[2], lse2[2];
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
-          const int ln = srow(h) + 8 * e;
+          const int ln = row0(h) + lr + 8 * e;
           const float2 s0 = seg_stats[ln], s1 = seg_stats[M + ln];
           const float l0 = has0 ? s0.y : 0.f, l1 = has1 ? s1.y : 0.f;
           const float ma = l0 > 0.f ? s0.x : -INFINITY, mb = l1 > 0.f ? s1.x : -INFINITY;
@@ -643,13 +659,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           if ((cc & 1) != (D == 128 ? grp : 0)) continue;       // the groups share the column chunks
           if (D == 64 && grp == 1) continue;
           uint32_t oa[32], ob[32];
-          const uint32_t oaddr = tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + kColO + cc * 64;
+          const uint32_t oaddr = tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + C::COL_O + cc * 64;
           if (has0) tmem_ld_16x256b_x8(oaddr, oa);
           if (has1) tmem_ld_16x256b_x8(oaddr + D, ob);
           tmem_ld_wait();
 #pragma unroll
           for (int e = 0; e < 2; ++e) {
-            const int r = 16 * (quarter + 4 * h) + lr + 8 * e;
+            const int r = row0(h) + lr + 8 * e;
             if (r >= p.rows) continue;
             float res[16];
 #pragma unroll
@@ -738,6 +754,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           }
         }
       }
+      // sub-tiles of this segment: two per tile, except that the item's last tile may hold one
+      {
+        const int s_end = 2 * (sg.tile0 + sg.n_tiles);
+        vc0 += (s_end < n_sub_seq ? s_end : n_sub_seq) - 2 * sg.tile0;
+      }
       i0 += sg.n_tiles;
       c.next_segment(prefix, p.batch, hkv);
     }
@@ -760,7 +781,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 // ---------------------------------------------------------------------------------------------
 static int tc_grid(const specvlm_kv_t* kv, int32_t batch) {
   const int64_t tiles_max = (int64_t)kv->n_layers * batch * kv->n_kv_heads *
-                            ((kv->max_seq_len + kTileTokens - 1) / kTileTokens);
+                            ((kv->max_seq_len + kBigTokens - 1) / kBigTokens);
   return sched_active_ctas(tiles_max, sm_count());
 }
 
@@ -771,14 +792,32 @@ size_t attn_tc_ws_bytes(const specvlm_kv_t* kv, int32_t batch, int rows) {
          round_up((size_t)2 * grid * rows * sizeof(float), 256) + round_up(items * sizeof(int32_t), 256);
 }
 
+// Queries as a 5-D tensor (channel, head in group, query token, KV head, layer * batch + sequence):
+// the box (64 channels, group, n_q, 1, 1) is one item's rows in the order r = t * group + head.
+static int32_t encode_q_map(CUtensorMap* map, const void* q, int D, int group, int n_q, int n_kv_heads,
+                            int64_t lb) {
+  encode_tiled_fn enc = get_encode_tiled();
+  if (!enc) return SPECVLM_ERR_CUDA;
+  const int hq = group * n_kv_heads;
+  const cuuint64_t dims[5] = {(cuuint64_t)D, (cuuint64_t)group, (cuuint64_t)n_q, (cuuint64_t)n_kv_heads, (cuuint64_t)lb};
+  const cuuint64_t strides[4] = {(cuuint64_t)D * 2, (cuuint64_t)hq * D * 2, (cuuint64_t)group * D * 2,
+                                 (cuuint64_t)n_q * hq * D * 2};
+  const cuuint32_t box[5] = {64u, (cuuint32_t)group, (cuuint32_t)n_q, 1u, 1u};
+  const cuuint32_t estr[5] = {1u, 1u, 1u, 1u, 1u};
+  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(q), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? SPECVLM_OK : SPECVLM_ERR_CUDA;
+}
+
 template <int D, int M>
-static int32_t launch_tc(const CUtensorMap& tk, const CUtensorMap& tv, const AttnTcParams& p, int grid,
-                         cudaStream_t st) {
+static int32_t launch_tc(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tq, const AttnTcParams& p,
+                         int grid, cudaStream_t st) {
   using C = TcCfg<D, M>;
   auto kern = attn_tc_kernel<D, M>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::TOTAL) != cudaSuccess)
     return SPECVLM_ERR_CUDA;
-  kern<<<grid, kTcThreads, C::TOTAL, st>>>(tk, tv, p);
+  kern<<<grid, kTcThreads, C::TOTAL, st>>>(tk, tv, tq, p);
   return launch_status();
 }
 
@@ -794,14 +833,15 @@ int32_t attn_tc_launch(const specvlm_kv_t* kv, const void* q, int32_t batch, int
   if (ws_bytes < attn_tc_ws_bytes(kv, batch, rows)) return SPECVLM_ERR_WORKSPACE_TOO_SMALL;
   const int grid = tc_grid(kv, batch);
 
-  CUtensorMap tk, tv;
+  CUtensorMap tk, tv, tq;
   int32_t rc = encode_kv_map(&tk, kv, kv->k, kTileTokens);
   if (rc != SPECVLM_OK) return rc;
   rc = encode_kv_map(&tv, kv, kv->v, kTileTokens);
   if (rc != SPECVLM_OK) return rc;
+  rc = encode_q_map(&tq, q, kv->head_dim, group, n_q, kv->n_kv_heads, (int64_t)kv->n_layers * batch);
+  if (rc != SPECVLM_OK) return rc;
 
   AttnTcParams p;
-  p.q = static_cast<const __nv_bfloat16*>(q);
   p.out = static_cast<__nv_bfloat16*>(out);
   p.lse = lse;
   uint8_t* w = static_cast<uint8_t*>(ws);
@@ -827,8 +867,8 @@ int32_t attn_tc_launch(const specvlm_kv_t* kv, const void* q, int32_t batch, int
 
   if (cudaMemsetAsync(p.ws_cnt, 0, (size_t)items * sizeof(int32_t), st) != cudaSuccess) return SPECVLM_ERR_CUDA;
   if (kv->head_dim == 128)
-    return rows <= 64 ? launch_tc<128, 64>(tk, tv, p, grid, st) : launch_tc<128, 128>(tk, tv, p, grid, st);
-  return rows <= 64 ? launch_tc<64, 64>(tk, tv, p, grid, st) : launch_tc<64, 128>(tk, tv, p, grid, st);
+    return rows <= 64 ? launch_tc<128, 64>(tk, tv, tq, p, grid, st) : launch_tc<128, 128>(tk, tv, tq, p, grid, st);
+  return rows <= 64 ? launch_tc<64, 64>(tk, tv, tq, p, grid, st) : launch_tc<64, 128>(tk, tv, tq, p, grid, st);
 }
 
 }  // namespace specvlm
