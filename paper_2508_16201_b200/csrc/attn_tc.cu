@@ -7,10 +7,11 @@
 // 64-token sub-tiles (one cache page each) as the TMA moves them.
 //
 // Roles inside a CTA (12 warps = 3 warpgroups; the first gives registers to the other two):
-//   warp 0     TMA producer: the item's query rows, 64-token K sub-tiles into pair slots (a K tile
-//              must be 128 contiguous rows for the N = 128 product), V sub-tiles into a ring of
-//              single slots.  K and V have rings of their own because a K tile is free again as
-//              soon as S = Q K^T has been computed, long before its V tiles.
+//   warp 0     TMA producer of the item's query rows and of the K tiles
+//   warp 3     TMA producer of the V tiles.  K and V have rings of their own because a K tile is
+//              free again as soon as S = Q K^T has been computed, long before its V tile; and
+//              producers of their own because one thread cannot issue all copies of a tile
+//              within the time HBM needs to deliver it.
 //   warp 1     issues S = Q K^T (one thread, tcgen05.mma, accumulator in TMEM)
 //   warp 2     issues O += P V (one thread)
 //   warps 4-7  softmax group 0: the even tiles of the slice
@@ -131,16 +132,16 @@ template <int D, int M>
 struct TcCfg {
   static constexpr int SUB_BYTES = kTileTokens * D * 2;         // one 64-token K (or V) sub-tile
   static constexpr int NKP = D == 128 ? 2 : 3;                  // K ring: pair slots (128 tokens)
-  static constexpr int NVS = D == 128 ? (M == 64 ? 6 : 3) : 6;  // V ring: single slots (64 tokens)
+  static constexpr int NVP = D == 128 ? (M == 64 ? 3 : 1) : 3;  // V ring: pair slots
   static constexpr int NQ = (D == 128 && M == 128) ? 1 : 2;     // query buffers
   static constexpr int Q_BYTES = M * D * 2;                     // A operand of S = Q K^T
   static constexpr int P_BYTES = M * kBigTokens * 2;            // A operand of O += P V
   static constexpr int OFF_K = 0;
   static constexpr int OFF_V = OFF_K + NKP * 2 * SUB_BYTES;
-  static constexpr int OFF_Q = OFF_V + NVS * SUB_BYTES;
+  static constexpr int OFF_Q = OFF_V + NVP * 2 * SUB_BYTES;
   static constexpr int OFF_P = OFF_Q + NQ * Q_BYTES;
   static constexpr int BIG = OFF_P + 2 * P_BYTES;
-  static constexpr int N_BARS = 2 * NKP + 2 * NVS + 17;
+  static constexpr int N_BARS = 2 * NKP + 2 * NVP + 17;
   static constexpr int SM_BAR = 0;
   static constexpr int SM_MISC = SM_BAR + 8 * N_BARS;
   static constexpr int SM_PREFIX = SM_MISC + 32;
@@ -160,7 +161,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ AttnTcParams p) {
   using C = TcCfg<D, M>;
-  constexpr int SUB_BYTES = C::SUB_BYTES, NKP = C::NKP, NVS = C::NVS, NQ = C::NQ;
+  constexpr int SUB_BYTES = C::SUB_BYTES, NKP = C::NKP, NVP = C::NVP, NQ = C::NQ;
   constexpr int Q_BYTES = C::Q_BYTES, P_BYTES = C::P_BYTES;
   constexpr int NH = M / 64;                          // 16-lane halves a softmax warp may own
   constexpr uint32_t kIdescQK = umma_idesc_bf16(M, kBigTokens, false, false);
@@ -173,8 +174,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   const uint32_t k_sm = big + C::OFF_K, v_sm = big + C::OFF_V, q_sm = big + C::OFF_Q, p_sm = big + C::OFF_P;
   const uint32_t bar0 = raw_addr + C::SM_BAR;
   const uint32_t bar_k_full = bar0, bar_k_empty = bar_k_full + 8 * NKP;
-  const uint32_t bar_v_full = bar_k_empty + 8 * NKP, bar_v_empty = bar_v_full + 8 * NVS;
-  const uint32_t bar_q_full = bar_v_empty + 8 * NVS;   // [2]
+  const uint32_t bar_v_full = bar_k_empty + 8 * NKP, bar_v_empty = bar_v_full + 8 * NVP;
+  const uint32_t bar_q_full = bar_v_empty + 8 * NVP;   // [2]
   const uint32_t bar_q_empty = bar_q_full + 16;        // [2]
   const uint32_t bar_s_full = bar_q_empty + 16;        // [2]: one per softmax group
   const uint32_t bar_s_empty = bar_s_full + 16;        // [2]
@@ -206,7 +207,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       mbar_init(bar_k_full + 8 * s, 1);
       mbar_init(bar_k_empty + 8 * s, 1);
     }
-    for (int s = 0; s < NVS; ++s) {
+    for (int s = 0; s < NVP; ++s) {
       mbar_init(bar_v_full + 8 * s, 1);
       mbar_init(bar_v_empty + 8 * s, 1);
     }
@@ -269,24 +270,33 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   const int n_items = p.n_layers * p.batch * hkv;
   const int n_my = (int)(T1 - T0);
 
-  if (warp == 0) {
-    // ================================================================ TMA producer
+  if (warp == 0 || warp == 3) {
+    // ================================================================ TMA producers
+    // warp 0: query rows + K tiles; warp 3: V tiles.  Both walk the same slice.
     setmaxnreg_dec<kRegsLight>();
     if (lane == 0 && active) {
-      tma_prefetch_desc(&tm_k);
-      tma_prefetch_desc(&tm_v);
-      tma_prefetch_desc(&tm_q);
+      const bool is_k = warp == 0;
+      const CUtensorMap* const tm = is_k ? &tm_k : &tm_v;
+      tma_prefetch_desc(tm);
+      if (is_k) tma_prefetch_desc(&tm_q);
       const uint64_t policy = l2_policy_evict_first();
       const uint64_t policy_q = l2_policy_evict_last();
       const int subs_per_block = p.block_table ? p.block_tokens / kTileTokens : 1;
+      const int n_ring = is_k ? NKP : NVP;
+      const uint32_t ring_sm = is_k ? k_sm : v_sm, bar_full = is_k ? bar_k_full : bar_v_full;
+      const uint32_t bar_empty = is_k ? bar_k_empty : bar_v_empty;
+      // K tile: [64-channel block][128 tokens][128 B], the two sub-tiles stacked inside each block;
+      // V tile: two sub-tiles of [64-channel block][64 tokens][128 B] one after the other
+      const uint32_t blk_stride = is_k ? kBigTokens * 128 : kTileTokens * 128;
+      const uint32_t sub_stride = is_k ? kTileTokens * 128 : SUB_BYTES;
       SliceCursor c;
       c.start(T0, T1, prefix, p.batch, hkv);
       bool ok = true;
-      int i = 0, vc = 0, k_issued = 0;      // tiles, V sub-tiles, K tiles issued so far
+      int i = 0;
       while (c.f < T1 && ok) {
         const Segment sg = c.sg;
-        // the item's query rows: a box of (64 channels) x (group heads) x (n_q tokens) per 64-channel block
-        {
+        if (is_k) {
+          // the item's query rows: a box of (64 channels) x (group heads) x (n_q tokens) per 64-channel block
           const int qb = c.seg_idx % NQ;
           if (c.seg_idx >= NQ) ok = mbar_wait(bar_q_empty + 8 * qb, ((c.seg_idx / NQ) - 1) & 1, abort_flag);
           if (!ok) break;
@@ -304,7 +314,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           blk_next[0] = __ldg(table + s0 / subs_per_block);
           blk_next[1] = s0 + 1 < n_sub_seq ? __ldg(table + (s0 + 1) / subs_per_block) : 0;
         }
-        for (int j = 0; j < sg.n_tiles && ok; ++j, ++i) {
+        for (int j = 0; j < sg.n_tiles; ++j, ++i) {
           const int s0 = 2 * (sg.tile0 + j);                    // first sub-tile of this tile
           const int n_sub = n_sub_seq - s0 < 2 ? n_sub_seq - s0 : 2;
           blk[0] = blk_next[0];
@@ -313,41 +323,26 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             blk_next[0] = __ldg(table + (s0 + 2) / subs_per_block);
             blk_next[1] = s0 + 3 < n_sub_seq ? __ldg(table + (s0 + 3) / subs_per_block) : 0;
           }
-          const int kp = i % NKP;
-          if (i >= NKP) ok = mbar_wait(bar_k_empty + 8 * kp, ((i / NKP) - 1) & 1, abort_flag);
+          const int slot = i % n_ring;
+          if (i >= n_ring) ok = mbar_wait(bar_empty + 8 * slot, ((i / n_ring) - 1) & 1, abort_flag);
           if (!ok) break;
-          mbar_arrive_expect_tx(bar_k_full + 8 * kp, n_sub * SUB_BYTES);
+          mbar_arrive_expect_tx(bar_full + 8 * slot, n_sub * SUB_BYTES);
           for (int u = 0; u < n_sub; ++u) {
             const int tok = table ? ((s0 + u) % subs_per_block) * kTileTokens : (s0 + u) * kTileTokens;
 #pragma unroll
-            for (int h = 0; h < D / 64; ++h)      // K tile: [64-channel block][128 tokens][128 B]
-              tma_load_5d(k_sm + kp * 2 * SUB_BYTES + h * (kBigTokens * 128) + u * (kTileTokens * 128), &tm_k,
-                          bar_k_full + 8 * kp, h * 64, tok, sg.g, blk[u], sg.layer, policy);
-          }
-          k_issued = i + 1;
-          for (int u = 0; u < n_sub && ok; ++u, ++vc) {
-            const int vs = vc % NVS;
-            if (vc >= NVS) ok = mbar_wait(bar_v_empty + 8 * vs, ((vc / NVS) - 1) & 1, abort_flag);
-            if (!ok) break;
-            const int tok = table ? ((s0 + u) % subs_per_block) * kTileTokens : (s0 + u) * kTileTokens;
-            mbar_arrive_expect_tx(bar_v_full + 8 * vs, SUB_BYTES);
-#pragma unroll
-            for (int h = 0; h < D / 64; ++h)      // V sub-tile: [64-channel block][64 tokens][128 B]
-              tma_load_5d(v_sm + vs * SUB_BYTES + h * (kTileTokens * 128), &tm_v, bar_v_full + 8 * vs, h * 64, tok,
-                          sg.g, blk[u], sg.layer, policy);
+            for (int h = 0; h < D / 64; ++h)
+              tma_load_5d(ring_sm + slot * 2 * SUB_BYTES + h * blk_stride + u * sub_stride, tm, bar_full + 8 * slot,
+                          h * 64, tok, sg.g, blk[u], sg.layer, policy);
           }
         }
-        c.next_segment(prefix, p.batch, hkv);
+        if (ok) c.next_segment(prefix, p.batch, hkv);
       }
       if (!ok) {
-        // a wait expired: report, then stay until this CTA's copies in flight have landed (bounded)
+        // a wait expired: report, then stay until this thread's copies in flight have landed (bounded)
         if (p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
         const uint64_t t0 = global_timer_ns();
-        for (int k = k_issued > NKP ? k_issued - NKP : 0; k < k_issued; ++k)
-          while (!mbar_test_wait(bar_k_full + 8 * (k % NKP), (k / NKP) & 1) && global_timer_ns() - t0 < kWaitLimitNs) {
-          }
-        for (int k = vc > NVS ? vc - NVS : 0; k < vc; ++k)
-          while (!mbar_test_wait(bar_v_full + 8 * (k % NVS), (k / NVS) & 1) && global_timer_ns() - t0 < kWaitLimitNs) {
+        for (int k = i > n_ring ? i - n_ring : 0; k < i; ++k)
+          while (!mbar_test_wait(bar_full + 8 * (k % n_ring), (k / n_ring) & 1) && global_timer_ns() - t0 < kWaitLimitNs) {
           }
       }
     }
@@ -383,48 +378,72 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     }
   } else if (warp == 2) {
     // ================================================================ O += P V issuer
+    // The whole warp walks the slice; lane 0 issues.  The other lanes are there for the one job
+    // that needs hands: where a sequence ends inside a sub-tile, the V rows past its end hold
+    // whatever the page held, and are cleared so that a zero probability times a stale non-finite
+    // value cannot reach O.
     setmaxnreg_dec<kRegsLight>();
-    if (lane == 0 && active) {
+    if (active) {
       SliceCursor c;
       c.start(T0, T1, prefix, p.batch, hkv);
       const uint64_t dp0 = umma_desc_sw128(p_sm, 16, 1024);
       const uint64_t dv0 = umma_desc_sw128(v_sm, kTileTokens * 128, 1024);   // 64-channel blocks 8 KB apart
       bool ok = true;
-      int vc = 0, n_sub_seq = 0;
+      int n_sub_seq = 0, kv_len = 0;
+#define PV_WAIT(bar, parity)                                                        \
+  do {                                                                              \
+    ok = __all_sync(0xffffffffu, mbar_wait((bar), (parity), abort_flag));           \
+  } while (0)
       for (int i = 0; i < n_my; ++i) {
-        const int g = i & 1;
-        if (c.j == 0) n_sub_seq = (clamp_len(p.seq_lens[c.sg.b], p.max_seq_len) + kTileTokens - 1) / kTileTokens;
+        const int g = i & 1, vp = i % NVP;
+        if (c.j == 0) {
+          kv_len = clamp_len(p.seq_lens[c.sg.b], p.max_seq_len);
+          n_sub_seq = (kv_len + kTileTokens - 1) / kTileTokens;
+        }
         const int s0 = 2 * (c.sg.tile0 + c.j);
         const int n_sub = n_sub_seq - s0 < 2 ? n_sub_seq - s0 : 2;
-        // the first product of each group overwrites that group's O: the previous item must be out
-        if (c.j < 2 && c.seg_idx >= 1) ok = mbar_wait(bar_o_empty, (c.seg_idx - 1) & 1, abort_flag);
-        if (ok) ok = mbar_wait(bar_p_full + 8 * g, (i >> 1) & 1, abort_flag);
+        PV_WAIT(bar_v_full + 8 * vp, (i / NVP) & 1);
         if (!ok) break;
-        const uint64_t da = umma_desc_advance(dp0, g * P_BYTES);
-        const uint32_t d_tmem = tmem_base + C::COL_O + g * D;
-        for (int u = 0; u < n_sub && ok; ++u, ++vc) {
-          const int vs = vc % NVS;
-          ok = mbar_wait(bar_v_full + 8 * vs, (vc / NVS) & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after_sync();
-          const uint64_t dau = umma_desc_advance(da, u * (M * 128)), db = umma_desc_advance(dv0, vs * SUB_BYTES);
-          const uint32_t acc0 = (c.j >= 2 || u > 0) ? 1u : 0u;
-#pragma unroll
-          for (int kt = 0; kt < kTileTokens / 16; ++kt)
-            // 16 tokens per step: 32 bytes along P's row, 16 rows of 128 bytes down the V sub-tile
-            umma_bf16_ss(d_tmem, umma_desc_advance(dau, kt * 32), umma_desc_advance(db, kt * 2048), kIdescPV,
-                         kt > 0 ? 1u : acc0);
-          umma_commit(bar_v_empty + 8 * vs);
+        if (s0 + n_sub == n_sub_seq && (kv_len & (kTileTokens - 1)) != 0) {
+          uint8_t* vt = big_ptr + C::OFF_V + vp * 2 * SUB_BYTES + (n_sub - 1) * SUB_BYTES;
+          const int first = kv_len - (n_sub_seq - 1) * kTileTokens;
+          for (int idx = lane; idx < (kTileTokens - first) * (D / 8); idx += 32) {
+            const int t = first + idx / (D / 8), c16 = idx % (D / 8);
+            *reinterpret_cast<uint4*>(vt + (c16 >> 3) * (kTileTokens * 128) + t * 128 + (c16 & 7) * 16) =
+                make_uint4(0, 0, 0, 0);
+          }
+          fence_proxy_async();
+          __syncwarp();
         }
+        // the first product of each group overwrites that group's O: the previous item must be out
+        if (c.j < 2 && c.seg_idx >= 1) PV_WAIT(bar_o_empty, (c.seg_idx - 1) & 1);
+        if (ok) PV_WAIT(bar_p_full + 8 * g, (i >> 1) & 1);
         if (!ok) break;
-        umma_commit(bar_p_empty + 8 * g);
-        if (c.last_of_segment()) umma_commit(bar_o_full);
+        if (lane == 0) {
+          tc_fence_after_sync();
+          const uint64_t da = umma_desc_advance(dp0, g * P_BYTES), db = umma_desc_advance(dv0, vp * 2 * SUB_BYTES);
+          const uint32_t d_tmem = tmem_base + C::COL_O + g * D;
+          const uint32_t acc0 = c.j >= 2 ? 1u : 0u;
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            if (u < n_sub) {
+#pragma unroll
+              for (int kt = 0; kt < kTileTokens / 16; ++kt)
+                // 16 tokens per step: 32 bytes along P's row, 16 rows of 128 bytes down the V sub-tile
+                umma_bf16_ss(d_tmem, umma_desc_advance(da, u * (M * 128) + kt * 32),
+                             umma_desc_advance(db, u * SUB_BYTES + kt * 2048), kIdescPV, (u > 0 || kt > 0) ? 1u : acc0);
+            }
+          }
+          umma_commit(bar_p_empty + 8 * g);
+          umma_commit(bar_v_empty + 8 * vp);
+          if (c.last_of_segment()) umma_commit(bar_o_full);
+        }
+        __syncwarp();
         c.next_tile(prefix, p.batch, hkv);
       }
-      if (!ok && p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
+#undef PV_WAIT
+      if (!ok && p.d_status && lane == 0) *p.d_status = SPECVLM_ERR_TIMEOUT;
     }
-  } else if (warp == 3) {
-    setmaxnreg_dec<kRegsLight>();
   } else {
     // ================================================================ softmax / epilogue (warps 4..11)
     setmaxnreg_inc<kRegsSoftmax>();
@@ -456,7 +475,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     c.start(T0, T1, prefix, p.batch, hkv);
     bool ok = true;
     int i0 = 0;           // index (inside the slice) of the current segment's first tile
-    int vc0 = 0;          // V sub-tiles of the slice before the current segment
     int n_partial = 0;    // partial epilogues so far
 #define SM_WAIT(bar, parity)                                                        \
   do {                                                                              \
@@ -590,20 +608,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           l_sum[h][1] += ps[2] + ps[3];
         }
         if (nh == 0 && i >= 2) SM_WAIT(bar_p_empty + 8 * grp, ((i >> 1) - 1) & 1);
-        if (tile_tok0 + kBigTokens > kv_len && (kv_len & (kTileTokens - 1)) != 0) {
-          // the sequence ends inside a sub-tile: the V rows past its end hold whatever the page held;
-          // clear them so that a zero probability times a stale non-finite value cannot reach O
-          const int last_sub = n_sub_seq - 1;
-          const int vcl = vc0 + 2 * j + (last_sub - 2 * (sg.tile0 + j));   // that sub-tile's place in the V ring
-          SM_WAIT(bar_v_full + 8 * (vcl % NVS), (vcl / NVS) & 1);
-          uint8_t* vt = big_ptr + C::OFF_V + (vcl % NVS) * SUB_BYTES;
-          const int first = kv_len - last_sub * kTileTokens;
-          for (int idx = gt; idx < (kTileTokens - first) * (D / 8); idx += 128) {
-            const int t = first + idx / (D / 8), c16 = idx % (D / 8);
-            *reinterpret_cast<uint4*>(vt + (c16 >> 3) * (kTileTokens * 128) + t * 128 + (c16 & 7) * 16) =
-                make_uint4(0, 0, 0, 0);
-          }
-        }
         fence_proxy_async();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_p_full + 8 * grp);
@@ -753,11 +757,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             if (p.lse && c4 == 0) p.lse[orow] = den > 0.f ? (mm + log2f(den)) * kLn2 : -INFINITY;
           }
         }
-      }
-      // sub-tiles of this segment: two per tile, except that the item's last tile may hold one
-      {
-        const int s_end = 2 * (sg.tile0 + sg.n_tiles);
-        vc0 += (s_end < n_sub_seq ? s_end : n_sub_seq) - 2 * sg.tile0;
       }
       i0 += sg.n_tiles;
       c.next_segment(prefix, p.batch, hkv);
