@@ -160,10 +160,10 @@ class Path:
         self.ws_acc = torch.empty(specvlm.accept_workspace_bytes(1, w.gamma, w.vocab), dtype=torch.uint8,
                                   device=device)
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
-        # launches of our kernels per step
-        dec_l = 1 + (specvlm.attn_workspace_bytes(inp["dpruned"][0], 1, w.d_q_heads, 0) > 256)
-        ver_l = 1 + (specvlm.attn_workspace_bytes(inp["tcache"], 1, w.t_q_heads, w.gamma) > 256)
-        self.launches_per_step = 1 + 2 + 1 + 1 + w.gamma * dec_l + ver_l + 2
+        # launches of our kernels per step: row LSE 1, rating 2 (column sums + finish), select 1,
+        # gather 1, one per draft decode step, verify 1, accept 2 (split merges run inside the
+        # attention kernels; the counter resets before them are memsets, not counted)
+        self.launches_per_step = 1 + 2 + 1 + 1 + w.gamma + 1 + 2
 
     # the calls, in path order ------------------------------------------------------------------
     def row_lse_call(self):
@@ -329,7 +329,7 @@ def run_ours(args, rank, world):
     flops_colsum = 2.0 * rows * nv * D
     flops_lse = 2.0 * w.t_layers * w.t_q_heads * D * sum(nv + i + 1 for i in range(nt))
     roofs = {
-        "verify": hbm("attn_rowsN_kernel (verify)", bytes_ver, mean["verify"], NCU_TRAFFIC_BYTES["verify"]),
+        "verify": hbm("attn_tc_kernel (verify, tcgen05)", bytes_ver, mean["verify"], NCU_TRAFFIC_BYTES["verify"]),
         "decode": hbm("attn_rows16_kernel (draft decode, pruned cache)", bytes_dec, mean["decode"],
                       NCU_TRAFFIC_BYTES["decode"]),
         "scores_colsum": tensor("scores_colsum_kernel", flops_colsum, mean["scores"],

@@ -10,6 +10,7 @@ struct AttnParams {
   float* lse;                 // [L][B][n_q][Hq] or null
   float* ws_o;                // split partials: [item][split][rows][D], normalised
   float* ws_lse;              // [item][split][rows], log2 units
+  int32_t* ws_cnt;            // [item] arrival counters of the splits, zero at launch
   const int32_t* block_table; // [B][max_blocks] or null
   const int32_t* seq_lens;    // [B]
   int32_t* d_status;
