@@ -1,0 +1,172 @@
+"""Parity at the benchmark's full sizes, through the C ABI, in the launch configuration bench.py
+times.  The CUDA side runs the whole workload; the fp64 oracle is run on sampled layers (each layer
+is an independent problem for every call on the path), on the very same tensors copied to the host.
+
+Workloads 3-5 keep their per-layer shapes (tokens, heads, rows, paging) and run a stated subset of
+layers, since a layer count only repeats the same problem."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import bits, f64, row_rel_err
+from paper_2508_16201_b200 import specvlm, synth
+
+pytestmark = pytest.mark.gpu
+
+ATTN_TOL = 1e-2
+SCORE_TOL = 1e-4
+
+
+def _contig_cache(L, Hkv, n, D, seed, tag):
+    k = synth.randn_bf16((L, 1, Hkv, n, D), "cuda", seed, tag + "K")
+    v = synth.randn_bf16((L, 1, Hkv, n, D), "cuda", seed, tag + "V")
+    lens = torch.tensor([n], dtype=torch.int32, device="cuda")
+    return specvlm.KvCache(k, v, lens, n), k, v
+
+
+def _check_layers(out, lse, q, k, v, n, scale, layers):
+    """oracle attention on the sampled layers of a batch-1 contiguous cache"""
+    worst = 0.0
+    for l in layers:
+        ref, ref_lse = oracle.attention(bits(q[l, 0]), bits(k[l, 0]), bits(v[l, 0]), n, scale)
+        got = f64(out[l, 0])
+        assert np.isfinite(got).all()
+        worst = max(worst, row_rel_err(got, ref))
+        np.testing.assert_allclose(lse[l, 0].cpu().numpy(), ref_lse, rtol=0, atol=2e-3)
+    assert worst <= ATTN_TOL, f"row rel err {worst}"
+
+
+def _verify_full(i, layers_run, sample, seed):
+    w = synth.workload(i)
+    D, g1 = w.head_dim, w.gamma + 1
+    n = w.seq_len() + g1                         # the cache already holds the gamma+1 new tokens
+    cache, k, v = _contig_cache(layers_run, w.t_kv_heads, n, D, seed, "t")
+    q = synth.randn_bf16((layers_run, 1, g1, w.t_q_heads, D), "cuda", seed, "Qv")
+    scale = 1.0 / math.sqrt(D)
+    lse = torch.empty((layers_run, 1, g1, w.t_q_heads), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = specvlm.verify_attn(cache, q, w.gamma, scale, lse=lse, d_status=status)
+    out2 = specvlm.verify_attn(cache, q, w.gamma, scale)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(out, out2)                # the merge order of cut items is fixed
+    _check_layers(out, lse, q, k, v, n, scale, sample)
+
+
+def test_verify_cfg2_all_80_layers_sampled():
+    _verify_full(2, 80, [0, 41, 79], seed=100)
+
+
+def test_verify_cfg3_all_64_layers_sampled():
+    _verify_full(3, 64, [0, 63], seed=101)       # 40 q / 8 kv heads: 30 rows, 23302 tokens
+
+
+def test_verify_cfg4_8_of_80_layers_sampled():
+    _verify_full(4, 8, [7], seed=102)            # 50311 tokens, gamma 6: 56 rows
+
+
+@pytest.mark.parametrize("pruned", [True, False])
+def test_decode_cfg2_all_28_layers(pruned):
+    w = synth.workload(2)
+    D = w.head_dim
+    n = (w.k_total() + w.n_text[0]) if pruned else w.seq_len()
+    cache, k, v = _contig_cache(w.d_layers, w.d_kv_heads, n, D, 103, "d")
+    q = synth.randn_bf16((w.d_layers, 1, 1, w.d_q_heads, D), "cuda", 103, "Qd")
+    scale = 1.0 / math.sqrt(D)
+    lse = torch.empty((w.d_layers, 1, w.d_q_heads), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = specvlm.draft_decode_attn(cache, q[:, :, 0].contiguous(), scale, lse=lse, d_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    layers = range(w.d_layers) if pruned else [0, 13, 27]
+    _check_layers(out[:, :, None], lse[:, :, None], q, k, v, n, scale, layers)
+
+
+@pytest.mark.parametrize("gamma", [3, 8])
+def test_cfg5_batched_paged_verify_and_decode(gamma):
+    """Workload 5: 16 ragged sequences, 64-token pages scattered over the pool; 2 of 80 verifier
+    layers and 2 of 28 draft layers.  gamma 3 gives 32 rows per KV head, gamma 8 gives 72."""
+    from gpu_util import make_cache
+    w = synth.workload(5, gamma=gamma)
+    D, g1, B, L = w.head_dim, gamma + 1, w.batch, 2
+    scale = 1.0 / math.sqrt(D)
+    # verification over the full target cache
+    lens = [w.seq_len(b) + g1 for b in range(B)]
+    cache, k_host, v_host = make_cache(L, w.t_kv_heads, D, lens, paged=True, seed=110 + gamma)
+    q = synth.randn_bf16((L, B, g1, w.t_q_heads, D), "cuda", 110 + gamma, "Qv")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = specvlm.verify_attn(cache, q, gamma, scale, d_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    qh, got = bits(q), f64(out)
+    assert np.isfinite(got).all()
+    worst = 0.0
+    for b in range(B):
+        ref, _ = oracle.attention(qh[1, b], k_host[b][1], v_host[b][1], lens[b], scale)
+        worst = max(worst, row_rel_err(got[1, b], ref))
+    assert worst <= ATTN_TOL, f"verify row rel err {worst}"
+    del cache, k_host, v_host
+    # draft decode over the pruned caches (10 % of the video tokens + the text)
+    plens = [w.k_total(b) + w.n_text[b] for b in range(B)]
+    dcache, dk, dv = make_cache(L, w.d_kv_heads, D, plens, paged=True, seed=120 + gamma)
+    qd = synth.randn_bf16((L, B, 1, w.d_q_heads, D), "cuda", 120 + gamma, "Qd")
+    od = specvlm.draft_decode_attn(dcache, qd[:, :, 0].contiguous(), scale, d_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    qh, got = bits(qd), f64(od)
+    worst = 0.0
+    for l in range(L):
+        for b in range(B):
+            ref, _ = oracle.attention(qh[l, b], dk[b][l], dv[b][l], plens[b], scale)
+            worst = max(worst, row_rel_err(got[l, b][None], ref))
+    assert worst <= ATTN_TOL, f"decode row rel err {worst}"
+
+
+def test_scores_cfg2_sampled_layers_and_layer_mean():
+    """Token rating at workload 2's size.  The oracle rates two sampled layers (a call on a one-layer
+    view of the same cache must match it); the 80-layer call must equal the mean of the 80
+    one-layer calls, which holds for Eq. 5's average at any size."""
+    w = synth.workload(2)
+    D, nv, nt, L = w.head_dim, w.n_video(), w.n_text[0], w.t_layers
+    scale = 1.0 / math.sqrt(D)
+    k = synth.randn_bf16((L, 1, w.t_kv_heads, nv + nt, D), "cuda", 130, "tK")
+    q = synth.randn_bf16((L, nt, w.t_q_heads, D), "cuda", 130, "Qtext")
+    synth.plant_salient_(k[:, 0, :, :nv, :], q, synth.salient_set(nv, w.planted_permille, 130))
+    lens = torch.tensor([nv + nt], dtype=torch.int32, device="cuda")
+    args = ([0, nt], [nv], [0], [nv], [0, nv], scale)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    full = specvlm.stage1_scores(specvlm.KvCache(k, k, lens, nv + nt), q, *args, d_status=status)
+    per_layer = []
+    for l in range(L):
+        per_layer.append(specvlm.stage1_scores(specvlm.KvCache(k[l:l + 1], k[l:l + 1], lens, nv + nt),
+                                               q[l:l + 1], *args, d_status=status).double())
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    mean = torch.stack(per_layer).mean(0)
+    rel = ((full.double() - mean).abs() / mean).max().item()
+    assert rel <= 1e-5, f"80-layer call vs mean of one-layer calls: {rel}"
+    for l in (3, 77):
+        ref = oracle.stage1_scores(bits(q[l:l + 1]), bits(k[l:l + 1, 0]), 0, nv, nv, scale)
+        got = per_layer[l].cpu().numpy()
+        rel = float((np.abs(got - ref) / ref).max())
+        assert rel <= SCORE_TOL, f"layer {l}: scores rel err {rel}"
+    assert float(full.sum()) <= 1.0 and float(full.min()) >= 0.0
+
+
+def test_gather_cfg2_all_28_layers():
+    w = synth.workload(2)
+    D, nv, nt, L, H = w.head_dim, w.n_video(), w.n_text[0], w.d_layers, w.d_kv_heads
+    kt = w.k_total()
+    src, sk, sv = _contig_cache(L, H, nv + nt, D, 140, "src")
+    dst, dk, dv = _contig_cache(L, H, kt + nt, D, 141, "dst")
+    g = torch.Generator().manual_seed(140)
+    kept = torch.sort(torch.randperm(nv, generator=g)[:kt]).values.to(torch.int32)
+    specvlm.gather_kv(src, kept.cuda(), [0, kt], [0], [nv], [nv + nt], dst)
+    torch.cuda.synchronize()
+    kept_np = kept.numpy()
+    for name, s_t, d_t in (("K", sk, dk), ("V", sv, dv)):
+        ref = oracle.gather_kv(bits(s_t[:, 0]), kept_np, 0, nv, nv + nt)
+        assert np.array_equal(bits(d_t[:, 0]), ref), name
