@@ -677,6 +677,192 @@ scores_colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Pass 1 on tcgen05.  CTA = (row tile, KV head, layer), two CTAs per SM.
+//   S[row][key] = Q_tile (A: 128 rows x d, K-major) * K_tile^T (B: 128 keys x d, K-major)
+// as a chain of tcgen05.mma (M = N = 128, K = 16 each) into one of two 128-column TMEM buffers.
+// With the rows on the TMEM lanes an epilogue thread owns one row: it reads its 128 logits of a
+// tile with tcgen05.ld and keeps the row's running (max, sum) in two registers -- the row
+// reduction needs no cross-thread step.  The kernel is bound by the exponentials (one per logit),
+// not by the tensor pipe; the second CTA on the SM fills the first one's TMEM-load latency.
+// Warps: 0 = TMA producer (Q tile once, K tiles through a ring), 1 = TMEM allocation + MMA issue,
+// 2..5 = epilogue (one TMEM lane quadrant each).
+// ---------------------------------------------------------------------------------------------
+template <int D, int STAGES>
+__global__ void __launch_bounds__(192, 2)
+scores_lse_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
+                     const __grid_constant__ ScoreParams p) {
+  constexpr int TILE_BYTES = kKeyTile * D * 2;
+  constexpr int KSTEPS = D / 16;
+  constexpr uint32_t kTmemCols = 256;
+  constexpr uint32_t kIdesc = umma_idesc_bf16(128, 128, false, false);
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t base = (raw_addr + 1023u) & ~1023u;
+  uint8_t* const smem = smem_raw + (base - raw_addr);
+  const uint32_t q_sm = base;                                    // the row tile
+  const uint32_t k_sm = base + TILE_BYTES;                       // K ring
+  constexpr int kTail = (1 + STAGES) * TILE_BYTES;
+  const uint32_t bar_qfull = base + kTail;
+  const uint32_t bar_kfull = bar_qfull + 8;                      // [STAGES]
+  const uint32_t bar_kempty = bar_kfull + 8 * STAGES;            // [STAGES]
+  const uint32_t bar_tfull = bar_kempty + 8 * STAGES;            // [2]
+  const uint32_t bar_tempty = bar_tfull + 16;                    // [2]
+  uint8_t* const tail = smem + kTail + 16 * STAGES + 40;
+  volatile int* const abort_flag = reinterpret_cast<volatile int*>(tail);
+  volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(tail + 8);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int b = find_seq(p, blockIdx.x);
+  const ScoreSeq sq = p.seq[b];
+  const int qtile = blockIdx.x - sq.tile_off;
+  const int g = blockIdx.y, layer = blockIdx.z;
+  const int i_first = qtile * p.qt;
+  const int n_i = min(p.qt, sq.n_text - i_first);               // queries in this tile
+  const int rows_valid = n_i * p.group;
+  const int key_end = sq.text_start + i_first + n_i;            // keys [0, key_end) are needed
+  const int n_kt = (key_end + kKeyTile - 1) / kKeyTile;
+
+  if (tid == 0) {
+    mbar_init(bar_qfull, 1);
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(bar_kfull + 8 * s, 1);
+      mbar_init(bar_kempty + 8 * s, 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar_tfull + 8 * i, 1);
+      mbar_init(bar_tempty + 8 * i, 4);
+    }
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      tma_prefetch_desc(&tm_k);
+      tma_prefetch_desc(&tm_q);
+      const uint64_t pol = l2_policy_evict_last();               // K is re-read by the other row tiles
+      mbar_arrive_expect_tx(bar_qfull, (D / 64) * p.qt * p.group * 128);
+#pragma unroll
+      for (int h = 0; h < D / 64; ++h)
+        tma_load_5d(q_sm + h * (kKeyTile * 128), &tm_q, bar_qfull, h * 64, 0, g, sq.text_off + i_first, layer, pol);
+      bool ok = true;
+      int i = 0;
+      for (; i < n_kt; ++i) {
+        const int s = i % STAGES;
+        if (i >= STAGES) ok = mbar_wait(bar_kempty + 8 * s, ((i / STAGES) - 1) & 1, abort_flag);
+        if (!ok) break;
+        mbar_arrive_expect_tx(bar_kfull + 8 * s, TILE_BYTES);
+        load_key_tile<D>(&tm_k, p, b, g, layer, i * kKeyTile, k_sm + s * TILE_BYTES, bar_kfull + 8 * s, pol);
+      }
+      if (!ok) {
+        if (p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
+        const uint64_t t0 = global_timer_ns();
+        for (int k = i > STAGES ? i - STAGES : 0; k < i; ++k)
+          while (!mbar_try_wait(bar_kfull + 8 * (k % STAGES), (k / STAGES) & 1) &&
+                 global_timer_ns() - t0 < kWaitLimitNs) {
+          }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issue (one thread)
+    if (lane == 0) {
+      bool ok = mbar_wait(bar_qfull, 0, abort_flag);
+      for (int i = 0; i < n_kt && ok; ++i) {
+        const int s = i % STAGES, buf = i & 1;
+        ok = mbar_wait(bar_kfull + 8 * s, (i / STAGES) & 1, abort_flag);
+        if (ok && i >= 2) ok = mbar_wait(bar_tempty + 8 * buf, ((i >> 1) - 1) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint64_t da = umma_desc_sw128(q_sm, 16, 1024), db = umma_desc_sw128(k_sm + s * TILE_BYTES, 16, 1024);
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS; ++ks) {
+          // 16 channels per step: 32 bytes along the swizzled 128-byte row; channels 64.. live in
+          // the second half-tile
+          const uint32_t off = (ks >> 2) * (kKeyTile * 128) + (ks & 3) * 32;
+          umma_bf16_ss(tmem_base + buf * 128, umma_desc_advance(da, off), umma_desc_advance(db, off), kIdesc,
+                       ks > 0 ? 1u : 0u);
+        }
+        umma_commit(bar_kempty + 8 * s);
+        umma_commit(bar_tfull + 8 * buf);
+      }
+      if (!ok && p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue: 4 warps, 128 rows
+    const int quad = warp & 3;                  // TMEM lanes [32 * quad, 32 * quad + 32)
+    const int r = quad * 32 + lane;             // this thread's row
+    const int il = r / p.group, hg = r - il * p.group;
+    const int lim = r < rows_valid ? sq.text_start + i_first + il + 1 : 0;   // keys [0, lim) are visible
+    const int first_lim = sq.text_start + i_first + 1;
+    float m = -INFINITY, l = 0.f;
+    bool alive = true;
+    for (int i = 0; i < n_kt; ++i) {
+      const int buf = i & 1;
+      if (alive && !mbar_wait(bar_tfull + 8 * buf, (i >> 1) & 1, abort_flag)) alive = false;
+      alive = __all_sync(0xffffffffu, alive);   // warp-uniform: the TMEM loads below are warp-collective
+      if (!alive) break;
+      tc_fence_after_sync();
+      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * 128;
+      const int key0 = i * kKeyTile;
+      const bool need_mask = key0 + kKeyTile > first_lim;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t v[32];
+        tmem_ld_x32(taddr + c * 32, v);
+        tmem_ld_wait();
+        if (c == 3) {
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);   // buffer free for the MMAs of tile i + 2
+        }
+        float x[32];
+        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        if (need_mask) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            x[j] = key0 + c * 32 + j < lim ? __uint_as_float(v[j]) * p.scale_log2 : -INFINITY;
+            mx[j & 3] = fmaxf(mx[j & 3], x[j]);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            x[j] = __uint_as_float(v[j]) * p.scale_log2;
+            mx[j & 3] = fmaxf(mx[j & 3], x[j]);
+          }
+        }
+        const float mn = fmaxf(m, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])));
+        const float mu = mn == -INFINITY ? 0.f : mn;
+        float ps[4] = {0.f, 0.f, 0.f, 0.f};       // four chains for instruction-level parallelism
+#pragma unroll
+        for (int j = 0; j < 32; ++j) ps[j & 3] += fast_exp2(x[j] - mu);
+        l = l * fast_exp2(m - mu) + ((ps[0] + ps[1]) + (ps[2] + ps[3]));
+        m = mn;
+      }
+    }
+    if (alive && !*abort_flag) {
+      if (r < rows_valid)
+        p.lse[((size_t)layer * p.sum_text + sq.text_off + i_first + il) * p.n_q_heads + g * p.group + hg] =
+            (m + log2f(l)) * kLn2;
+    } else if (p.d_status && r == 0) {
+      *p.d_status = SPECVLM_ERR_TIMEOUT;
+    }
+  }
+  // every role ends here; the allocating warp returns the tensor memory
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
 // scores[j] = (sum over layers, in order, of partial[l][j]) / (L * Hq * n_text of j's sequence)
 __global__ void scores_finish_kernel(const __grid_constant__ ScoreParams p, float* __restrict__ scores) {
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
@@ -789,22 +975,35 @@ static int32_t setup_scores(const specvlm_kv_t* target_kv, const void* q_text, c
   return SPECVLM_OK;
 }
 
+static bool scores_legacy_mma() {
+  const char* impl = getenv("SPECVLM_SCORES_IMPL");
+  return impl && impl[0] == 'm';      // "mma": the mma.sync kernels
+}
+
 template <int D>
 static int32_t launch_lse(ScoreSetup& su, cudaStream_t st) {
-  constexpr int STAGES = 4;
-  constexpr int SMEM = STAGES * kKeyTile * D * 2 + 1024 + 16 * STAGES + 16 + 2 * 128 * 2 * 4;
-  auto k = scores_lse_kernel<D, STAGES>;
+  const dim3 grid((unsigned)su.n_row_tiles, (unsigned)su.kv.n_kv_heads, (unsigned)su.kv.n_layers);
+  if (scores_legacy_mma()) {
+    constexpr int STAGES = 4;
+    constexpr int SMEM = STAGES * kKeyTile * D * 2 + 1024 + 16 * STAGES + 16 + 2 * 128 * 2 * 4;
+    auto k = scores_lse_kernel<D, STAGES>;
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
+      return SPECVLM_ERR_CUDA;
+    k<<<grid, 288, SMEM, st>>>(su.tk, su.p1);
+    return launch_status();
+  }
+  constexpr int STAGES = 2;                              // two CTAs per SM: 3 x 32 KB each at d = 128
+  constexpr int SMEM = (1 + STAGES) * kKeyTile * D * 2 + 1024 + 16 * STAGES + 40 + 16;
+  auto k = scores_lse_tc_kernel<D, STAGES>;
   if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
     return SPECVLM_ERR_CUDA;
-  k<<<dim3((unsigned)su.n_row_tiles, (unsigned)su.kv.n_kv_heads, (unsigned)su.kv.n_layers), 288, SMEM, st>>>(
-      su.tk, su.p1);
+  k<<<grid, 192, SMEM, st>>>(su.tk, su.tq, su.p1);
   return launch_status();
 }
 
 template <int D>
 static int32_t launch_colsum(ScoreSetup& su, float* scores, cudaStream_t st) {
-  const char* impl = getenv("SPECVLM_SCORES_IMPL");
-  const bool legacy = impl && impl[0] == 'm';      // "mma": the mma.sync kernel
+  const bool legacy = scores_legacy_mma();
   int32_t rc;
   if (legacy) {
     constexpr int STAGES = 3;
