@@ -470,11 +470,12 @@ scores_colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
 // tile's epilogue).  With the keys on the TMEM lanes, an epilogue thread owns one key: it reads
 // its 128 row values with tcgen05.ld and adds up 2^(s - lse_row) in a single register for the
 // whole layer -- the column sum needs no cross-thread reduction at all.
-// Warps: 0 = TMA producer, 1 = TMEM allocation + MMA issue, 2..5 = epilogue (one TMEM lane
-// quadrant each).
+// Warps: 0 = TMA producer, 1 = TMEM allocation + MMA issue, 2..5 and 6..9 = two epilogue groups
+// (one TMEM lane quadrant per warp) that take alternate tiles, each on its own accumulator
+// buffer, so that one group's exponentials run while the other waits for its TMEM load.
 // ---------------------------------------------------------------------------------------------
 template <int D, int STAGES>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(320, 1)
 scores_colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
                         const __grid_constant__ ScoreParams p) {
   constexpr int TILE_BYTES = kKeyTile * D * 2;
@@ -596,10 +597,11 @@ scores_colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
       if (!ok && p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
     }
   } else {
-    // ---------------------------------------------------------------- epilogue: 4 warps, 128 keys
+    // ---------------------------------------------------------------- epilogue: 2 groups x 4 warps, 128 keys
+    const int grp = (warp - 2) >> 2;            // tiles with (index & 1) == grp, accumulator buffer grp
     const int quad = warp & 3;                  // TMEM lanes [32 * quad, 32 * quad + 32)
     const int key_l = quad * 32 + lane;         // this thread's key inside the block
-    const int et = (warp - 2) * 32 + lane;      // 0..127: used to stage the row LSEs
+    const int et = ((warp - 2) & 3) * 32 + lane;   // 0..127 inside the group: used to stage the row LSEs
     float acc = 0.f;
     bool alive = true;
     int it = 0;
@@ -607,6 +609,7 @@ scores_colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
       const float* lse_u = p.lse + ((size_t)layer * p.sum_text + sq.text_off) * p.n_q_heads + u * p.group;
       for (int t = 0; t < n_qt; ++t, ++it) {
         const int buf = it & 1;
+        if (buf != grp) continue;
         const int rows_valid = min(p.qt, sq.n_text - t * p.qt) * p.group;
         {
           float v = 0.f;
@@ -616,7 +619,7 @@ scores_colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
           }
           lse_sm[buf * 128 + et] = v;
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory");
         if (alive && !mbar_wait(bar_tfull + 8 * buf, (it >> 1) & 1, abort_flag)) alive = false;
         alive = __all_sync(0xffffffffu, alive); // warp-uniform: the TMEM loads below are warp-collective
         if (!alive) continue;                   // keep taking part in the barrier above
@@ -661,9 +664,15 @@ scores_colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
         }
       }
     }
+    // the key's column sum = group 0's tiles + group 1's tiles (fixed order)
+    float* const acc_sm = lse_sm;               // [128]: the staging area is free after the last tile
+    asm volatile("bar.sync 3, 256;" ::: "memory");
+    if (grp == 1) acc_sm[key_l] = acc;
+    asm volatile("bar.sync 3, 256;" ::: "memory");
     if (alive && !*abort_flag) {
       const int j = key0 + key_l - sq.video_start;           // video token index of this key
-      if (j >= 0 && j < sq.n_video) p.partial[(size_t)layer * p.sum_video + sq.score_off + j] = acc;
+      if (grp == 0 && j >= 0 && j < sq.n_video)
+        p.partial[(size_t)layer * p.sum_video + sq.score_off + j] = acc + acc_sm[key_l];
     } else if (p.d_status && et == 0) {
       *p.d_status = SPECVLM_ERR_TIMEOUT;
     }
@@ -1019,7 +1028,7 @@ static int32_t launch_colsum(ScoreSetup& su, float* scores, cudaStream_t st) {
     auto k = scores_colsum_tc_kernel<D, STAGES>;
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
       return SPECVLM_ERR_CUDA;
-    k<<<dim3((unsigned)su.n_key_blocks, (unsigned)su.kv.n_layers), 192, SMEM, st>>>(su.tk, su.tq, su.p2);
+    k<<<dim3((unsigned)su.n_key_blocks, (unsigned)su.kv.n_layers), 320, SMEM, st>>>(su.tk, su.tq, su.p2);
     rc = launch_status();
   }
   if (rc != SPECVLM_OK) return rc;
