@@ -136,6 +136,25 @@ int32_t specvlm_select(const float* scores, const int32_t* video_cu, const int32
                        const int32_t* kept_cu, int32_t batch, int32_t* kept_idx, int32_t* d_status,
                        void* stream);
 
+/*
+ * The same selection with the Stage-I count chosen by the paper's Top-P rule (Section 4.2, Eq. 6):
+ * V_R is the shortest prefix of the ranking (score descending, index ascending) whose cumulative
+ * score reaches lambda_r times the sum of all scores; the paper uses lambda_r = 0.4 and 0.5.  The
+ * count is bounded by k_total[b] (Stage II then adds nothing); otherwise Stage II fills the rest
+ * of the budget exactly as in specvlm_select.
+ *   lambda_permille   host int32 [batch]: lambda_r in thousandths, 0..1000
+ *   k_stage1_out_or_null   device int32 [batch] out: the Stage-I count of each sequence
+ * The cumulative comparison runs in integers so that the count is a function of the scores alone,
+ * not of a summation order: each score is truncated to a multiple of 2^-36 (values above 1 count
+ * as 1) and  1000 * sum_{i<c} q_(i) >= lambda_permille * sum q  is evaluated exactly.
+ * Other arguments, requirements and errors as for specvlm_select.
+ */
+int32_t specvlm_select_top_p(const float* scores, const int32_t* video_cu, const int32_t* n_frames,
+                             int32_t tokens_per_frame, const int32_t* lambda_permille,
+                             const int32_t* k_total, const int32_t* kept_cu, int32_t batch,
+                             int32_t* kept_idx, int32_t* k_stage1_out_or_null, int32_t* d_status,
+                             void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * Step 3 -- pruned draft context (end of Section 4.2: the draft sees V_R u V_U and the language
  * prompt, its cache reduced to 1-r of the original).

@@ -136,6 +136,34 @@ def stage1_top_p(scores_f32: np.ndarray, lambda_r: float, k_cap: int | None = No
     return c
 
 
+TOP_P_FRAC_BITS = 36
+
+
+def stage1_top_p_fixed(scores_f32: np.ndarray, lambda_permille: int, k_cap: int | None = None) -> int:
+    """Count c of Eq. 6 in the arithmetic the GPU library takes the decision in.
+
+    Eq. 6 compares a cumulative score with lambda_r times the total; in floating point the
+    result of that comparison can depend on the order of the additions.  So that the count is
+    a function of the scores alone, each fp32 score is first truncated to a multiple of
+    2^-36 (and capped at 1, the largest value a mean probability can take), lambda_r is given
+    in thousandths, and the comparison  1000 * sum_{i<c} q_(i) >= lambda * sum q  runs in
+    exact integers.  `stage1_top_p` above is the same rule in fp64; a test checks that the
+    two agree on long-tailed scores.
+    """
+    s = np.asarray(scores_f32, dtype=np.float32)
+    one = 1 << TOP_P_FRAC_BITS
+    q = [min(int(float(x) * one), one) for x in s]        # float(x) * 2^36 is exact in fp64
+    order = sorted(range(s.shape[0]), key=lambda j: (-float(s[j]), j))
+    target = int(lambda_permille) * sum(q)
+    c, run = 0, 0
+    while c < len(order) and not (1000 * run >= target):
+        run += q[order[c]]
+        c += 1
+    if k_cap is not None:
+        c = min(c, k_cap)
+    return c
+
+
 # --------------------------------------------------------------------------------------
 # Step 2: Stage II spatially uniform reduction (Eq. 7 and the text after it)
 # --------------------------------------------------------------------------------------
@@ -180,6 +208,14 @@ def select(scores_f32: np.ndarray, n_frames: int, tokens_per_frame: int, k1: int
     kept = sorted(set(v_r) | set(v_u))
     assert len(kept) == len(v_r) + len(v_u) == k_total
     return np.asarray(kept, dtype=np.int32)
+
+
+def select_top_p(scores_f32: np.ndarray, n_frames: int, tokens_per_frame: int, lambda_permille: int,
+                 k_total: int) -> tuple[np.ndarray, int]:
+    """Retention set with the Stage-I count chosen by Eq. 6 (Top-P), bounded by the whole
+    budget k_total (then Stage II adds nothing).  Returns (kept indices, Stage-I count)."""
+    k1 = stage1_top_p_fixed(scores_f32, lambda_permille, k_cap=k_total)
+    return select(scores_f32, n_frames, tokens_per_frame, k1, k_total), k1
 
 
 # --------------------------------------------------------------------------------------

@@ -7,6 +7,12 @@
 //      hence its rank inside its frame, (c) the output position of each kept token;
 //   3. the Stage-II pick test is integer arithmetic per token.
 // Everything is deterministic: no atomics decide an output.
+//
+// Top-P mode (Eq. 6): the Stage-I count is the shortest prefix of the ranking whose cumulative
+// score reaches lambda_r of the total.  The same radix descent runs on score mass instead of
+// counts.  Masses are the scores truncated to multiples of 2^-36 (capped at 1) and summed as
+// 64-bit integers, lambda_r is in thousandths: integer sums do not depend on the order of the
+// additions, so the count is a function of the scores alone.
 #include "common.cuh"
 #include "host_util.h"
 
@@ -14,14 +20,25 @@ namespace specvlm {
 
 constexpr int kSelThreads = 1024;
 constexpr int kSelMaxBatch = 64;
+constexpr int kTopPFracBits = 36;
+
+// score mass of a key (keys of non-negative floats are their bits with the top bit set)
+__device__ __forceinline__ unsigned long long key_mass(uint32_t key) {
+  const double a = (double)__uint_as_float(key & 0x7fffffffu) * (double)(1ull << kTopPFracBits);
+  const unsigned long long one = 1ull << kTopPFracBits;
+  return a >= (double)one ? one : (unsigned long long)a;
+}
 
 struct SelSeq {
   int32_t score_off, n_frames, k1, k_total, kept_off;
+  int32_t lambda_pm;                   // >= 0: Top-P mode, k1 is computed; < 0: k1 as given
 };
 struct SelParams {
   const float* scores;
   int32_t* kept_idx;
+  int32_t* k1_out;                     // [batch] Stage-I counts or null
   int32_t tokens_per_frame;
+  int32_t k1_out_base;                 // index of seq[0] in k1_out
   SelSeq seq[kSelMaxBatch];
 };
 
@@ -57,12 +74,15 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const __grid_con
   extern __shared__ uint32_t sel_smem[];
   const SelSeq sq = p.seq[blockIdx.x];
   const int T = p.tokens_per_frame, F = sq.n_frames, n_v = F * T;
-  const int k1 = sq.k1, k_total = sq.k_total;
+  int k1 = sq.k1;
+  const int k_total = sq.k_total;
   uint32_t* const key = sel_smem;                                  // [n_v] keys, later states
   int* const cf = reinterpret_cast<int*>(sel_smem + n_v);         // [F + 1] unselected before frame f
   int* const hist = cf + F + 1;                                    // [256]
   int* const warp_sums = hist + 256;                               // [32]
   int* const misc = warp_sums + 32;                                // [8]
+  unsigned long long* const mass = reinterpret_cast<unsigned long long*>(                // [256 + 2]
+      (reinterpret_cast<uintptr_t>(misc + 8) + 7) & ~static_cast<uintptr_t>(7));
   const int tid = threadIdx.x;
 
   // order-preserving map float -> uint32 (larger float <=> larger key)
@@ -70,6 +90,69 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const __grid_con
   for (int j = tid; j < n_v; j += kSelThreads) {
     const uint32_t u = __float_as_uint(sc[j]);
     key[j] = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+  }
+
+  // ---- 0. Top-P: the Stage-I count from the score mass
+  if (sq.lambda_pm >= 0) {
+    __syncthreads();
+    if (tid == 0) mass[256] = 0ull;
+    __syncthreads();
+    {
+      unsigned long long part = 0ull;
+      for (int j = tid; j < n_v; j += kSelThreads) part += key_mass(key[j]);
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+      if ((tid & 31) == 0) atomicAdd(&mass[256], part);            // integer: order-independent
+    }
+    __syncthreads();
+    const unsigned long long target = (unsigned long long)sq.lambda_pm * mass[256];   // vs 1000 * prefix mass
+    int c = 0;
+    if (target > 0ull) {
+      uint32_t pfx = 0, pfx_mask = 0;
+      unsigned long long above = 0ull;     // mass of the keys ranked before every key matching pfx
+      int n_above = 0;
+      for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int i = tid; i < 256; i += kSelThreads) {
+          hist[i] = 0;
+          mass[i] = 0ull;
+        }
+        __syncthreads();
+        for (int j = tid; j < n_v; j += kSelThreads) {
+          if ((key[j] & pfx_mask) == pfx) {
+            const uint32_t digit = (key[j] >> shift) & 255u;
+            atomicAdd(&hist[digit], 1);
+            atomicAdd(&mass[digit], key_mass(key[j]));
+          }
+        }
+        __syncthreads();
+        if (tid == 0) {
+          int d = 255;
+          unsigned long long acc = above;
+          int n = n_above;
+          for (; d > 0; --d) {
+            if (1000ull * (acc + mass[d]) >= target) break;
+            acc += mass[d];
+            n += hist[d];
+          }
+          misc[0] = d;
+          misc[1] = n;
+          mass[257] = acc;
+        }
+        __syncthreads();
+        pfx |= static_cast<uint32_t>(misc[0]) << shift;
+        pfx_mask |= 255u << shift;
+        n_above = misc[1];
+        above = mass[257];
+        __syncthreads();
+      }
+      // every key equal to pfx carries the same mass: take as many as still needed
+      const unsigned long long q = key_mass(pfx);
+      const unsigned long long need = target - 1000ull * above;      // > 0: `above` alone does not reach
+      const unsigned long long e = q > 0ull ? (need + 1000ull * q - 1ull) / (1000ull * q) : 0ull;
+      c = n_above + (int)e;
+    }
+    k1 = c < k_total ? c : k_total;
+    if (tid == 0 && p.k1_out) p.k1_out[blockIdx.x + p.k1_out_base] = k1;
   }
 
   // ---- 1. radix select of the k1-th largest key
@@ -167,26 +250,28 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const __grid_con
     if (key[j] != 0u) out[pos++] = j;
 }
 
-}  // namespace specvlm
-
-using namespace specvlm;
-
-extern "C" int32_t specvlm_select(const float* scores, const int32_t* video_cu, const int32_t* n_frames,
-                                  int32_t tokens_per_frame, const int32_t* k_stage1,
-                                  const int32_t* k_total, const int32_t* kept_cu, int32_t batch,
-                                  int32_t* kept_idx, int32_t* d_status, void* stream) {
-  (void)d_status;
-  if (!scores || !video_cu || !n_frames || !k_stage1 || !k_total || !kept_cu || !kept_idx ||
+static int32_t select_common(const float* scores, const int32_t* video_cu, const int32_t* n_frames,
+                             int32_t tokens_per_frame, const int32_t* k_stage1, const int32_t* lambda_permille,
+                             const int32_t* k_total, const int32_t* kept_cu, int32_t batch, int32_t* kept_idx,
+                             int32_t* k1_out, void* stream) {
+  if (!scores || !video_cu || !n_frames || (!k_stage1 && !lambda_permille) || !k_total || !kept_cu || !kept_idx ||
       batch < 1 || tokens_per_frame < 1)
     return SPECVLM_ERR_INVALID_ARG;
   size_t max_smem = 0;
   for (int b = 0; b < batch; ++b) {
     const int64_t n_v = (int64_t)n_frames[b] * tokens_per_frame;
     if (n_frames[b] < 1 || n_frames[b] > 1024 || n_v > 57344) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
-    if (k_stage1[b] < 0 || k_stage1[b] > k_total[b] || k_total[b] > n_v) return SPECVLM_ERR_INVALID_ARG;
+    if (k_total[b] < 0 || k_total[b] > n_v) return SPECVLM_ERR_INVALID_ARG;
+    if (lambda_permille) {
+      if (lambda_permille[b] < 0 || lambda_permille[b] > 1000) return SPECVLM_ERR_INVALID_ARG;
+    } else if (k_stage1[b] < 0 || k_stage1[b] > k_total[b]) {
+      return SPECVLM_ERR_INVALID_ARG;
+    }
     if (video_cu[b + 1] - video_cu[b] < n_v || kept_cu[b + 1] - kept_cu[b] < k_total[b])
       return SPECVLM_ERR_INVALID_ARG;
-    const size_t sm = ((size_t)n_v + n_frames[b] + 1 + 256 + 32 + 8) * 4;
+    // keys, per-frame counts, histogram, scan scratch, flags, then the 64-bit mass bins (8-byte aligned)
+    const size_t words = (size_t)n_v + n_frames[b] + 1 + 256 + 32 + 8;
+    const size_t sm = (words + (words & 1)) * 4 + (256 + 2) * 8;
     if (sm > max_smem) max_smem = sm;
   }
   if (max_smem > 232448) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
@@ -197,16 +282,44 @@ extern "C" int32_t specvlm_select(const float* scores, const int32_t* video_cu, 
   SelParams p;
   p.scores = scores;
   p.kept_idx = kept_idx;
+  p.k1_out = k1_out;
   p.tokens_per_frame = tokens_per_frame;
   for (int b0 = 0; b0 < batch; b0 += kSelMaxBatch) {
     const int nb = batch - b0 < kSelMaxBatch ? batch - b0 : kSelMaxBatch;
+    p.k1_out_base = b0;
     for (int i = 0; i < nb; ++i) {
       const int b = b0 + i;
-      p.seq[i] = SelSeq{video_cu[b], n_frames[b], k_stage1[b], k_total[b], kept_cu[b]};
+      p.seq[i] = SelSeq{video_cu[b], n_frames[b], lambda_permille ? 0 : k_stage1[b], k_total[b], kept_cu[b],
+                        lambda_permille ? lambda_permille[b] : -1};
     }
     select_kernel<<<(unsigned)nb, kSelThreads, max_smem, st>>>(p);
     const int32_t rc = launch_status();
     if (rc != SPECVLM_OK) return rc;
   }
   return SPECVLM_OK;
+}
+
+}  // namespace specvlm
+
+using namespace specvlm;
+
+extern "C" int32_t specvlm_select(const float* scores, const int32_t* video_cu, const int32_t* n_frames,
+                                  int32_t tokens_per_frame, const int32_t* k_stage1,
+                                  const int32_t* k_total, const int32_t* kept_cu, int32_t batch,
+                                  int32_t* kept_idx, int32_t* d_status, void* stream) {
+  (void)d_status;
+  if (!k_stage1) return SPECVLM_ERR_INVALID_ARG;
+  return select_common(scores, video_cu, n_frames, tokens_per_frame, k_stage1, nullptr, k_total, kept_cu, batch,
+                       kept_idx, nullptr, stream);
+}
+
+extern "C" int32_t specvlm_select_top_p(const float* scores, const int32_t* video_cu, const int32_t* n_frames,
+                                        int32_t tokens_per_frame, const int32_t* lambda_permille,
+                                        const int32_t* k_total, const int32_t* kept_cu, int32_t batch,
+                                        int32_t* kept_idx, int32_t* k_stage1_out_or_null, int32_t* d_status,
+                                        void* stream) {
+  (void)d_status;
+  if (!lambda_permille) return SPECVLM_ERR_INVALID_ARG;
+  return select_common(scores, video_cu, n_frames, tokens_per_frame, nullptr, lambda_permille, k_total, kept_cu,
+                       batch, kept_idx, k_stage1_out_or_null, stream);
 }

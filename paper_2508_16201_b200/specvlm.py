@@ -48,7 +48,7 @@ _lib = None
 EXPORTS = [
     "specvlm_version", "specvlm_status_string",
     "specvlm_stage1_scores_workspace_bytes", "specvlm_stage1_row_lse", "specvlm_stage1_scores",
-    "specvlm_select", "specvlm_gather_kv",
+    "specvlm_select", "specvlm_select_top_p", "specvlm_gather_kv",
     "specvlm_attn_workspace_bytes", "specvlm_draft_decode_attn", "specvlm_verify_attn",
     "specvlm_accept_workspace_bytes", "specvlm_accept", "specvlm_accept_noalloc",
 ]
@@ -79,6 +79,9 @@ def lib():
         L.specvlm_select.restype = c_int32
         L.specvlm_select.argtypes = [c_void_p, i32p, i32p, c_int32, i32p, i32p, i32p, c_int32, c_void_p,
                                      c_void_p, c_void_p]
+        L.specvlm_select_top_p.restype = c_int32
+        L.specvlm_select_top_p.argtypes = [c_void_p, i32p, i32p, c_int32, i32p, i32p, i32p, c_int32, c_void_p,
+                                           c_void_p, c_void_p, c_void_p]
         L.specvlm_gather_kv.restype = c_int32
         L.specvlm_gather_kv.argtypes = [kvp, c_void_p, i32p, i32p, i32p, i32p, c_int32, kvp, c_void_p,
                                         c_void_p]
@@ -267,6 +270,23 @@ def select(scores: torch.Tensor, video_cu, n_frames, tokens_per_frame: int, k_st
                               _ptr(d_status), _stream())
     _check(rc, "specvlm_select")
     return kept_idx
+
+
+def select_top_p(scores: torch.Tensor, video_cu, n_frames, tokens_per_frame: int, lambda_permille, k_total,
+                 kept_cu, kept_idx: torch.Tensor | None = None, k_stage1_out: torch.Tensor | None = None,
+                 d_status: torch.Tensor | None = None):
+    """Returns (kept_idx, k_stage1_out): the retention sets and the Stage-I counts Eq. 6 chose."""
+    batch = len(n_frames)
+    assert scores.dtype == torch.float32 and scores.is_contiguous()
+    if kept_idx is None:
+        kept_idx = torch.empty(max(int(kept_cu[-1]), 1), dtype=torch.int32, device=scores.device)
+    if k_stage1_out is None:
+        k_stage1_out = torch.empty(batch, dtype=torch.int32, device=scores.device)
+    rc = lib().specvlm_select_top_p(_ptr(scores), _i32(video_cu), _i32(n_frames), int(tokens_per_frame),
+                                    _i32(lambda_permille), _i32(k_total), _i32(kept_cu), batch, _ptr(kept_idx),
+                                    _ptr(k_stage1_out), _ptr(d_status), _stream())
+    _check(rc, "specvlm_select_top_p")
+    return kept_idx, k_stage1_out
 
 
 # ---------------------------------------------------------------------------------- gather

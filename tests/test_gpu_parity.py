@@ -237,6 +237,52 @@ def test_select_stage_split_extremes():
         assert np.array_equal(got, oracle.select(s, 4, 196, k1, kt))
 
 
+def _long_tailed(rng, n):
+    a = rng.pareto(1.5, size=n).astype(np.float64)
+    return (a / a.sum()).astype(np.float32)
+
+
+@pytest.mark.parametrize("lam", [0, 400, 500, 900, 1000])
+def test_select_top_p_bit_exact(lam):
+    """Eq. 6 as a mode of the selection: Stage-I counts and kept sets equal the oracle's, on
+    long-tailed scores, on scores full of ties, and on a ragged batch with per-sequence lambda."""
+    rng = np.random.default_rng(40 + lam)
+    frames, T = [32, 4, 128, 1], 196
+    scores, video_cu, kts, kept_cu = [], [0], [], [0]
+    for i, F in enumerate(frames):
+        nv = F * T
+        s = _long_tailed(rng, nv) if i != 1 else (rng.integers(0, 4, nv) * 0.0078125).astype(np.float32)
+        scores.append(s)
+        video_cu.append(video_cu[-1] + nv)
+        kts.append(nv // 10 if i != 3 else nv)          # last sequence: budget = everything
+        kept_cu.append(kept_cu[-1] + kts[-1])
+    lams = [lam, lam, max(lam - 100, 0), lam]
+    dev = torch.from_numpy(np.concatenate(scores)).cuda()
+    kept, k1 = specvlm.select_top_p(dev, video_cu, frames, T, lams, kts, kept_cu)
+    kept, k1 = kept.cpu().numpy(), k1.cpu().numpy()
+    for b, F in enumerate(frames):
+        ref, ref_k1 = oracle.select_top_p(scores[b], F, T, lams[b], kts[b])
+        assert int(k1[b]) == ref_k1, f"sequence {b}: Stage-I count {int(k1[b])} vs {ref_k1}"
+        assert np.array_equal(kept[kept_cu[b]:kept_cu[b + 1]], ref), f"sequence {b}"
+
+
+def test_select_top_p_on_rated_scores_cfg1():
+    """Top-P on real ratings of the tiny workload: the oracle's fp32 scores through both sides."""
+    from gpu_util import make_cache, host_view
+    w = synth.workload(1)
+    nv, nt = w.n_video(), w.n_text[0]
+    cache, _, _ = make_cache(w.t_layers, w.t_kv_heads, w.head_dim, [nv + nt], paged=False, seed=0)
+    q = synth.randn_bf16((w.t_layers, nt, w.t_q_heads, w.head_dim), "cuda", 0, "Qtext")
+    synth.plant_salient_(cache.k[:, 0, :, :nv, :], q, synth.salient_set(nv, w.planted_permille, 0))
+    k_host = host_view(cache.k, None, [nv + nt])
+    a = oracle.stage1_scores(bits(q), k_host[0], 0, nv, nv, 1.0 / math.sqrt(w.head_dim)).astype(np.float32)
+    for lam in (400, 500):
+        kept, k1 = specvlm.select_top_p(torch.from_numpy(a).cuda(), [0, nv], [w.n_frames[0]], w.tokens_per_frame,
+                                        [lam], [nv // 2], [0, nv // 2])
+        ref, ref_k1 = oracle.select_top_p(a, w.n_frames[0], w.tokens_per_frame, lam, nv // 2)
+        assert int(k1[0]) == ref_k1 and np.array_equal(kept.cpu().numpy(), ref)
+
+
 # ------------------------------------------------------------------------------- gather
 @pytest.mark.parametrize("src_paged,dst_paged", [(False, False), (True, True), (True, False)])
 def test_gather_bit_exact(src_paged, dst_paged):

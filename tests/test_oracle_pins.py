@@ -197,6 +197,32 @@ def test_top_p_count():
     assert oracle.stage1_top_p(s[::-1].copy(), 0.41) == 2        # order of the input is irrelevant
 
 
+def test_top_p_fixed_point_count():
+    """The integer form of Eq. 6 that the GPU decision uses: hand-worked dyadic cases (every value
+    exact in 2^-36 units), ties, the budget cap, and agreement with the fp64 form on long-tailed
+    random scores, where no cumulative sum sits within rounding of the threshold."""
+    s = np.array([0.125, 0.5, 0.125, 0.25], dtype=np.float32)       # ranking: 1, 3, 0, 2; total 1
+    assert oracle.stage1_top_p_fixed(s, 500) == 1                    # 0.5 >= 0.5
+    assert oracle.stage1_top_p_fixed(s, 501) == 2
+    assert oracle.stage1_top_p_fixed(s, 750) == 2
+    assert oracle.stage1_top_p_fixed(s, 751) == 3
+    assert oracle.stage1_top_p_fixed(s, 876) == 4
+    assert oracle.stage1_top_p_fixed(s, 1000) == 4
+    assert oracle.stage1_top_p_fixed(s, 0) == 0
+    assert oracle.stage1_top_p_fixed(s, 1000, k_cap=3) == 3
+    kept, k1 = oracle.select_top_p(s, 1, 4, 751, 3)
+    assert k1 == 3 and kept.tolist() == [0, 1, 3]                    # the tie 0.125 goes to the lower index
+    kept, k1 = oracle.select_top_p(s, 1, 4, 500, 3)                  # Stage I keeps 1, Stage II adds 2 of the rest
+    assert k1 == 1 and len(kept) == 3 and 1 in kept.tolist()
+    assert oracle.stage1_top_p_fixed(np.zeros(5, dtype=np.float32), 400) == 0   # no mass: nothing to reach
+    rng = np.random.default_rng(11)
+    for lam in (400, 500, 900):
+        for _ in range(5):
+            a = rng.pareto(1.5, size=3000).astype(np.float32)
+            a = (a / a.sum()).astype(np.float32)                     # long-tailed, sums to ~1 like a rating
+            assert oracle.stage1_top_p_fixed(a, lam) == oracle.stage1_top_p(a, lam / 1000.0)
+
+
 # ----------------------------------------------------------------------------- gather
 def test_gather_is_fancy_index():
     g = torch.Generator().manual_seed(3)
