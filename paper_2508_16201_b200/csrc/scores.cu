@@ -693,12 +693,14 @@ scores_colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
 // With the rows on the TMEM lanes an epilogue thread owns one row: it reads its 128 logits of a
 // tile with tcgen05.ld and keeps the row's running (max, sum) in two registers -- the row
 // reduction needs no cross-thread step.  The kernel is bound by the exponentials (one per logit),
-// not by the tensor pipe; the second CTA on the SM fills the first one's TMEM-load latency.
+// not by the tensor pipe; two epilogue groups per CTA (alternate tiles, one accumulator buffer
+// each, their (max, sum) pairs merged at the end) and a second CTA on the SM keep the
+// special-function units fed while other warps wait for their TMEM loads.
 // Warps: 0 = TMA producer (Q tile once, K tiles through a ring), 1 = TMEM allocation + MMA issue,
-// 2..5 = epilogue (one TMEM lane quadrant each).
+// 2..5 and 6..9 = the epilogue groups (one TMEM lane quadrant per warp).
 // ---------------------------------------------------------------------------------------------
 template <int D, int STAGES>
-__global__ void __launch_bounds__(192, 2)
+__global__ void __launch_bounds__(320, 2)
 scores_lse_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
                      const __grid_constant__ ScoreParams p) {
   constexpr int TILE_BYTES = kKeyTile * D * 2;
@@ -720,6 +722,7 @@ scores_lse_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
   uint8_t* const tail = smem + kTail + 16 * STAGES + 40;
   volatile int* const abort_flag = reinterpret_cast<volatile int*>(tail);
   volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(tail + 8);
+  float2* const ml_sm = reinterpret_cast<float2*>(tail + 16);    // [128] group 1's (max, sum) per row
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int b = find_seq(p, blockIdx.x);
@@ -804,7 +807,8 @@ scores_lse_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
       if (!ok && p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
     }
   } else {
-    // ---------------------------------------------------------------- epilogue: 4 warps, 128 rows
+    // ---------------------------------------------------------------- epilogue: 2 groups x 4 warps, 128 rows
+    const int grp = (warp - 2) >> 2;            // tiles with (index & 1) == grp, accumulator buffer grp
     const int quad = warp & 3;                  // TMEM lanes [32 * quad, 32 * quad + 32)
     const int r = quad * 32 + lane;             // this thread's row
     const int il = r / p.group, hg = r - il * p.group;
@@ -812,8 +816,8 @@ scores_lse_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     const int first_lim = sq.text_start + i_first + 1;
     float m = -INFINITY, l = 0.f;
     bool alive = true;
-    for (int i = 0; i < n_kt; ++i) {
-      const int buf = i & 1;
+    for (int i = grp; i < n_kt; i += 2) {
+      const int buf = grp;
       if (alive && !mbar_wait(bar_tfull + 8 * buf, (i >> 1) & 1, abort_flag)) alive = false;
       alive = __all_sync(0xffffffffu, alive);   // warp-uniform: the TMEM loads below are warp-collective
       if (!alive) break;
@@ -855,10 +859,17 @@ scores_lse_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         m = mn;
       }
     }
+    // merge the two groups' running pairs (every wait above is bounded, so both get here)
+    if (grp == 1) ml_sm[r] = make_float2(m, l);
+    asm volatile("bar.sync 1, 256;" ::: "memory");
     if (alive && !*abort_flag) {
-      if (r < rows_valid)
+      if (grp == 0 && r < rows_valid) {
+        const float2 o = ml_sm[r];
+        const float mm = fmaxf(m, o.x);
+        const float ll = (l > 0.f ? l * fast_exp2(m - mm) : 0.f) + (o.y > 0.f ? o.y * fast_exp2(o.x - mm) : 0.f);
         p.lse[((size_t)layer * p.sum_text + sq.text_off + i_first + il) * p.n_q_heads + g * p.group + hg] =
-            (m + log2f(l)) * kLn2;
+            (mm + log2f(ll)) * kLn2;
+      }
     } else if (p.d_status && r == 0) {
       *p.d_status = SPECVLM_ERR_TIMEOUT;
     }
@@ -1002,11 +1013,11 @@ static int32_t launch_lse(ScoreSetup& su, cudaStream_t st) {
     return launch_status();
   }
   constexpr int STAGES = 2;                              // two CTAs per SM: 3 x 32 KB each at d = 128
-  constexpr int SMEM = (1 + STAGES) * kKeyTile * D * 2 + 1024 + 16 * STAGES + 40 + 16;
+  constexpr int SMEM = (1 + STAGES) * kKeyTile * D * 2 + 1024 + 16 * STAGES + 40 + 16 + 128 * 8;
   auto k = scores_lse_tc_kernel<D, STAGES>;
   if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
     return SPECVLM_ERR_CUDA;
-  k<<<grid, 192, SMEM, st>>>(su.tk, su.tq, su.p1);
+  k<<<grid, 320, SMEM, st>>>(su.tk, su.tq, su.p1);
   return launch_status();
 }
 
