@@ -214,6 +214,32 @@ int32_t specvlm_accept(const float* target_logits, const int32_t* draft_tokens, 
                        int32_t* target_argmax_or_null, void* ws, size_t ws_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Cache maintenance around a step (Section 3.1: the gamma drafted tokens are generated by the
+ * draft one at a time and verified by the target in one pass; rejected tokens are discarded).
+ *
+ * specvlm_append_kv writes the K/V rows of n_new new tokens of every sequence behind its current
+ * end -- token t of sequence b goes to position seq_lens[b] + t of every layer and KV head -- and
+ * then adds n_new to seq_lens[b].  The attention calls expect exactly that state (the cache
+ * already holds the new tokens).
+ *   kv           host struct of the cache to extend (kv->seq_lens is ignored, see seq_lens_inout)
+ *   new_k, new_v device bf16 [n_layers][batch][n_new][n_kv_heads][head_dim]
+ *   seq_lens_inout  device int32 [batch], read then updated on the stream
+ * A sequence without room (seq_lens[b] + n_new > kv->max_seq_len) is left unchanged and
+ * SPECVLM_ERR_INVALID_ARG is stored to d_status.  With a block table the pages of the new
+ * positions must already be mapped.
+ *
+ * specvlm_rollback_kv drops the rejected drafts after verification: a cache that held the
+ * gamma + 1 tokens of the window keeps accept_len[b] + 1 of them,
+ *   seq_lens[b] -= gamma - accept_len[b].
+ * No row is moved: rows past a sequence's length are never read.
+ *   accept_len   device int32 [batch], as written by specvlm_accept (0 .. gamma)
+ */
+int32_t specvlm_append_kv(const specvlm_kv_t* kv, const void* new_k, const void* new_v, int32_t batch,
+                          int32_t n_new, int32_t* seq_lens_inout, int32_t* d_status, void* stream);
+int32_t specvlm_rollback_kv(int32_t* seq_lens_inout, const int32_t* accept_len, int32_t batch,
+                            int32_t gamma, int32_t* d_status, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * specvlm_accept without any caller-provided scratch.  (The paper has no counterpart: this is a
  * packaging variant of step 4c, same results.)
  *

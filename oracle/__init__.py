@@ -233,6 +233,27 @@ def gather_kv(src: np.ndarray, kept_idx: np.ndarray, video_start: int, n_video: 
 
 
 # --------------------------------------------------------------------------------------
+# Cache maintenance around a step (Section 3.1: drafted tokens enter the caches before the
+# attention over them; rejected ones are discarded after verification)
+# --------------------------------------------------------------------------------------
+def append_kv(cache: np.ndarray, new: np.ndarray, seq_len: int) -> tuple[np.ndarray, int]:
+    """cache: [n_layers][Hkv][capacity][d] of one sequence, new: [n_layers][n_new][Hkv][d].
+    Returns (cache with the new rows at positions seq_len .. seq_len + n_new - 1, new length)."""
+    out = cache.copy()
+    n_new = new.shape[1]
+    assert seq_len + n_new <= cache.shape[2]
+    for t in range(n_new):
+        out[:, :, seq_len + t, :] = new[:, t, :, :]
+    return out, seq_len + n_new
+
+
+def rollback_len(seq_len: int, gamma: int, accept_len: int) -> int:
+    """Of the gamma + 1 tokens of the verification window, accept_len + 1 stay in the cache."""
+    assert 0 <= accept_len <= gamma <= seq_len - 1
+    return seq_len - (gamma + 1) + (accept_len + 1)
+
+
+# --------------------------------------------------------------------------------------
 # Step 4a/4b: attention
 # --------------------------------------------------------------------------------------
 def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, kv_len: int, sm_scale: float):

@@ -1,0 +1,115 @@
+// Cache maintenance around a speculative step: the K/V of the tokens a step feeds to a model are
+// appended to that model's cache before its attention runs, and the rows of rejected drafts are
+// dropped afterwards by shortening the sequence.  Pure byte movement and integer arithmetic.
+#include "common.cuh"
+#include "host_util.h"
+
+namespace specvlm {
+
+struct AppendParams {
+  const uint4* new_k;      // [L][B][n_new][Hkv][D] in 16-byte units
+  const uint4* new_v;
+  uint4* k;
+  uint4* v;
+  const int32_t* table;
+  const int32_t* seq_lens; // lengths before the append
+  int32_t* d_status;
+  int64_t s_layer, s_block, s_head, s_token;   // cache strides in 16-byte units
+  int32_t block_tokens, max_blocks, max_seq_len;
+  int32_t n_layers, batch, n_new, n_kv_heads, chunks_per_row;
+};
+
+// one thread per 16-byte chunk of a new token row
+__global__ void __launch_bounds__(256) append_kv_kernel(const __grid_constant__ AppendParams p) {
+  const int64_t total = (int64_t)p.n_layers * p.batch * p.n_new * p.n_kv_heads * p.chunks_per_row;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    int64_t r = i;
+    const int chunk = (int)(r % p.chunks_per_row); r /= p.chunks_per_row;
+    const int head = (int)(r % p.n_kv_heads); r /= p.n_kv_heads;
+    const int t = (int)(r % p.n_new); r /= p.n_new;
+    const int b = (int)(r % p.batch);
+    const int layer = (int)(r / p.batch);
+    const int len = p.seq_lens[b];
+    const int pos = len + t;
+    if (len < 0 || pos >= p.max_seq_len) {
+      // no room (or a corrupt length): leave the cache alone and report
+      if (p.d_status) *p.d_status = SPECVLM_ERR_INVALID_ARG;
+      continue;
+    }
+    int blk = b, off = pos;
+    if (p.table) {
+      blk = __ldg(p.table + (size_t)b * p.max_blocks + pos / p.block_tokens);
+      off = pos % p.block_tokens;
+    }
+    const int64_t dst = layer * p.s_layer + blk * p.s_block + head * p.s_head + off * p.s_token + chunk;
+    p.k[dst] = __ldcs(p.new_k + i);
+    p.v[dst] = __ldcs(p.new_v + i);
+  }
+}
+
+// seq_lens[b] += delta, or, with accept_len, seq_lens[b] -= gamma - accept_len[b]
+__global__ void seq_len_update_kernel(int32_t* seq_lens, const int32_t* accept_len, int batch, int delta, int gamma,
+                                      int max_seq_len, int32_t* d_status) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= batch) return;
+  int n = seq_lens[b];
+  if (accept_len) {
+    const int a = accept_len[b];
+    if (a < 0 || a > gamma || n < gamma + 1) {
+      if (d_status) *d_status = SPECVLM_ERR_INVALID_ARG;
+      return;
+    }
+    n -= gamma - a;
+  } else {
+    if (n < 0 || n + delta > max_seq_len) return;     // the append kernel has reported it
+    n += delta;
+  }
+  seq_lens[b] = n;
+}
+
+}  // namespace specvlm
+
+using namespace specvlm;
+
+extern "C" int32_t specvlm_append_kv(const specvlm_kv_t* kv, const void* new_k, const void* new_v, int32_t batch,
+                                     int32_t n_new, int32_t* seq_lens_inout, int32_t* d_status, void* stream) {
+  if (!kv || !new_k || !new_v || !seq_lens_inout || n_new < 1) return SPECVLM_ERR_INVALID_ARG;
+  specvlm_kv_t c = *kv;
+  c.seq_lens = seq_lens_inout;
+  int32_t rc = validate_kv(&c, batch, true);
+  if (rc != SPECVLM_OK) return rc;
+  if (!aligned16(new_k) || !aligned16(new_v) || n_new > c.max_seq_len) return SPECVLM_ERR_INVALID_ARG;
+  AppendParams p;
+  p.new_k = static_cast<const uint4*>(new_k);
+  p.new_v = static_cast<const uint4*>(new_v);
+  p.k = static_cast<uint4*>(c.k);
+  p.v = static_cast<uint4*>(c.v);
+  p.table = c.block_table;
+  p.seq_lens = seq_lens_inout;
+  p.d_status = d_status;
+  p.s_layer = c.stride_layer / 8; p.s_block = c.stride_block / 8; p.s_head = c.stride_head / 8;
+  p.s_token = c.stride_token / 8;
+  p.block_tokens = c.block_tokens; p.max_blocks = c.max_blocks; p.max_seq_len = c.max_seq_len;
+  p.n_layers = c.n_layers; p.batch = batch; p.n_new = n_new; p.n_kv_heads = c.n_kv_heads;
+  p.chunks_per_row = c.head_dim / 8;
+  const int64_t total = (int64_t)p.n_layers * batch * n_new * p.n_kv_heads * p.chunks_per_row;
+  int64_t blocks = (total + 255) / 256;
+  const int64_t cap = (int64_t)sm_count() * 8;
+  if (blocks > cap) blocks = cap;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  append_kv_kernel<<<(unsigned)blocks, 256, 0, st>>>(p);
+  rc = launch_status();
+  if (rc != SPECVLM_OK) return rc;
+  // the lengths change only after every row has been placed by the kernel above
+  seq_len_update_kernel<<<(unsigned)((batch + 127) / 128), 128, 0, st>>>(seq_lens_inout, nullptr, batch, n_new, 0,
+                                                                         c.max_seq_len, d_status);
+  return launch_status();
+}
+
+extern "C" int32_t specvlm_rollback_kv(int32_t* seq_lens_inout, const int32_t* accept_len, int32_t batch,
+                                       int32_t gamma, int32_t* d_status, void* stream) {
+  if (!seq_lens_inout || !accept_len || batch < 1 || gamma < 0) return SPECVLM_ERR_INVALID_ARG;
+  seq_len_update_kernel<<<(unsigned)((batch + 127) / 128), 128, 0, static_cast<cudaStream_t>(stream)>>>(
+      seq_lens_inout, accept_len, batch, 0, gamma, 0, d_status);
+  return launch_status();
+}

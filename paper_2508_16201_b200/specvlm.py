@@ -51,6 +51,7 @@ EXPORTS = [
     "specvlm_select", "specvlm_select_top_p", "specvlm_gather_kv",
     "specvlm_attn_workspace_bytes", "specvlm_draft_decode_attn", "specvlm_verify_attn",
     "specvlm_accept_workspace_bytes", "specvlm_accept", "specvlm_accept_noalloc",
+    "specvlm_append_kv", "specvlm_rollback_kv",
 ]
 
 
@@ -82,6 +83,10 @@ def lib():
         L.specvlm_select_top_p.restype = c_int32
         L.specvlm_select_top_p.argtypes = [c_void_p, i32p, i32p, c_int32, i32p, i32p, i32p, c_int32, c_void_p,
                                            c_void_p, c_void_p, c_void_p]
+        L.specvlm_append_kv.restype = c_int32
+        L.specvlm_append_kv.argtypes = [kvp, c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p]
+        L.specvlm_rollback_kv.restype = c_int32
+        L.specvlm_rollback_kv.argtypes = [c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p]
         L.specvlm_gather_kv.restype = c_int32
         L.specvlm_gather_kv.argtypes = [kvp, c_void_p, i32p, i32p, i32p, i32p, c_int32, kvp, c_void_p,
                                         c_void_p]
@@ -298,6 +303,24 @@ def gather_kv(src: KvCache, kept_idx: torch.Tensor, kept_cu, video_start, video_
                                  _i32(video_len), _i32(src_len), batch, byref(dst.struct), _ptr(d_status),
                                  _stream())
     _check(rc, "specvlm_gather_kv")
+
+
+# ---------------------------------------------------------------------------------- cache maintenance
+def append_kv(kv: KvCache, new_k: torch.Tensor, new_v: torch.Tensor, d_status: torch.Tensor | None = None) -> None:
+    """new_k / new_v: bf16 [n_layers][batch][n_new][n_kv_heads][head_dim]; kv.seq_lens is updated."""
+    assert new_k.dtype == torch.bfloat16 and new_k.is_contiguous() and new_v.is_contiguous()
+    assert new_k.shape == new_v.shape and new_k.dim() == 5
+    rc = lib().specvlm_append_kv(byref(kv.struct), _ptr(new_k), _ptr(new_v), new_k.shape[1], new_k.shape[2],
+                                 _ptr(kv.seq_lens), _ptr(d_status), _stream())
+    _check(rc, "specvlm_append_kv")
+
+
+def rollback_kv(seq_lens: torch.Tensor, accept_len: torch.Tensor, gamma: int,
+                d_status: torch.Tensor | None = None) -> None:
+    assert seq_lens.dtype == torch.int32 and accept_len.dtype == torch.int32
+    rc = lib().specvlm_rollback_kv(_ptr(seq_lens), _ptr(accept_len), seq_lens.numel(), int(gamma), _ptr(d_status),
+                                   _stream())
+    _check(rc, "specvlm_rollback_kv")
 
 
 # ---------------------------------------------------------------------------------- accept

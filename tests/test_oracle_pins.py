@@ -328,3 +328,19 @@ def test_speedup_formula():
     # Eq. 3 special cases: a free draft and memory-bound verification give speedup = tau
     assert oracle.sd_speedup(3.0, 5, 0.0, 1.0, 1.0) == 3.0
     assert abs(oracle.sd_speedup(3.48, 5, 0.1, 1.0, 1.0) - 3.48 / 1.5) < 1e-12
+
+
+# ----------------------------------------------------------------------------- cache maintenance
+def test_append_and_rollback():
+    rng = np.random.default_rng(8)
+    cache = rng.integers(0, 65535, (2, 3, 10, 4)).astype(np.uint16)
+    new = rng.integers(0, 65535, (2, 2, 3, 4)).astype(np.uint16)
+    out, n = oracle.append_kv(cache, new, 5)
+    assert n == 7
+    assert np.array_equal(out[:, :, :5], cache[:, :, :5]) and np.array_equal(out[:, :, 7:], cache[:, :, 7:])
+    assert np.array_equal(out[1, 2, 6], new[1, 1, 2]) and np.array_equal(out[0, 0, 5], new[0, 0, 0])
+    # window of gamma + 1 = 5 tokens at the end of 20: all drafts accepted keeps them all, none keeps one
+    assert oracle.rollback_len(20, 4, 4) == 20 and oracle.rollback_len(20, 4, 0) == 16
+    assert oracle.rollback_len(20, 4, 2) == 18
+    # appending gamma + 1 tokens then rolling back with n accepted leaves old + n + 1 tokens
+    assert oracle.rollback_len(13 + 6, 5, 3) == 13 + 3 + 1
