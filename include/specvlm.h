@@ -184,7 +184,7 @@ int32_t specvlm_gather_kv(const specvlm_kv_t* src, const int32_t* kept_idx, cons
  *   ws          device scratch, specvlm_attn_workspace_bytes(kv, batch, n_q_heads, gamma)
  * fp32 softmax and accumulation; probabilities are rounded to bf16 before the PV product.
  * Supported: head_dim 64/128; group = n_q_heads/n_kv_heads in 1..16; 0 <= gamma <= 8;
- * group * (gamma+1) <= 96.
+ * group * (gamma+1) <= 128; batch <= 127 when group * (gamma+1) > 16.
  */
 size_t specvlm_attn_workspace_bytes(const specvlm_kv_t* kv, int32_t batch, int32_t n_q_heads,
                                     int32_t gamma);
@@ -238,6 +238,49 @@ int32_t specvlm_append_kv(const specvlm_kv_t* kv, const void* new_k, const void*
                           int32_t n_new, int32_t* seq_lens_inout, int32_t* d_status, void* stream);
 int32_t specvlm_rollback_kv(int32_t* seq_lens_inout, const int32_t* accept_len, int32_t batch,
                             int32_t gamma, int32_t* d_status, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Tree drafting (the paper's experimental set-up drafts a static token tree and reports chain
+ * drafting as the ablation): the verification window holds the n_nodes nodes of a tree instead
+ * of a chain.  Node 0 is the root (the last committed token); parents[b][t] < t is the parent of
+ * node t, -1 marks a root.  A chain is the tree parents[t] = t - 1.
+ *
+ * specvlm_verify_tree_attn: as specvlm_verify_attn, but query node t sees the keys before the
+ * window (positions 0 .. seq_len - n_nodes - 1) and, inside the window, the rows of its
+ * ancestors and its own.
+ *   parents   device int32 [batch][n_nodes]
+ *   q, out    device bf16 [n_layers][batch][n_nodes][n_q_heads][head_dim]
+ *   ws        device scratch, specvlm_verify_tree_workspace_bytes(kv, batch, n_q_heads, n_nodes)
+ * Supported: n_nodes <= 32 and (n_q_heads / n_kv_heads) * n_nodes <= 128.  A parents array that is
+ * not in topological order stores SPECVLM_ERR_INVALID_ARG to d_status.
+ *
+ * specvlm_accept_tree: greedy acceptance along the tree.  With g[t] = argmax of node t's target
+ * logits (lowest index among equal maxima), start at the root and step to the child whose token is
+ * g[current] (lowest node index among equal children) until no child matches.
+ *   target_logits  device fp32 [batch][n_nodes][vocab]
+ *   node_tokens    device int32 [batch][n_nodes]: the drafted token of each node (entry 0 unused)
+ *   accept_len     device int32 [batch] out: accepted drafts
+ *   next_token     device int32 [batch] out: g of the last accepted node
+ *   path           device int32 [batch][n_nodes] out: the accepted nodes in order, then -1
+ *   ws             device scratch, specvlm_accept_workspace_bytes(batch, n_nodes - 1, vocab)
+ *
+ * specvlm_compact_tree_kv: after acceptance the rows of the accepted nodes move up behind the
+ * root (window position path[i] -> position 1 + i) and the sequence keeps 1 + accept_len of the
+ * window's n_nodes rows, so that the cache is a plain sequence again.
+ */
+size_t specvlm_verify_tree_workspace_bytes(const specvlm_kv_t* kv, int32_t batch, int32_t n_q_heads,
+                                           int32_t n_nodes);
+int32_t specvlm_verify_tree_attn(const specvlm_kv_t* kv, const void* q, const int32_t* parents,
+                                 int32_t batch, int32_t n_q_heads, int32_t n_nodes, float sm_scale,
+                                 void* out, float* lse_or_null, void* ws, size_t ws_bytes,
+                                 int32_t* d_status, void* stream);
+int32_t specvlm_accept_tree(const float* target_logits, const int32_t* node_tokens, const int32_t* parents,
+                            int32_t batch, int32_t n_nodes, int32_t vocab, int32_t* accept_len,
+                            int32_t* next_token, int32_t* path, int32_t* target_argmax_or_null, void* ws,
+                            size_t ws_bytes, void* stream);
+int32_t specvlm_compact_tree_kv(const specvlm_kv_t* kv, const int32_t* path, const int32_t* accept_len,
+                                int32_t batch, int32_t n_nodes, int32_t* seq_lens_inout, int32_t* d_status,
+                                void* stream);
 
 /* ---------------------------------------------------------------------------------------------
  * specvlm_accept without any caller-provided scratch.  (The paper has no counterpart: this is a

@@ -330,3 +330,84 @@ def accept_fast(target_logits: np.ndarray, draft_tokens: np.ndarray):
 def sd_speedup(tau: float, gamma: int, t_draft: float, t_target: float, t_verify: float) -> float:
     """Eq. 3: speedup = tau / (gamma * T_d / T_t + T_t^gamma / T_t)."""
     return tau / (gamma * t_draft / t_target + t_verify / t_target)
+
+
+# --------------------------------------------------------------------------------------
+# Tree drafting (the paper's default draft shape, experimental set-up): the window holds a tree
+# of drafted tokens instead of a chain.  Node 0 is the root (the last committed token);
+# parents[t] < t is node t's parent, -1 for a root.
+# --------------------------------------------------------------------------------------
+def tree_ancestors(parents) -> list[list[int]]:
+    """For every node the window positions it attends: its ancestors and itself, ascending."""
+    out = []
+    for t in range(len(parents)):
+        chain, cur = [t], int(parents[t])
+        while cur >= 0:
+            assert cur < chain[-1], "parents must point to earlier nodes"
+            chain.append(cur)
+            cur = int(parents[cur])
+        out.append(sorted(chain))
+    return out
+
+
+def attention_tree(q: np.ndarray, k: np.ndarray, v: np.ndarray, kv_len: int, parents, sm_scale: float):
+    """Verification attention over a drafted tree.  q: uint16 [n_nodes][Hq][d]; k, v: uint16
+    [Hkv][>= kv_len][d], whose last n_nodes valid rows are the tree's nodes in node order.  Node t
+    sees every key before the window and the window rows of its ancestors and itself.
+    Plain two-pass softmax in fp64.  Returns (out [n_nodes][Hq][d], lse [n_nodes][Hq])."""
+    qf, kf, vf = bf16_bits_to_f64(_u16(q)), bf16_bits_to_f64(_u16(k)), bf16_bits_to_f64(_u16(v))
+    n_nodes, hq, d = qf.shape
+    hkv = kf.shape[0]
+    group = hq // hkv
+    old = kv_len - n_nodes
+    anc = tree_ancestors(parents)
+    out = np.zeros((n_nodes, hq, d))
+    lse = np.zeros((n_nodes, hq))
+    for t in range(n_nodes):
+        keys = list(range(old)) + [old + a for a in anc[t]]
+        for h in range(hq):
+            g = h // group
+            s = (kf[g, keys, :] @ qf[t, h, :]) * sm_scale
+            m = s.max()
+            e = np.exp(s - m)
+            z = e.sum()
+            out[t, h] = (e / z) @ vf[g, keys, :]
+            lse[t, h] = m + math.log(z)
+    return out, lse
+
+
+def accept_tree(logits: np.ndarray, node_tokens, parents) -> tuple[int, int, list[int]]:
+    """Greedy acceptance along the tree: starting at the root, step to the child whose token is
+    the target's arg-max at the current node (lowest node index among equal children) until no
+    child matches.  Returns (accepted drafts, the target's token after the last accepted node,
+    accepted node indices in order)."""
+    n_nodes = logits.shape[0]
+    g = []
+    for t in range(n_nodes):
+        best, arg = -math.inf, 0
+        for i, x in enumerate(logits[t].tolist()):
+            if x > best:
+                best, arg = x, i
+        g.append(arg)
+    cur, path = 0, []
+    while True:
+        nxt = -1
+        for c in range(cur + 1, n_nodes):
+            if int(parents[c]) == cur and int(node_tokens[c]) == g[cur]:
+                nxt = c
+                break
+        if nxt < 0:
+            break
+        path.append(nxt)
+        cur = nxt
+    return len(path), g[cur], path
+
+
+def compact_tree_kv(cache: np.ndarray, seq_len: int, n_nodes: int, path) -> tuple[np.ndarray, int]:
+    """After tree acceptance: the accepted nodes' rows move up behind the root so that the cache is
+    a plain sequence again.  cache: [..., tokens, d].  Returns (cache, new length = old + 1 + len(path))."""
+    out = cache.copy()
+    old = seq_len - n_nodes
+    for i, node in enumerate(path):
+        out[..., old + 1 + i, :] = cache[..., old + node, :]
+    return out, old + 1 + len(path)

@@ -97,6 +97,52 @@ __global__ void accept_finish_kernel(const Cand* __restrict__ part, int n_chunks
   }
 }
 
+// Tree drafting: one warp per node finishes its arg-max, then one thread walks from the root to
+// the child whose token is the target's choice at the current node, as long as there is one.
+__global__ void accept_tree_finish_kernel(const Cand* __restrict__ part, int n_chunks,
+                                          const int32_t* __restrict__ node_tokens,
+                                          const int32_t* __restrict__ parents, int n_nodes,
+                                          int32_t* __restrict__ accept_len, int32_t* __restrict__ next_token,
+                                          int32_t* __restrict__ path, int32_t* __restrict__ g_out) {
+  __shared__ int g_sm[32];
+  const int b = blockIdx.x, t = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const Cand* row = part + ((size_t)b * n_nodes + t) * n_chunks;
+  float bv = -INFINITY;
+  int bi = 0x7fffffff;
+  for (int c = lane; c < n_chunks; c += 32) take_better(bv, bi, row[c].v, row[c].i);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+    const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+    take_better(bv, bi, ov, oi);
+  }
+  if (lane == 0) {
+    g_sm[t] = bi;
+    if (g_out) g_out[(size_t)b * n_nodes + t] = bi;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int32_t* tok = node_tokens + (size_t)b * n_nodes;
+    const int32_t* par = parents + (size_t)b * n_nodes;
+    int32_t* pth = path + (size_t)b * n_nodes;
+    int cur = 0, n = 0;
+    while (true) {
+      int nxt = -1;
+      for (int c = cur + 1; c < n_nodes; ++c)
+        if (par[c] == cur && tok[c] == g_sm[cur]) {
+          nxt = c;
+          break;
+        }
+      if (nxt < 0) break;
+      pth[n++] = nxt;
+      cur = nxt;
+    }
+    for (int i = n; i < n_nodes; ++i) pth[i] = -1;
+    accept_len[b] = n;
+    next_token[b] = g_sm[cur];
+  }
+}
+
 // Built-in scratch of specvlm_accept_noalloc: room for kStaticCands (row, vocab chunk) candidates.
 // Every GPU that loads the library holds these 128 KB until the process exits.
 constexpr int kStaticCands = 16384;
@@ -176,5 +222,29 @@ extern "C" int32_t specvlm_accept_noalloc(const float* target_logits, const int3
   accept_finish_kernel<<<(unsigned)batch, 32 * (gamma + 1), 0, st>>>(part, n_chunks, draft_tokens, gamma,
                                                                      accept_len, next_token,
                                                                      target_argmax_or_null);
+  return launch_status();
+}
+
+extern "C" int32_t specvlm_accept_tree(const float* target_logits, const int32_t* node_tokens,
+                                       const int32_t* parents, int32_t batch, int32_t n_nodes, int32_t vocab,
+                                       int32_t* accept_len, int32_t* next_token, int32_t* path,
+                                       int32_t* target_argmax_or_null, void* ws, size_t ws_bytes, void* stream) {
+  if (!target_logits || !node_tokens || !parents || !accept_len || !next_token || !path || !ws || batch < 1 ||
+      n_nodes < 1 || vocab < 1)
+    return SPECVLM_ERR_INVALID_ARG;
+  if (n_nodes > 32 || (int64_t)batch * n_nodes > 65535) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(target_logits) & 3u) || (reinterpret_cast<uintptr_t>(ws) & 7u))
+    return SPECVLM_ERR_INVALID_ARG;
+  if (ws_bytes < specvlm_accept_workspace_bytes(batch, n_nodes - 1, vocab)) return SPECVLM_ERR_WORKSPACE_TOO_SMALL;
+  const int n_chunks = (vocab + kAcceptChunk - 1) / kAcceptChunk;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  Cand* part = static_cast<Cand*>(ws);
+  accept_partial_kernel<<<dim3((unsigned)n_chunks, (unsigned)(batch * n_nodes)), kAcceptThreads, 0, st>>>(
+      target_logits, vocab, n_chunks, part);
+  int32_t rc = launch_status();
+  if (rc != SPECVLM_OK) return rc;
+  accept_tree_finish_kernel<<<(unsigned)batch, 32 * n_nodes, 0, st>>>(part, n_chunks, node_tokens, parents, n_nodes,
+                                                                      accept_len, next_token, path,
+                                                                      target_argmax_or_null);
   return launch_status();
 }

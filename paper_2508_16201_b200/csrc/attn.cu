@@ -395,9 +395,10 @@ static size_t rows16_ws_bytes(const specvlm_kv_t* kv, int32_t batch, int rows) {
 
 // tcgen05 path (attn_tc.cu)
 size_t attn_tc_ws_bytes(const specvlm_kv_t* kv, int32_t batch, int rows);
+size_t attn_tc_tree_extra_bytes(int32_t batch, int32_t n_nodes);
 int32_t attn_tc_launch(const specvlm_kv_t* kv, const void* q, int32_t batch, int32_t n_q_heads, int32_t n_q,
                        float sm_scale, void* out, float* lse, void* ws, size_t ws_bytes, int32_t* d_status,
-                       cudaStream_t st);
+                       cudaStream_t st, const int32_t* tree_parents);
 
 template <int D>
 static int32_t launch_rows16(const CUtensorMap& tk, const CUtensorMap& tv, const AttnParams& p,
@@ -425,7 +426,7 @@ static int32_t attn_common(const specvlm_kv_t* kv, const void* q, int32_t batch,
   if (rows > 128) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (rows > kRows16Max)
-    return attn_tc_launch(kv, q, batch, n_q_heads, n_q, sm_scale, out, lse, ws, ws_bytes, d_status, st);
+    return attn_tc_launch(kv, q, batch, n_q_heads, n_q, sm_scale, out, lse, ws, ws_bytes, d_status, st, nullptr);
 
   const int64_t lb64 = (int64_t)kv->n_layers * batch;
   if (lb64 > 65535 || kv->n_kv_heads > 65535) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
@@ -506,4 +507,28 @@ extern "C" int32_t specvlm_verify_attn(const specvlm_kv_t* kv, const void* q, in
   if (gamma < 0 || gamma > 8) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   return attn_common(kv, q, batch, n_q_heads, gamma + 1, sm_scale, out, lse_or_null, ws, ws_bytes,
                      d_status, stream);
+}
+
+extern "C" size_t specvlm_verify_tree_workspace_bytes(const specvlm_kv_t* kv, int32_t batch, int32_t n_q_heads,
+                                                      int32_t n_nodes) {
+  if (!kv || batch < 1 || batch > kSchedMaxBatch || n_q_heads < 1 || n_nodes < 1 || n_nodes > 32 ||
+      kv->n_kv_heads < 1 || n_q_heads % kv->n_kv_heads != 0 || kv->n_layers < 1 || kv->max_seq_len < 1)
+    return 0;
+  const int rows = (n_q_heads / kv->n_kv_heads) * n_nodes;
+  if (rows > 128) return 0;
+  return attn_tc_ws_bytes(kv, batch, rows) + attn_tc_tree_extra_bytes(batch, n_nodes);
+}
+
+extern "C" int32_t specvlm_verify_tree_attn(const specvlm_kv_t* kv, const void* q, const int32_t* parents,
+                                            int32_t batch, int32_t n_q_heads, int32_t n_nodes, float sm_scale,
+                                            void* out, float* lse_or_null, void* ws, size_t ws_bytes,
+                                            int32_t* d_status, void* stream) {
+  int32_t rc = validate_kv(kv, batch, true);
+  if (rc != SPECVLM_OK) return rc;
+  if (!q || !out || !parents || n_q_heads < 1 || n_nodes < 1 || !(sm_scale > 0.f)) return SPECVLM_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(out) || n_q_heads % kv->n_kv_heads != 0) return SPECVLM_ERR_INVALID_ARG;
+  const int group = n_q_heads / kv->n_kv_heads;
+  if (group > 16 || n_nodes > 32 || group * n_nodes > 128) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  return attn_tc_launch(kv, q, batch, n_q_heads, n_nodes, sm_scale, out, lse_or_null, ws, ws_bytes, d_status,
+                        static_cast<cudaStream_t>(stream), parents);
 }

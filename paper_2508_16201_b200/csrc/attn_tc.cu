@@ -41,6 +41,7 @@ struct AttnTcParams {
   const int32_t* block_table; // [B][max_blocks] or null
   const int32_t* seq_lens;    // [B]
   int32_t* d_status;
+  const uint32_t* anc;        // [B][n_q] ancestor masks of a draft tree, or null: the window is a chain
   int32_t batch, n_layers, n_q, n_q_heads, n_kv_heads, group, rows;
   int32_t max_blocks, block_tokens, max_seq_len;
   float scale_log2;           // sm_scale * log2(e)
@@ -487,14 +488,21 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       const int seg_idx = c.seg_idx;
       const int kv_len = clamp_len(p.seq_lens[sg.b], p.max_seq_len);
       const int n_sub_seq = (kv_len + kTileTokens - 1) / kTileTokens;
-      int lim[NH][2];
+      // Visibility of key `tok` for a row of query token t: every key before the window of the n_q
+      // new tokens, and inside the window the positions whose bit is set in the row's mask -- bits
+      // 0..t for a chain, the token's ancestors and itself for a tree.  Rows no item uses see nothing.
+      const int win0 = kv_len - p.n_q;
+      int old_r[NH][2];
+      uint32_t vis[NH][2];
       float m_used[NH][2], l_sum[NH][2];
 #pragma unroll
       for (int h = 0; h < NH; ++h)
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
           const int r = row0(h) + lr + 8 * e;
-          lim[h][e] = r < p.rows ? kv_len - p.n_q + r / p.group + 1 : 0;
+          const int t = r / p.group;
+          old_r[h][e] = r < p.rows ? win0 : 0;
+          vis[h][e] = r < p.rows ? (p.anc ? __ldg(p.anc + (size_t)sg.b * p.n_q + t) : (2u << t) - 1u) : 0u;
           m_used[h][e] = -INFINITY;
           l_sum[h][e] = 0.f;
         }
@@ -502,7 +510,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       for (int j = (i0 + grp) & 1; j < sg.n_tiles; j += 2) {
         const int i = i0 + j;
         const int tile_tok0 = (sg.tile0 + j) * kBigTokens;
-        const bool need_mask = tile_tok0 + kBigTokens > kv_len - p.n_q + 1;
+        const bool need_mask = tile_tok0 + kBigTokens > win0;
         SM_WAIT(bar_s_full + 8 * grp, (i >> 1) & 1);
         tc_fence_after_sync();
         if (nh == 0) {
@@ -531,9 +539,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 #pragma unroll
             for (int k = 0; k < 32; ++k) {
               const int tok = tile_tok0 + (k >> 2) * 8 + lc + (k & 1);
-              const int lm = lim[h][(k >> 1) & 1];
-              const float x0 = tok < lm ? __uint_as_float(v0[k]) * p.scale_log2 : -INFINITY;
-              const float x1 = tok + kTileTokens < lm ? __uint_as_float(v1[k]) * p.scale_log2 : -INFINITY;
+              const int e = (k >> 1) & 1;
+              const int w0 = tok - old_r[h][e], w1 = w0 + kTileTokens;      // position inside the window, if >= 0
+              const bool s0 = w0 < 0 || (w0 < 32 && ((vis[h][e] >> w0) & 1u));
+              const bool s1 = w1 < 0 || (w1 < 32 && ((vis[h][e] >> w1) & 1u));
+              const float x0 = s0 ? __uint_as_float(v0[k]) * p.scale_log2 : -INFINITY;
+              const float x1 = s1 ? __uint_as_float(v1[k]) * p.scale_log2 : -INFINITY;
               v0[k] = __float_as_uint(x0);
               v1[k] = __float_as_uint(x1);
               mx[k & 3] = fmaxf(mx[k & 3], fmaxf(x0, x1));
@@ -820,16 +831,47 @@ static int32_t launch_tc(const CUtensorMap& tk, const CUtensorMap& tv, const CUt
   return launch_status();
 }
 
+// Ancestor masks of a draft tree: bit w of anc[b][t] says that node t attends window position w
+// (itself and the nodes on its path to a root).  parents[b][t] < t, -1 for a root.
+__global__ void tree_ancestors_kernel(const int32_t* __restrict__ parents, int n, int n_nodes,
+                                      uint32_t* __restrict__ anc, int32_t* d_status) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const int t = i % n_nodes;
+  const int32_t* par = parents + (i - t);
+  uint32_t a = 1u << t;
+  int cur = t;
+  for (int step = 0; step < n_nodes; ++step) {
+    const int pp = par[cur];
+    if (pp < 0) break;
+    if (pp >= cur) {                      // not a tree in topological order: the node sees itself only
+      if (d_status) *d_status = SPECVLM_ERR_INVALID_ARG;
+      a = 1u << t;
+      break;
+    }
+    a |= 1u << pp;
+    cur = pp;
+  }
+  anc[i] = a;
+}
+
+size_t attn_tc_tree_extra_bytes(int32_t batch, int32_t n_nodes) {
+  return round_up((size_t)batch * n_nodes * sizeof(uint32_t), 256);
+}
+
 int32_t attn_tc_launch(const specvlm_kv_t* kv, const void* q, int32_t batch, int32_t n_q_heads, int32_t n_q,
                        float sm_scale, void* out, float* lse, void* ws, size_t ws_bytes, int32_t* d_status,
-                       cudaStream_t st) {
+                       cudaStream_t st, const int32_t* tree_parents) {
   const int group = n_q_heads / kv->n_kv_heads;
   const int rows = group * n_q;
   if (rows > 128 || batch > kSchedMaxBatch) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   const int64_t items = (int64_t)kv->n_layers * batch * kv->n_kv_heads;
   if (items > 0x3fffffff) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) return SPECVLM_ERR_INVALID_ARG;
-  if (ws_bytes < attn_tc_ws_bytes(kv, batch, rows)) return SPECVLM_ERR_WORKSPACE_TOO_SMALL;
+  const size_t base_bytes = attn_tc_ws_bytes(kv, batch, rows);
+  if (ws_bytes < base_bytes + (tree_parents ? attn_tc_tree_extra_bytes(batch, n_q) : 0))
+    return SPECVLM_ERR_WORKSPACE_TOO_SMALL;
+  if (tree_parents && n_q > 32) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   const int grid = tc_grid(kv, batch);
 
   CUtensorMap tk, tv, tq;
@@ -863,6 +905,15 @@ int32_t attn_tc_launch(const specvlm_kv_t* kv, const void* q, int32_t batch, int
   p.block_tokens = kv->block_tokens;
   p.max_seq_len = kv->max_seq_len;
   p.scale_log2 = sm_scale * kLog2e;
+  p.anc = nullptr;
+  if (tree_parents) {
+    uint32_t* anc = reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(ws) + base_bytes);
+    const int n = batch * n_q;
+    tree_ancestors_kernel<<<(unsigned)((n + 127) / 128), 128, 0, st>>>(tree_parents, n, n_q, anc, d_status);
+    rc = launch_status();
+    if (rc != SPECVLM_OK) return rc;
+    p.anc = anc;
+  }
 
   if (cudaMemsetAsync(p.ws_cnt, 0, (size_t)items * sizeof(int32_t), st) != cudaSuccess) return SPECVLM_ERR_CUDA;
   if (kv->head_dim == 128)

@@ -67,6 +67,71 @@ __global__ void seq_len_update_kernel(int32_t* seq_lens, const int32_t* accept_l
   seq_lens[b] = n;
 }
 
+struct CompactParams {
+  uint4* k;
+  uint4* v;
+  const int32_t* table;
+  const int32_t* seq_lens;   // lengths including the n_nodes window
+  const int32_t* path;       // [B][n_nodes]: accepted nodes in order, then -1
+  const int32_t* accept_len; // [B]
+  int64_t s_layer, s_block, s_head, s_token;
+  int32_t block_tokens, max_blocks, n_nodes, n_kv_heads, chunks_per_row;
+};
+
+// One CTA per (layer, KV head, sequence): the accepted nodes' rows move up behind the root.  A
+// destination row can be a later move's source, so every row is read before any is written.
+__global__ void __launch_bounds__(256) compact_tree_kernel(const __grid_constant__ CompactParams p) {
+  const int b = blockIdx.y;
+  const int layer = blockIdx.x / p.n_kv_heads, head = blockIdx.x - layer * p.n_kv_heads;
+  const int n = min(max(p.accept_len[b], 0), p.n_nodes - 1);
+  const int old = p.seq_lens[b] - p.n_nodes;
+  const int cpr = p.chunks_per_row;
+  auto addr = [&](int pos, int chunk) -> int64_t {
+    int blk = b, off = pos;
+    if (p.table) {
+      blk = __ldg(p.table + (size_t)b * p.max_blocks + pos / p.block_tokens);
+      off = pos % p.block_tokens;
+    }
+    return layer * p.s_layer + blk * p.s_block + head * p.s_head + off * p.s_token + chunk;
+  };
+  constexpr int kMaxPerThread = 2;          // 31 rows x 16 chunks = 496 chunks <= 2 x 256
+  uint4 kk[kMaxPerThread], vv[kMaxPerThread];
+  if (old < 0) return;
+#pragma unroll
+  for (int u = 0; u < kMaxPerThread; ++u) {
+    const int idx = u * 256 + threadIdx.x;
+    if (idx < n * cpr) {
+      const int node = p.path[(size_t)b * p.n_nodes + idx / cpr];
+      const int64_t a = addr(old + node, idx % cpr);
+      kk[u] = p.k[a];
+      vv[u] = p.v[a];
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int u = 0; u < kMaxPerThread; ++u) {
+    const int idx = u * 256 + threadIdx.x;
+    if (idx < n * cpr) {
+      const int64_t a = addr(old + 1 + idx / cpr, idx % cpr);
+      p.k[a] = kk[u];
+      p.v[a] = vv[u];
+    }
+  }
+}
+
+// seq_lens[b] = seq_lens[b] - n_nodes + 1 + accept_len[b]
+__global__ void tree_len_kernel(int32_t* seq_lens, const int32_t* accept_len, int batch, int n_nodes,
+                                int32_t* d_status) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= batch) return;
+  const int a = accept_len[b], n = seq_lens[b];
+  if (a < 0 || a > n_nodes - 1 || n < n_nodes) {
+    if (d_status) *d_status = SPECVLM_ERR_INVALID_ARG;
+    return;
+  }
+  seq_lens[b] = n - n_nodes + 1 + a;
+}
+
 }  // namespace specvlm
 
 using namespace specvlm;
@@ -111,5 +176,35 @@ extern "C" int32_t specvlm_rollback_kv(int32_t* seq_lens_inout, const int32_t* a
   if (!seq_lens_inout || !accept_len || batch < 1 || gamma < 0) return SPECVLM_ERR_INVALID_ARG;
   seq_len_update_kernel<<<(unsigned)((batch + 127) / 128), 128, 0, static_cast<cudaStream_t>(stream)>>>(
       seq_lens_inout, accept_len, batch, 0, gamma, 0, d_status);
+  return launch_status();
+}
+
+extern "C" int32_t specvlm_compact_tree_kv(const specvlm_kv_t* kv, const int32_t* path, const int32_t* accept_len,
+                                           int32_t batch, int32_t n_nodes, int32_t* seq_lens_inout,
+                                           int32_t* d_status, void* stream) {
+  if (!kv || !path || !accept_len || !seq_lens_inout || n_nodes < 1) return SPECVLM_ERR_INVALID_ARG;
+  if (n_nodes > 32) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  specvlm_kv_t c = *kv;
+  c.seq_lens = seq_lens_inout;
+  int32_t rc = validate_kv(&c, batch, true);
+  if (rc != SPECVLM_OK) return rc;
+  if ((int64_t)c.n_layers * c.n_kv_heads > 0x7fffffff || batch > 65535) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  CompactParams p;
+  p.k = static_cast<uint4*>(c.k);
+  p.v = static_cast<uint4*>(c.v);
+  p.table = c.block_table;
+  p.seq_lens = seq_lens_inout;
+  p.path = path;
+  p.accept_len = accept_len;
+  p.s_layer = c.stride_layer / 8; p.s_block = c.stride_block / 8; p.s_head = c.stride_head / 8;
+  p.s_token = c.stride_token / 8;
+  p.block_tokens = c.block_tokens; p.max_blocks = c.max_blocks; p.n_nodes = n_nodes;
+  p.n_kv_heads = c.n_kv_heads; p.chunks_per_row = c.head_dim / 8;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  compact_tree_kernel<<<dim3((unsigned)(c.n_layers * c.n_kv_heads), (unsigned)batch), 256, 0, st>>>(p);
+  rc = launch_status();
+  if (rc != SPECVLM_OK) return rc;
+  tree_len_kernel<<<(unsigned)((batch + 127) / 128), 128, 0, st>>>(seq_lens_inout, accept_len, batch, n_nodes,
+                                                                   d_status);
   return launch_status();
 }

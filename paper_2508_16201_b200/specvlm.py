@@ -52,6 +52,8 @@ EXPORTS = [
     "specvlm_attn_workspace_bytes", "specvlm_draft_decode_attn", "specvlm_verify_attn",
     "specvlm_accept_workspace_bytes", "specvlm_accept", "specvlm_accept_noalloc",
     "specvlm_append_kv", "specvlm_rollback_kv",
+    "specvlm_verify_tree_workspace_bytes", "specvlm_verify_tree_attn", "specvlm_accept_tree",
+    "specvlm_compact_tree_kv",
 ]
 
 
@@ -83,6 +85,16 @@ def lib():
         L.specvlm_select_top_p.restype = c_int32
         L.specvlm_select_top_p.argtypes = [c_void_p, i32p, i32p, c_int32, i32p, i32p, i32p, c_int32, c_void_p,
                                            c_void_p, c_void_p, c_void_p]
+        L.specvlm_verify_tree_workspace_bytes.restype = c_size_t
+        L.specvlm_verify_tree_workspace_bytes.argtypes = [kvp, c_int32, c_int32, c_int32]
+        L.specvlm_verify_tree_attn.restype = c_int32
+        L.specvlm_verify_tree_attn.argtypes = [kvp, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_float, c_void_p,
+                                               c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]
+        L.specvlm_accept_tree.restype = c_int32
+        L.specvlm_accept_tree.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p,
+                                          c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+        L.specvlm_compact_tree_kv.restype = c_int32
+        L.specvlm_compact_tree_kv.argtypes = [kvp, c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p]
         L.specvlm_append_kv.restype = c_int32
         L.specvlm_append_kv.argtypes = [kvp, c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p]
         L.specvlm_rollback_kv.restype = c_int32
@@ -321,6 +333,51 @@ def rollback_kv(seq_lens: torch.Tensor, accept_len: torch.Tensor, gamma: int,
     rc = lib().specvlm_rollback_kv(_ptr(seq_lens), _ptr(accept_len), seq_lens.numel(), int(gamma), _ptr(d_status),
                                    _stream())
     _check(rc, "specvlm_rollback_kv")
+
+
+# ---------------------------------------------------------------------------------- tree drafting
+def verify_tree_attn(kv: KvCache, q: torch.Tensor, parents: torch.Tensor, sm_scale: float,
+                     out: torch.Tensor | None = None, lse: torch.Tensor | None = None,
+                     ws: torch.Tensor | None = None, d_status: torch.Tensor | None = None) -> torch.Tensor:
+    """q: bf16 [n_layers][batch][n_nodes][n_q_heads][head_dim]; parents: int32 [batch][n_nodes]."""
+    L, B, N, Hq, D = q.shape
+    assert q.dtype == torch.bfloat16 and q.is_contiguous()
+    assert parents.dtype == torch.int32 and parents.is_contiguous() and tuple(parents.shape) == (B, N)
+    if out is None:
+        out = torch.empty_like(q)
+    if ws is None:
+        ws = _ws(int(lib().specvlm_verify_tree_workspace_bytes(byref(kv.struct), B, Hq, N)), q.device)
+    rc = lib().specvlm_verify_tree_attn(byref(kv.struct), _ptr(q), _ptr(parents), B, Hq, N, float(sm_scale),
+                                        _ptr(out), _ptr(lse), _ptr(ws), ws.numel(), _ptr(d_status), _stream())
+    _check(rc, "specvlm_verify_tree_attn")
+    return out
+
+
+def accept_tree(target_logits: torch.Tensor, node_tokens: torch.Tensor, parents: torch.Tensor,
+                want_argmax: bool = False):
+    """Returns (accept_len [B], next_token [B], path [B][n_nodes], argmax [B][n_nodes] or None)."""
+    B, N, V = target_logits.shape
+    assert target_logits.dtype == torch.float32 and target_logits.is_contiguous()
+    assert node_tokens.dtype == torch.int32 and parents.dtype == torch.int32
+    dev = target_logits.device
+    n = torch.empty(B, dtype=torch.int32, device=dev)
+    nxt = torch.empty(B, dtype=torch.int32, device=dev)
+    path = torch.empty((B, N), dtype=torch.int32, device=dev)
+    g = torch.empty((B, N), dtype=torch.int32, device=dev) if want_argmax else None
+    ws = _ws(accept_workspace_bytes(B, N - 1, V), dev)
+    rc = lib().specvlm_accept_tree(_ptr(target_logits), _ptr(node_tokens), _ptr(parents), B, N, V, _ptr(n), _ptr(nxt),
+                                   _ptr(path), _ptr(g), _ptr(ws), ws.numel(), _stream())
+    _check(rc, "specvlm_accept_tree")
+    return n, nxt, path, g
+
+
+def compact_tree_kv(kv: KvCache, path: torch.Tensor, accept_len: torch.Tensor,
+                    d_status: torch.Tensor | None = None) -> None:
+    """Moves the accepted nodes' rows behind the root and shortens kv.seq_lens accordingly."""
+    B, N = path.shape
+    rc = lib().specvlm_compact_tree_kv(byref(kv.struct), _ptr(path), _ptr(accept_len), B, N, _ptr(kv.seq_lens),
+                                       _ptr(d_status), _stream())
+    _check(rc, "specvlm_compact_tree_kv")
 
 
 # ---------------------------------------------------------------------------------- accept

@@ -344,3 +344,56 @@ def test_append_and_rollback():
     assert oracle.rollback_len(20, 4, 2) == 18
     # appending gamma + 1 tokens then rolling back with n accepted leaves old + n + 1 tokens
     assert oracle.rollback_len(13 + 6, 5, 3) == 13 + 3 + 1
+
+
+# ----------------------------------------------------------------------------- tree drafting
+def test_tree_attention_reduces_to_chain_and_is_path_local():
+    rng = np.random.default_rng(12)
+    hq, hkv, d, old = 4, 2, 16, 9
+    bf = lambda shape: (rng.standard_normal(shape).astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
+    # a chain is the tree parents[t] = t - 1: must equal the chain attention (C routine) exactly
+    n = 5
+    q, k, v = bf((n, hq, d)), bf((hkv, old + n, d)), bf((hkv, old + n, d))
+    o_tree, l_tree = oracle.attention_tree(q, k, v, old + n, [-1, 0, 1, 2, 3], 0.25)
+    o_chain, l_chain = oracle.attention(q, k, v, old + n, 0.25)
+    np.testing.assert_allclose(o_tree, o_chain, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(l_tree, l_chain, rtol=0, atol=1e-12)
+    # a node's output depends on its own root path only: node 3 (path 0-1-3) must equal the last
+    # row of the chain attention over the cache with rows (0, 1, 3) of the window kept
+    parents = [-1, 0, 0, 1, 2]
+    assert oracle.tree_ancestors(parents) == [[0], [0, 1], [0, 2], [0, 1, 3], [0, 2, 4]]
+    o_tree, _ = oracle.attention_tree(q, k, v, old + n, parents, 0.25)
+    keep = list(range(old)) + [old + 0, old + 1, old + 3]
+    o_path, _ = oracle.attention(q[[0, 1, 3]], k[:, keep], v[:, keep], len(keep), 0.25)
+    np.testing.assert_allclose(o_tree[3], o_path[2], rtol=0, atol=1e-12)
+    np.testing.assert_allclose(o_tree[1], o_path[1], rtol=0, atol=1e-12)
+
+
+def test_tree_acceptance_and_compaction():
+    # logits rows put all mass on one token: g = [7, 3, 9, 5, 1]
+    g = [7, 3, 9, 5, 1]
+    logits = np.full((5, 12), -1.0, dtype=np.float32)
+    for t, a in enumerate(g):
+        logits[t, a] = 2.0
+    parents = [-1, 0, 0, 1, 1]
+    # children of the root carry tokens 4 and 7 -> node 2 accepted; node 2 has no children
+    assert oracle.accept_tree(logits, [0, 4, 7, 5, 3], parents) == (1, 9, [2])
+    # root -> node 1 (token 7) -> node 4 (token 3 = g[1]) ; next token g[4]
+    assert oracle.accept_tree(logits, [0, 7, 8, 5, 3], parents) == (2, 1, [1, 4])
+    # nothing matches
+    assert oracle.accept_tree(logits, [0, 1, 2, 3, 4], parents) == (0, 7, [])
+    # a chain tree gives the chain rule
+    rng = np.random.default_rng(13)
+    for _ in range(20):
+        lg = rng.standard_normal((5, 30)).astype(np.float32)
+        am = lg.argmax(1)
+        drafts = np.where(rng.random(4) < 0.6, am[:4], rng.integers(0, 30, 4))
+        n, nxt, _ = oracle.accept(lg, drafts)
+        tn, tnxt, path = oracle.accept_tree(lg, [0] + drafts.tolist(), [-1, 0, 1, 2, 3])
+        assert (tn, tnxt) == (n, nxt) and path == list(range(1, n + 1))
+    # compaction: rows old+path[i] move to old+1+i
+    cache = np.arange(2 * 12 * 3, dtype=np.uint16).reshape(2, 12, 3)
+    out, n = oracle.compact_tree_kv(cache, 12, 5, [2, 4])
+    assert n == 7 + 1 + 2
+    assert np.array_equal(out[:, :8], cache[:, :8]) and np.array_equal(out[:, 8], cache[:, 9])
+    assert np.array_equal(out[:, 9], cache[:, 11])
