@@ -155,6 +155,31 @@ int32_t specvlm_select_top_p(const float* scores, const int32_t* video_cu, const
                              int32_t* kept_idx, int32_t* k_stage1_out_or_null, int32_t* d_status,
                              void* stream);
 
+/*
+ * Attention-agnostic selectors the paper compares its method with (random token pruning in the
+ * sensitivity study of Section 3.2; a window over the front, middle or end of the video tokens
+ * and full-frame dropping at regular temporal intervals in the ablations).  Uniform-only and
+ * attention-only pruning are specvlm_select with k_stage1 = 0 and k_stage1 = k_total.
+ *   WINDOW_*  the k_total consecutive tokens at the front / centred ((n_video - k_total) / 2) / end
+ *   FRAMES    floor(k_total / tokens_per_frame) whole frames, the i-th of n being frame floor(i F / n)
+ *   RANDOM    the k_total tokens with the largest keys, the key of token j of sequence b being the top
+ *             24 bits of the first word of Philox-4x32-10 at counter (j, b, 0, 0) under the 64-bit
+ *             seed; equal keys go to the lower index
+ *   kept_idx  device int32 out, ascending, sequence b at kept_cu[b]
+ *   kept_n_out_or_null  device int32 [batch] out: indices written (k_total, less for FRAMES)
+ * Arguments as in specvlm_select; n_video <= 57344 per sequence for RANDOM.
+ */
+typedef enum specvlm_selector {
+  SPECVLM_SEL_WINDOW_FRONT = 0,
+  SPECVLM_SEL_WINDOW_MIDDLE = 1,
+  SPECVLM_SEL_WINDOW_END = 2,
+  SPECVLM_SEL_FRAMES = 3,
+  SPECVLM_SEL_RANDOM = 4
+} specvlm_selector;
+int32_t specvlm_select_baseline(int32_t mode, uint64_t seed, const int32_t* n_frames,
+                                int32_t tokens_per_frame, const int32_t* k_total, const int32_t* kept_cu,
+                                int32_t batch, int32_t* kept_idx, int32_t* kept_n_out_or_null, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * Step 3 -- pruned draft context (end of Section 4.2: the draft sees V_R u V_U and the language
  * prompt, its cache reduced to 1-r of the original).

@@ -411,3 +411,54 @@ def compact_tree_kv(cache: np.ndarray, seq_len: int, n_nodes: int, path) -> tupl
     for i, node in enumerate(path):
         out[..., old + 1 + i, :] = cache[..., old + node, :]
     return out, old + 1 + len(path)
+
+
+# --------------------------------------------------------------------------------------
+# Attention-agnostic selectors the paper compares against (random pruning in its sensitivity
+# study; a window over the front / middle / end of the video tokens and full-frame dropping at
+# regular temporal intervals in its ablations).  Uniform-only and attention-only are `select`
+# with k1 = 0 and k1 = k_total.
+# --------------------------------------------------------------------------------------
+SEL_WINDOW_FRONT, SEL_WINDOW_MIDDLE, SEL_WINDOW_END, SEL_FRAMES, SEL_RANDOM = 0, 1, 2, 3, 4
+
+
+def philox4x32_10(counter, key) -> list[int]:
+    """Philox-4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy
+    as 1, 2, 3", SC'11): the counter-based generator both sides implement for random pruning."""
+    m0, m1, w0, w1 = 0xD2511F53, 0xCD9E8D57, 0x9E3779B9, 0xBB67AE85
+    c, k = [int(x) & 0xFFFFFFFF for x in counter], [int(x) & 0xFFFFFFFF for x in key]
+    for _ in range(10):
+        p0, p1 = m0 * c[0], m1 * c[2]
+        c = [(p1 >> 32) ^ c[1] ^ k[0], p1 & 0xFFFFFFFF, (p0 >> 32) ^ c[3] ^ k[1], p0 & 0xFFFFFFFF]
+        k = [(k[0] + w0) & 0xFFFFFFFF, (k[1] + w1) & 0xFFFFFFFF]
+    return c
+
+
+def random_scores(n_video: int, seed: int, b: int = 0) -> np.ndarray:
+    """One fp32 key per video token: the top 24 bits of the first Philox word at counter
+    (token, sequence, 0, 0) under the 64-bit seed.  The largest keys are kept."""
+    key = [seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF]
+    return np.array([philox4x32_10([j, b, 0, 0], key)[0] >> 8 for j in range(n_video)], dtype=np.float32)
+
+
+def select_baseline(mode: int, n_frames: int, tokens_per_frame: int, k_total: int, seed: int = 0, b: int = 0
+                    ) -> np.ndarray:
+    """Kept video indices (ascending) of an attention-agnostic selector under the budget k_total.
+    Frame dropping keeps floor(k_total / T) whole frames, frame i of them being floor(i F / n)."""
+    n_v = n_frames * tokens_per_frame
+    assert 0 <= k_total <= n_v
+    if mode == SEL_WINDOW_FRONT:
+        kept = range(0, k_total)
+    elif mode == SEL_WINDOW_MIDDLE:
+        start = (n_v - k_total) // 2
+        kept = range(start, start + k_total)
+    elif mode == SEL_WINDOW_END:
+        kept = range(n_v - k_total, n_v)
+    elif mode == SEL_FRAMES:
+        nf = k_total // tokens_per_frame
+        kept = [((i * n_frames) // nf) * tokens_per_frame + t for i in range(nf) for t in range(tokens_per_frame)]
+    elif mode == SEL_RANDOM:
+        kept = stage1_topk(random_scores(n_v, seed, b), k_total)
+    else:
+        raise ValueError("unknown selector")
+    return np.asarray(list(kept), dtype=np.int32)

@@ -32,13 +32,32 @@ __device__ __forceinline__ unsigned long long key_mass(uint32_t key) {
 struct SelSeq {
   int32_t score_off, n_frames, k1, k_total, kept_off;
   int32_t lambda_pm;                   // >= 0: Top-P mode, k1 is computed; < 0: k1 as given
+  int32_t seq_index;                   // position in the batch (random selector's counter word)
 };
+
+// Philox-4x32, 10 rounds (Salmon et al., SC'11), first output word: the counter-based generator
+// of the random selector
+__device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t c0, uint32_t c1, uint32_t k0, uint32_t k1) {
+  uint32_t c2 = 0u, c3 = 0u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return c0;
+}
 struct SelParams {
   const float* scores;
   int32_t* kept_idx;
   int32_t* k1_out;                     // [batch] Stage-I counts or null
   int32_t tokens_per_frame;
   int32_t k1_out_base;                 // index of seq[0] in k1_out
+  int32_t random_keys;                 // 1: rank Philox keys instead of scores
+  uint32_t seed_lo, seed_hi;
   SelSeq seq[kSelMaxBatch];
 };
 
@@ -86,10 +105,18 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const __grid_con
   const int tid = threadIdx.x;
 
   // order-preserving map float -> uint32 (larger float <=> larger key)
-  const float* sc = p.scores + sq.score_off;
-  for (int j = tid; j < n_v; j += kSelThreads) {
-    const uint32_t u = __float_as_uint(sc[j]);
-    key[j] = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+  if (p.random_keys) {
+    // random selector: the key of token j is the top 24 bits of a Philox word, as an fp32 value
+    for (int j = tid; j < n_v; j += kSelThreads) {
+      const float r = (float)(philox4x32_10_word0((uint32_t)j, (uint32_t)sq.seq_index, p.seed_lo, p.seed_hi) >> 8);
+      key[j] = __float_as_uint(r) | 0x80000000u;
+    }
+  } else {
+    const float* sc = p.scores + sq.score_off;
+    for (int j = tid; j < n_v; j += kSelThreads) {
+      const uint32_t u = __float_as_uint(sc[j]);
+      key[j] = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    }
   }
 
   // ---- 0. Top-P: the Stage-I count from the score mass
@@ -250,11 +277,38 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const __grid_con
     if (key[j] != 0u) out[pos++] = j;
 }
 
+// window / frame selectors: closed-form index lists, one CTA per sequence
+struct RangeParams {
+  int32_t* kept_idx;
+  int32_t* kept_n_out;
+  int32_t mode, tokens_per_frame, batch0;
+  int32_t n_frames[kSelMaxBatch], k_total[kSelMaxBatch], kept_off[kSelMaxBatch];
+};
+
+__global__ void baseline_ranges_kernel(const __grid_constant__ RangeParams p) {
+  const int i = blockIdx.x;
+  const int F = p.n_frames[i], T = p.tokens_per_frame, K = p.k_total[i], n_v = F * T;
+  int32_t* out = p.kept_idx + p.kept_off[i];
+  int n = K;
+  if (p.mode == SPECVLM_SEL_FRAMES) {
+    const int nf = K / T;                       // whole frames that fit the budget
+    n = nf * T;
+    for (int j = threadIdx.x; j < n; j += blockDim.x) {
+      const int fi = j / T;
+      out[j] = (int)(((long long)fi * F) / nf) * T + (j - fi * T);
+    }
+  } else {
+    const int start = p.mode == SPECVLM_SEL_WINDOW_FRONT ? 0 : (p.mode == SPECVLM_SEL_WINDOW_END ? n_v - K : (n_v - K) / 2);
+    for (int j = threadIdx.x; j < n; j += blockDim.x) out[j] = start + j;
+  }
+  if (threadIdx.x == 0 && p.kept_n_out) p.kept_n_out[p.batch0 + i] = n;
+}
+
 static int32_t select_common(const float* scores, const int32_t* video_cu, const int32_t* n_frames,
                              int32_t tokens_per_frame, const int32_t* k_stage1, const int32_t* lambda_permille,
                              const int32_t* k_total, const int32_t* kept_cu, int32_t batch, int32_t* kept_idx,
-                             int32_t* k1_out, void* stream) {
-  if (!scores || !video_cu || !n_frames || (!k_stage1 && !lambda_permille) || !k_total || !kept_cu || !kept_idx ||
+                             int32_t* k1_out, void* stream, bool random_keys = false, uint64_t seed = 0) {
+  if ((!scores && !random_keys) || !video_cu || !n_frames || (!k_stage1 && !lambda_permille) || !k_total || !kept_cu || !kept_idx ||
       batch < 1 || tokens_per_frame < 1)
     return SPECVLM_ERR_INVALID_ARG;
   size_t max_smem = 0;
@@ -267,7 +321,7 @@ static int32_t select_common(const float* scores, const int32_t* video_cu, const
     } else if (k_stage1[b] < 0 || k_stage1[b] > k_total[b]) {
       return SPECVLM_ERR_INVALID_ARG;
     }
-    if (video_cu[b + 1] - video_cu[b] < n_v || kept_cu[b + 1] - kept_cu[b] < k_total[b])
+    if ((!random_keys && video_cu[b + 1] - video_cu[b] < n_v) || kept_cu[b + 1] - kept_cu[b] < k_total[b])
       return SPECVLM_ERR_INVALID_ARG;
     // keys, per-frame counts, histogram, scan scratch, flags, then the 64-bit mass bins (8-byte aligned)
     const size_t words = (size_t)n_v + n_frames[b] + 1 + 256 + 32 + 8;
@@ -284,13 +338,16 @@ static int32_t select_common(const float* scores, const int32_t* video_cu, const
   p.kept_idx = kept_idx;
   p.k1_out = k1_out;
   p.tokens_per_frame = tokens_per_frame;
+  p.random_keys = random_keys ? 1 : 0;
+  p.seed_lo = (uint32_t)(seed & 0xffffffffu);
+  p.seed_hi = (uint32_t)(seed >> 32);
   for (int b0 = 0; b0 < batch; b0 += kSelMaxBatch) {
     const int nb = batch - b0 < kSelMaxBatch ? batch - b0 : kSelMaxBatch;
     p.k1_out_base = b0;
     for (int i = 0; i < nb; ++i) {
       const int b = b0 + i;
       p.seq[i] = SelSeq{video_cu[b], n_frames[b], lambda_permille ? 0 : k_stage1[b], k_total[b], kept_cu[b],
-                        lambda_permille ? lambda_permille[b] : -1};
+                        lambda_permille ? lambda_permille[b] : -1, b};
     }
     select_kernel<<<(unsigned)nb, kSelThreads, max_smem, st>>>(p);
     const int32_t rc = launch_status();
@@ -322,4 +379,48 @@ extern "C" int32_t specvlm_select_top_p(const float* scores, const int32_t* vide
   if (!lambda_permille) return SPECVLM_ERR_INVALID_ARG;
   return select_common(scores, video_cu, n_frames, tokens_per_frame, nullptr, lambda_permille, k_total, kept_cu,
                        batch, kept_idx, k_stage1_out_or_null, stream);
+}
+
+extern "C" int32_t specvlm_select_baseline(int32_t mode, uint64_t seed, const int32_t* n_frames,
+                                           int32_t tokens_per_frame, const int32_t* k_total,
+                                           const int32_t* kept_cu, int32_t batch, int32_t* kept_idx,
+                                           int32_t* kept_n_out_or_null, void* stream) {
+  if (!n_frames || !k_total || !kept_cu || !kept_idx || batch < 1 || tokens_per_frame < 1)
+    return SPECVLM_ERR_INVALID_ARG;
+  if (mode < SPECVLM_SEL_WINDOW_FRONT || mode > SPECVLM_SEL_RANDOM) return SPECVLM_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (mode == SPECVLM_SEL_RANDOM) {
+    // the k_total largest Philox keys: the selection kernel with keys in place of scores and
+    // Stage I taking the whole budget
+    int32_t rc = select_common(nullptr, kept_cu /*unused*/, n_frames, tokens_per_frame, k_total, nullptr, k_total,
+                               kept_cu, batch, kept_idx, nullptr, stream, true, seed);
+    if (rc != SPECVLM_OK || !kept_n_out_or_null) return rc;
+    return cudaMemcpyAsync(kept_n_out_or_null, k_total, (size_t)batch * sizeof(int32_t), cudaMemcpyHostToDevice, st) ==
+                   cudaSuccess
+               ? SPECVLM_OK
+               : SPECVLM_ERR_CUDA;
+  }
+  RangeParams p;
+  p.kept_idx = kept_idx;
+  p.kept_n_out = kept_n_out_or_null;
+  p.mode = mode;
+  p.tokens_per_frame = tokens_per_frame;
+  for (int b0 = 0; b0 < batch; b0 += kSelMaxBatch) {
+    const int nb = batch - b0 < kSelMaxBatch ? batch - b0 : kSelMaxBatch;
+    p.batch0 = b0;
+    for (int i = 0; i < nb; ++i) {
+      const int b = b0 + i;
+      const int64_t n_v = (int64_t)n_frames[b] * tokens_per_frame;
+      if (n_frames[b] < 1 || n_v > 0x7fffffff || k_total[b] < 0 || k_total[b] > n_v ||
+          kept_cu[b + 1] - kept_cu[b] < k_total[b])
+        return SPECVLM_ERR_INVALID_ARG;
+      p.n_frames[i] = n_frames[b];
+      p.k_total[i] = k_total[b];
+      p.kept_off[i] = kept_cu[b];
+    }
+    baseline_ranges_kernel<<<(unsigned)nb, 256, 0, st>>>(p);
+    const int32_t rc = launch_status();
+    if (rc != SPECVLM_OK) return rc;
+  }
+  return SPECVLM_OK;
 }

@@ -48,7 +48,7 @@ _lib = None
 EXPORTS = [
     "specvlm_version", "specvlm_status_string",
     "specvlm_stage1_scores_workspace_bytes", "specvlm_stage1_row_lse", "specvlm_stage1_scores",
-    "specvlm_select", "specvlm_select_top_p", "specvlm_gather_kv",
+    "specvlm_select", "specvlm_select_top_p", "specvlm_select_baseline", "specvlm_gather_kv",
     "specvlm_attn_workspace_bytes", "specvlm_draft_decode_attn", "specvlm_verify_attn",
     "specvlm_accept_workspace_bytes", "specvlm_accept", "specvlm_accept_noalloc",
     "specvlm_append_kv", "specvlm_rollback_kv",
@@ -82,6 +82,9 @@ def lib():
         L.specvlm_select.restype = c_int32
         L.specvlm_select.argtypes = [c_void_p, i32p, i32p, c_int32, i32p, i32p, i32p, c_int32, c_void_p,
                                      c_void_p, c_void_p]
+        L.specvlm_select_baseline.restype = c_int32
+        L.specvlm_select_baseline.argtypes = [c_int32, ctypes.c_uint64, i32p, c_int32, i32p, i32p, c_int32, c_void_p,
+                                              c_void_p, c_void_p]
         L.specvlm_select_top_p.restype = c_int32
         L.specvlm_select_top_p.argtypes = [c_void_p, i32p, i32p, c_int32, i32p, i32p, i32p, c_int32, c_void_p,
                                            c_void_p, c_void_p, c_void_p]
@@ -304,6 +307,21 @@ def select_top_p(scores: torch.Tensor, video_cu, n_frames, tokens_per_frame: int
                                     _ptr(k_stage1_out), _ptr(d_status), _stream())
     _check(rc, "specvlm_select_top_p")
     return kept_idx, k_stage1_out
+
+
+SEL_WINDOW_FRONT, SEL_WINDOW_MIDDLE, SEL_WINDOW_END, SEL_FRAMES, SEL_RANDOM = 0, 1, 2, 3, 4
+
+
+def select_baseline(mode: int, n_frames, tokens_per_frame: int, k_total, kept_cu, seed: int = 0,
+                    device="cuda"):
+    """Returns (kept_idx, kept_n): the index lists of an attention-agnostic selector."""
+    batch = len(n_frames)
+    kept_idx = torch.empty(max(int(kept_cu[-1]), 1), dtype=torch.int32, device=device)
+    kept_n = torch.empty(batch, dtype=torch.int32, device=device)
+    rc = lib().specvlm_select_baseline(int(mode), int(seed), _i32(n_frames), int(tokens_per_frame), _i32(k_total),
+                                       _i32(kept_cu), batch, _ptr(kept_idx), _ptr(kept_n), _stream())
+    _check(rc, "specvlm_select_baseline")
+    return kept_idx, kept_n
 
 
 # ---------------------------------------------------------------------------------- gather

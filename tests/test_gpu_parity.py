@@ -283,6 +283,22 @@ def test_select_top_p_on_rated_scores_cfg1():
         assert int(k1[0]) == ref_k1 and np.array_equal(kept.cpu().numpy(), ref)
 
 
+@pytest.mark.parametrize("mode", [0, 1, 2, 3, 4])
+def test_select_baselines_bit_exact(mode):
+    """Window / frame-dropping / random (Philox) selectors equal the oracle's index lists."""
+    frames, T = [32, 5, 256, 1], 196
+    kts = [627, 400, 2508, 196]
+    kept_cu = [0]
+    for k in kts:
+        kept_cu.append(kept_cu[-1] + k)
+    kept, kept_n = specvlm.select_baseline(mode, frames, T, kts, kept_cu, seed=0x1234567890ABCDEF)
+    kept, kept_n = kept.cpu().numpy(), kept_n.cpu().numpy()
+    for b, F in enumerate(frames):
+        ref = oracle.select_baseline(mode, F, T, kts[b], seed=0x1234567890ABCDEF, b=b)
+        assert int(kept_n[b]) == len(ref), f"sequence {b}"
+        assert np.array_equal(kept[kept_cu[b]:kept_cu[b] + len(ref)], ref), f"sequence {b}"
+
+
 # ------------------------------------------------------------------------------- gather
 @pytest.mark.parametrize("src_paged,dst_paged", [(False, False), (True, True), (True, False)])
 def test_gather_bit_exact(src_paged, dst_paged):

@@ -397,3 +397,24 @@ def test_tree_acceptance_and_compaction():
     assert n == 7 + 1 + 2
     assert np.array_equal(out[:, :8], cache[:, :8]) and np.array_equal(out[:, 8], cache[:, 9])
     assert np.array_equal(out[:, 9], cache[:, 11])
+
+
+# ----------------------------------------------------------------------------- baseline selectors
+def test_philox_known_answers_and_baseline_selectors():
+    for line in open(os.path.join(GOLDEN, "philox4x32_10_kat.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        w = [int(x, 16) for x in line.split()]
+        assert oracle.philox4x32_10(w[0:4], w[4:6]) == w[6:10]
+    F, T, K = 5, 6, 13
+    assert oracle.select_baseline(oracle.SEL_WINDOW_FRONT, F, T, K).tolist() == list(range(13))
+    assert oracle.select_baseline(oracle.SEL_WINDOW_MIDDLE, F, T, K).tolist() == list(range(8, 21))
+    assert oracle.select_baseline(oracle.SEL_WINDOW_END, F, T, K).tolist() == list(range(17, 30))
+    # 13 // 6 = 2 whole frames at regular intervals: frames 0 and 2 of 5
+    assert oracle.select_baseline(oracle.SEL_FRAMES, F, T, K).tolist() == list(range(0, 6)) + list(range(12, 18))
+    r = oracle.select_baseline(oracle.SEL_RANDOM, 32, 196, 627, seed=7)
+    assert len(r) == 627 and len(set(r.tolist())) == 627 and (np.diff(r) > 0).all()
+    assert not np.array_equal(r, oracle.select_baseline(oracle.SEL_RANDOM, 32, 196, 627, seed=8))
+    # roughly uniform over the frames: every frame keeps between 5 and 40 of its 196 tokens (mean 19.6)
+    per_frame = np.bincount(r // 196, minlength=32)
+    assert per_frame.min() >= 5 and per_frame.max() <= 40
