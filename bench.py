@@ -17,6 +17,7 @@ cores, on a bounded sample of the same workload.
 from __future__ import annotations
 
 import argparse
+import ctypes
 import json
 import math
 import os
@@ -101,6 +102,10 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------------
+def ctypes_byref(cache):
+    return ctypes.byref(cache.struct)
+
+
 def max_over_ranks(times_ms, world, device):
     """Each rank runs an independent replica of the path (it does not shard: no data-path
     collective); the job's time for a step is the slowest rank's."""
@@ -322,6 +327,52 @@ def run_ours(args, rank, world):
     bytes_unpruned = 2 * (nv + nt) * w.d_kv_heads * D * 2 * w.d_layers
     extra["decode_unpruned_us"] = statistics.median(ts) * 1e3
     extra["decode_unpruned_kv_gbs"] = bytes_unpruned / (statistics.median(ts) * 1e-3) / 1e9
+
+    # the calls outside the step's fixed path (Top-P selection, tree drafting, cache maintenance),
+    # one after the other, median of 10 after 3 warm-ups; launches back to back without a host sync
+    # inside the timed pair would hide nothing here, each is a single short call
+    def timed(fn, reps=10):
+        out = []
+        for i in range(3 + reps):
+            a, b = E(), E()
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                out.append(a.elapsed_time(b))
+        return statistics.median(out) * 1e3
+
+    extra["select_top_p_us"] = timed(lambda: specvlm.select_top_p(path.scores, [0, nv], [w.n_frames[0]],
+                                                                  w.tokens_per_frame, [400], [path.kt], [0, path.kt]))
+    extra["select_random_us"] = timed(lambda: specvlm.select_baseline(specvlm.SEL_RANDOM, [w.n_frames[0]],
+                                                                      w.tokens_per_frame, [path.kt], [0, path.kt],
+                                                                      seed=1, device=device))
+    n_nodes = 128 // (w.t_q_heads // w.t_kv_heads)              # the widest tree one 128-row tile holds
+    n_tree = nv + nt + n_nodes
+    if n_tree <= inp["tcache"].max_seq_len + n_nodes:
+        tk = synth.randn_bf16((w.t_layers, 1, w.t_kv_heads, n_tree, D), device, 1, "treeK")
+        tcache = specvlm.KvCache(tk, tk, torch.tensor([n_tree], dtype=torch.int32, device=device), n_tree)
+        q_tree = synth.randn_bf16((w.t_layers, 1, n_nodes, w.t_q_heads, D), device, 1, "treeQ")
+        parents = torch.tensor([[-1] + [(t - 1) // 2 for t in range(1, n_nodes)]], dtype=torch.int32, device=device)
+        o_tree = torch.empty_like(q_tree)
+        ws_t = torch.empty(specvlm.lib().specvlm_verify_tree_workspace_bytes(ctypes_byref(tcache), 1, w.t_q_heads, n_nodes),
+                           dtype=torch.uint8, device=device)
+        us = timed(lambda: specvlm.verify_tree_attn(tcache, q_tree, parents, path.scale, out=o_tree, ws=ws_t), reps=5)
+        extra["verify_tree_%d_nodes_us" % n_nodes] = us
+        extra["verify_tree_kv_gbs"] = 2 * n_tree * w.t_kv_heads * D * 2 * w.t_layers / (us * 1e-6) / 1e9
+        lg = torch.randn((1, n_nodes, w.vocab), device=device)
+        toks = torch.zeros((1, n_nodes), dtype=torch.int32, device=device)
+        extra["accept_tree_us"] = timed(lambda: specvlm.accept_tree(lg, toks, parents))
+        del tk, tcache, q_tree, o_tree, lg
+    new_kv = synth.randn_bf16((w.t_layers, 1, gamma + 1, w.t_kv_heads, D), device, 2, "newKV")
+    lens_keep = inp["tcache"].seq_lens.clone()
+
+    def append_once():
+        inp["tcache"].seq_lens.fill_(nv + nt)                    # room for the gamma+1 new rows again
+        specvlm.append_kv(inp["tcache"], new_kv, new_kv)
+    extra["append_kv_us_incl_len_reset"] = timed(append_once)
+    inp["tcache"].seq_lens.copy_(lens_keep)
 
     # max over ranks
     total_ms, attn_ms = max_over_ranks([total_ms, attn_ms], world, device)

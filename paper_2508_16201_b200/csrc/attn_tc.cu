@@ -157,7 +157,10 @@ struct TcCfg {
   static_assert(SMALL + BIG <= kMaxSmem, "shared-memory plan does not fit");
 };
 
-template <int D, int M>
+// TREE: the window's visibility comes from per-token ancestor masks instead of the chain rule.
+// A template parameter, not a run-time branch: the chain kernel's code is untouched by the tree
+// variant (the softmax loop's speed proved sensitive to what is compiled around it).
+template <int D, int M, bool TREE>
 __global__ void __launch_bounds__(kTcThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ AttnTcParams p) {
@@ -491,9 +494,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       // Visibility of key `tok` for a row of query token t: every key before the window of the n_q
       // new tokens, and inside the window the positions whose bit is set in the row's mask -- bits
       // 0..t for a chain, the token's ancestors and itself for a tree.  Rows no item uses see nothing.
+      // (A used row always has its own bit set, so a zero mask also marks an unused row.)
+      // The chain keeps the equivalent limit form: key tok is visible to token t when tok < lim.
       const int win0 = kv_len - p.n_q;
-      int old_r[NH][2];
       uint32_t vis[NH][2];
+      int lim[NH][2];
       float m_used[NH][2], l_sum[NH][2];
 #pragma unroll
       for (int h = 0; h < NH; ++h)
@@ -501,8 +506,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         for (int e = 0; e < 2; ++e) {
           const int r = row0(h) + lr + 8 * e;
           const int t = r / p.group;
-          old_r[h][e] = r < p.rows ? win0 : 0;
-          vis[h][e] = r < p.rows ? (p.anc ? __ldg(p.anc + (size_t)sg.b * p.n_q + t) : (2u << t) - 1u) : 0u;
+          if constexpr (TREE) {
+            vis[h][e] = r < p.rows ? __ldg(p.anc + (size_t)sg.b * p.n_q + t) : 0u;
+          } else {
+            lim[h][e] = r < p.rows ? win0 + t + 1 : 0;
+          }
           m_used[h][e] = -INFINITY;
           l_sum[h][e] = 0.f;
         }
@@ -510,7 +518,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       for (int j = (i0 + grp) & 1; j < sg.n_tiles; j += 2) {
         const int i = i0 + j;
         const int tile_tok0 = (sg.tile0 + j) * kBigTokens;
-        const bool need_mask = tile_tok0 + kBigTokens > win0;
+        const bool need_mask = tile_tok0 + kBigTokens > win0 + (TREE ? 0 : 1);
         SM_WAIT(bar_s_full + 8 * grp, (i >> 1) & 1);
         tc_fence_after_sync();
         if (nh == 0) {
@@ -536,18 +544,42 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 
           float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
           if (need_mask) {
+            if constexpr (TREE) {
+              // 128 visibility bits of the tile per row: the keys before the window, then the row's
+              // window mask at the window's offset in the tile; shifted by this thread's first column
+              uint64_t mlo[2], mhi[2];
+              const int sh = win0 - tile_tok0;                       // tile column of window position 0
+  #pragma unroll
+              for (int e = 0; e < 2; ++e) {
+                unsigned __int128 full = 0;
+                if (vis[h][e]) {
+                  if (sh > 0) full = sh >= 128 ? ~(unsigned __int128)0 : (((unsigned __int128)1 << sh) - 1);
+                  const unsigned __int128 w = vis[h][e];
+                  full |= sh >= 0 ? (sh < 128 ? w << sh : (unsigned __int128)0) : (sh > -32 ? w >> (-sh) : (unsigned __int128)0);
+                }
+                mlo[e] = (uint64_t)full >> lc;
+                mhi[e] = (uint64_t)(full >> 64) >> lc;
+              }
+  #pragma unroll
+              for (int k = 0; k < 32; ++k) {
+                const int e = (k >> 1) & 1, bit = (k >> 2) * 8 + (k & 1);
+                const float x0 = ((mlo[e] >> bit) & 1ull) ? __uint_as_float(v0[k]) * p.scale_log2 : -INFINITY;
+                const float x1 = ((mhi[e] >> bit) & 1ull) ? __uint_as_float(v1[k]) * p.scale_log2 : -INFINITY;
+                v0[k] = __float_as_uint(x0);
+                v1[k] = __float_as_uint(x1);
+                mx[k & 3] = fmaxf(mx[k & 3], fmaxf(x0, x1));
+              }
+            } else {
 #pragma unroll
-            for (int k = 0; k < 32; ++k) {
-              const int tok = tile_tok0 + (k >> 2) * 8 + lc + (k & 1);
-              const int e = (k >> 1) & 1;
-              const int w0 = tok - old_r[h][e], w1 = w0 + kTileTokens;      // position inside the window, if >= 0
-              const bool s0 = w0 < 0 || (w0 < 32 && ((vis[h][e] >> w0) & 1u));
-              const bool s1 = w1 < 0 || (w1 < 32 && ((vis[h][e] >> w1) & 1u));
-              const float x0 = s0 ? __uint_as_float(v0[k]) * p.scale_log2 : -INFINITY;
-              const float x1 = s1 ? __uint_as_float(v1[k]) * p.scale_log2 : -INFINITY;
-              v0[k] = __float_as_uint(x0);
-              v1[k] = __float_as_uint(x1);
-              mx[k & 3] = fmaxf(mx[k & 3], fmaxf(x0, x1));
+              for (int k = 0; k < 32; ++k) {
+                const int tok = tile_tok0 + (k >> 2) * 8 + lc + (k & 1);
+                const int lm = lim[h][(k >> 1) & 1];
+                const float x0 = tok < lm ? __uint_as_float(v0[k]) * p.scale_log2 : -INFINITY;
+                const float x1 = tok + kTileTokens < lm ? __uint_as_float(v1[k]) * p.scale_log2 : -INFINITY;
+                v0[k] = __float_as_uint(x0);
+                v1[k] = __float_as_uint(x1);
+                mx[k & 3] = fmaxf(mx[k & 3], fmaxf(x0, x1));
+              }
             }
           } else {
 #pragma unroll
@@ -820,11 +852,11 @@ static int32_t encode_q_map(CUtensorMap* map, const void* q, int D, int group, i
   return r == CUDA_SUCCESS ? SPECVLM_OK : SPECVLM_ERR_CUDA;
 }
 
-template <int D, int M>
-static int32_t launch_tc(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tq, const AttnTcParams& p,
+template <int D, int M, bool TREE>
+static int32_t launch_tc_t(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tq, const AttnTcParams& p,
                          int grid, cudaStream_t st) {
   using C = TcCfg<D, M>;
-  auto kern = attn_tc_kernel<D, M>;
+  auto kern = attn_tc_kernel<D, M, TREE>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::TOTAL) != cudaSuccess)
     return SPECVLM_ERR_CUDA;
   kern<<<grid, kTcThreads, C::TOTAL, st>>>(tk, tv, tq, p);
@@ -857,6 +889,12 @@ __global__ void tree_ancestors_kernel(const int32_t* __restrict__ parents, int n
 
 size_t attn_tc_tree_extra_bytes(int32_t batch, int32_t n_nodes) {
   return round_up((size_t)batch * n_nodes * sizeof(uint32_t), 256);
+}
+
+template <int D, int M>
+static int32_t launch_tc(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tq, const AttnTcParams& p,
+                         int grid, cudaStream_t st) {
+  return p.anc ? launch_tc_t<D, M, true>(tk, tv, tq, p, grid, st) : launch_tc_t<D, M, false>(tk, tv, tq, p, grid, st);
 }
 
 int32_t attn_tc_launch(const specvlm_kv_t* kv, const void* q, int32_t batch, int32_t n_q_heads, int32_t n_q,
