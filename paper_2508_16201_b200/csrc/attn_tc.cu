@@ -528,80 +528,67 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 #pragma unroll
         for (int h = 0; h < NH; ++h) {
           if (h >= nh) break;
-          // S rows of this half: 128 columns = two loads of 64
-          uint32_t v0[32], v1[32];
+          // The half's 16 rows x 128 columns are read from TMEM twice, 64 columns at a time, by the
+          // same (rolled) code: once for the row maxima, once for the probabilities.  That halves
+          // the live registers and the code of the loop; a TMEM load costs far less than the spills.
           const uint32_t saddr = tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + C::COL_S + grp * kBigTokens;
-          tmem_ld_16x256b_x8(saddr, v0);
-          tmem_ld_16x256b_x8(saddr + 64, v1);
-          tmem_ld_wait();
-          if (h == nh - 1) {
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_s_empty + 8 * grp);
-          }
-          // the group's previous product has completed: P may be overwritten, O may be rescaled
-          if (h == 0 && i >= 2) SM_WAIT(bar_p_empty + 8 * grp, ((i >> 1) - 1) & 1);
-
-          float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-          if (need_mask) {
-            if constexpr (TREE) {
-              // 128 visibility bits of the tile per row: the keys before the window, then the row's
-              // window mask at the window's offset in the tile; shifted by this thread's first column
-              uint64_t mlo[2], mhi[2];
-              const int sh = win0 - tile_tok0;                       // tile column of window position 0
-  #pragma unroll
-              for (int e = 0; e < 2; ++e) {
+          // visibility of this thread's columns of chunk c, when the tile needs masking
+          auto chunk_mask = [&](int c, uint64_t (&mk)[2]) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              if constexpr (TREE) {
+                // 128 visibility bits of the tile: the keys before the window, then the row's window
+                // mask at the window's offset in the tile
+                const int sh = win0 - tile_tok0;                       // tile column of window position 0
                 unsigned __int128 full = 0;
                 if (vis[h][e]) {
                   if (sh > 0) full = sh >= 128 ? ~(unsigned __int128)0 : (((unsigned __int128)1 << sh) - 1);
                   const unsigned __int128 w = vis[h][e];
-                  full |= sh >= 0 ? (sh < 128 ? w << sh : (unsigned __int128)0) : (sh > -32 ? w >> (-sh) : (unsigned __int128)0);
+                  full |= sh >= 0 ? (sh < 128 ? w << sh : (unsigned __int128)0)
+                                  : (sh > -32 ? w >> (-sh) : (unsigned __int128)0);
                 }
-                mlo[e] = (uint64_t)full >> lc;
-                mhi[e] = (uint64_t)(full >> 64) >> lc;
+                mk[e] = (uint64_t)(full >> (64 * c)) >> lc;
+              } else {
+                const int n_vis = lim[h][e] - tile_tok0 - 64 * c;       // visible columns of the chunk
+                mk[e] = (n_vis <= 0 ? 0ull : (n_vis >= 64 ? ~0ull : ((1ull << n_vis) - 1ull))) >> lc;
               }
-  #pragma unroll
-              for (int k = 0; k < 32; ++k) {
-                const int e = (k >> 1) & 1, bit = (k >> 2) * 8 + (k & 1);
-                const float x0 = ((mlo[e] >> bit) & 1ull) ? __uint_as_float(v0[k]) * p.scale_log2 : -INFINITY;
-                const float x1 = ((mhi[e] >> bit) & 1ull) ? __uint_as_float(v1[k]) * p.scale_log2 : -INFINITY;
-                v0[k] = __float_as_uint(x0);
-                v1[k] = __float_as_uint(x1);
-                mx[k & 3] = fmaxf(mx[k & 3], fmaxf(x0, x1));
-              }
+            }
+          };
+          float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll 1
+          for (int c = 0; c < 2; ++c) {
+            uint32_t v[32];
+            tmem_ld_16x256b_x8(saddr + 64 * c, v);
+            tmem_ld_wait();
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            if (__builtin_expect(need_mask, 0)) {
+              uint64_t mk[2];
+              chunk_mask(c, mk);
+#pragma unroll
+              for (int k = 0; k < 32; ++k)
+                if ((mk[(k >> 1) & 1] >> ((k >> 2) * 8 + (k & 1))) & 1ull) mx[k & 3] = fmaxf(mx[k & 3], __uint_as_float(v[k]));
             } else {
 #pragma unroll
-              for (int k = 0; k < 32; ++k) {
-                const int tok = tile_tok0 + (k >> 2) * 8 + lc + (k & 1);
-                const int lm = lim[h][(k >> 1) & 1];
-                const float x0 = tok < lm ? __uint_as_float(v0[k]) * p.scale_log2 : -INFINITY;
-                const float x1 = tok + kTileTokens < lm ? __uint_as_float(v1[k]) * p.scale_log2 : -INFINITY;
-                v0[k] = __float_as_uint(x0);
-                v1[k] = __float_as_uint(x1);
-                mx[k & 3] = fmaxf(mx[k & 3], fmaxf(x0, x1));
-              }
+              for (int k = 0; k < 32; ++k) mx[k & 3] = fmaxf(mx[k & 3], __uint_as_float(v[k]));
             }
-          } else {
-#pragma unroll
-            for (int k = 0; k < 32; ++k) {
-              const float x0 = __uint_as_float(v0[k]) * p.scale_log2, x1 = __uint_as_float(v1[k]) * p.scale_log2;
-              v0[k] = __float_as_uint(x0);
-              v1[k] = __float_as_uint(x1);
-              mx[k & 3] = fmaxf(mx[k & 3], fmaxf(x0, x1));
-            }
+            mx0 = fmaxf(mx0, fmaxf(mx[0], mx[1]));
+            mx1 = fmaxf(mx1, fmaxf(mx[2], mx[3]));
           }
-          float mx0 = fmaxf(mx[0], mx[1]), mx1 = fmaxf(mx[2], mx[3]);
+          mx0 *= p.scale_log2;                                     // the scale is positive
+          mx1 *= p.scale_log2;
           mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
           mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
           mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
           mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+          // the group's previous product has completed: P may be overwritten, O may be rescaled
+          if (h == 0 && i >= 2) SM_WAIT(bar_p_empty + 8 * grp, ((i >> 1) - 1) & 1);
           if (j < 2) {
             // the group's first tile of the item: O is overwritten by this tile's product
             m_used[h][0] = mx0;
             m_used[h][1] = mx1;
           } else {
             const bool up0 = mx0 > m_used[h][0] + kRescaleThreshold, up1 = mx1 > m_used[h][1] + kRescaleThreshold;
-            if (__any_sync(0xffffffffu, up0 || up1)) {
+            if (__builtin_expect(__any_sync(0xffffffffu, up0 || up1) != 0, 0)) {
               // raise the reference maximum of those rows and rescale their O rows in TMEM
               const float a0 = up0 ? fast_exp2(m_used[h][0] - mx0) : 1.f;
               const float a1 = up1 ? fast_exp2(m_used[h][1] - mx1) : 1.f;
@@ -610,7 +597,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               l_sum[h][0] *= a0;
               l_sum[h][1] *= a1;
               tc_fence_after_sync();
-#pragma unroll
+#pragma unroll 1
               for (int cc = 0; cc < D / 64; ++cc) {
                 uint32_t o[32];
                 const uint32_t oaddr = tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + C::COL_O + grp * D + cc * 64;
@@ -625,25 +612,42 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               tc_fence_before_sync();
             }
           }
-          const float mu0 = m_used[h][0] == -INFINITY ? 0.f : m_used[h][0];
-          const float mu1 = m_used[h][1] == -INFINITY ? 0.f : m_used[h][1];
+          // probabilities: p = 2^(s * scale - m), with a row that sees nothing yet kept at zero
+          const float nmu0 = m_used[h][0] == -INFINITY ? 0.f : -m_used[h][0];
+          const float nmu1 = m_used[h][1] == -INFINITY ? 0.f : -m_used[h][1];
           float ps[4] = {0.f, 0.f, 0.f, 0.f};
           // rows of the A operand of O += P V: the item's rows
           const int m0 = row0(h) + lr, m1 = m0 + 8;
           const uint32_t prow0 = p_sm + grp * P_BYTES + m0 * 128 + lc * 2;
           const uint32_t prow1 = p_sm + grp * P_BYTES + m1 * 128 + lc * 2;
+#pragma unroll 1
+          for (int c = 0; c < 2; ++c) {                            // the tile's two 64-token blocks
+            uint32_t v[32];
+            tmem_ld_16x256b_x8(saddr + 64 * c, v);
+            tmem_ld_wait();
+            if (c == 1 && h == nh - 1) {
+              tc_fence_before_sync();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(bar_s_empty + 8 * grp);
+            }
+            if (__builtin_expect(need_mask, 0)) {
+              uint64_t mk[2];
+              chunk_mask(c, mk);
 #pragma unroll
-          for (int half = 0; half < 2; ++half) {          // the tile's two 64-token blocks
+              for (int k = 0; k < 32; ++k)
+                if (!((mk[(k >> 1) & 1] >> ((k >> 2) * 8 + (k & 1))) & 1ull)) v[k] = 0xff800000u;   // -inf
+            }
 #pragma unroll
             for (int jj = 0; jj < 8; ++jj) {
-              const uint32_t* vv = half ? v1 : v0;
-              const float p0 = fast_exp2(__uint_as_float(vv[4 * jj]) - mu0), p1 = fast_exp2(__uint_as_float(vv[4 * jj + 1]) - mu0);
-              const float p2 = fast_exp2(__uint_as_float(vv[4 * jj + 2]) - mu1), p3 = fast_exp2(__uint_as_float(vv[4 * jj + 3]) - mu1);
+              const float p0 = fast_exp2(fmaf(__uint_as_float(v[4 * jj]), p.scale_log2, nmu0));
+              const float p1 = fast_exp2(fmaf(__uint_as_float(v[4 * jj + 1]), p.scale_log2, nmu0));
+              const float p2 = fast_exp2(fmaf(__uint_as_float(v[4 * jj + 2]), p.scale_log2, nmu1));
+              const float p3 = fast_exp2(fmaf(__uint_as_float(v[4 * jj + 3]), p.scale_log2, nmu1));
               ps[jj & 1] += p0 + p1;
               ps[2 + (jj & 1)] += p2 + p3;
-              asm volatile("st.shared.b32 [%0], %1;" ::"r"(prow0 + half * (M * 128) + ((jj ^ (m0 & 7)) << 4)),
+              asm volatile("st.shared.b32 [%0], %1;" ::"r"(prow0 + c * (M * 128) + ((jj ^ (m0 & 7)) << 4)),
                            "r"(pack_bf16x2(p0, p1)) : "memory");
-              asm volatile("st.shared.b32 [%0], %1;" ::"r"(prow1 + half * (M * 128) + ((jj ^ (m1 & 7)) << 4)),
+              asm volatile("st.shared.b32 [%0], %1;" ::"r"(prow1 + c * (M * 128) + ((jj ^ (m1 & 7)) << 4)),
                            "r"(pack_bf16x2(p2, p3)) : "memory");
             }
           }
