@@ -19,8 +19,10 @@ namespace specvlm {
 // 4 consumer warps each own 16 of a tile's 64 tokens and keep private running (max, sum, O);
 // they are merged once at the end.  Warp 4 is the TMA producer.
 // ---------------------------------------------------------------------------------------------
-template <int D, int STAGES>
-__global__ void __launch_bounds__(160)
+// NG consumer groups of 4 warps take alternate tiles (NG = 2 where an SM holds a single CTA, so
+// that eight warps hide each other's latencies as two resident CTAs would).
+template <int D, int STAGES, int NG>
+__global__ void __launch_bounds__(32 * (4 * NG + 1))
 attn_rows16_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                    const AttnParams p) {
   constexpr int TILE_BYTES = kTileTokens * D * 2;
@@ -57,7 +59,7 @@ attn_rows16_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
   }
   __syncthreads();
 
-  if (warp == 4) {
+  if (warp == 4 * NG) {
     // ------------------------------------------------------------------ producer
     if (lane == 0 && n_my > 0) {
       tma_prefetch_desc(&tm_k);
@@ -138,11 +140,12 @@ attn_rows16_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 
   // per-lane ldmatrix row/chunk selectors
   const int mi = lane >> 3, r8 = lane & 7;
-  const int k_tok = warp * 16 + (mi >> 1) * 8 + r8, k_chunk = mi & 1;   // K: non-transposed
-  const int v_tok = warp * 16 + (mi & 1) * 8 + r8, v_chunk = mi >> 1;   // V: transposed
+  const int cw = warp & 3, grp = warp >> 2;                           // token slice, consumer group
+  const int k_tok = cw * 16 + (mi >> 1) * 8 + r8, k_chunk = mi & 1;   // K: non-transposed
+  const int v_tok = cw * 16 + (mi & 1) * 8 + r8, v_chunk = mi >> 1;   // V: transposed
 
   bool alive = true;
-  for (int i = 0; i < n_my; ++i) {
+  for (int i = grp; i < n_my; i += NG) {
     const int s = i % STAGES;
     if (!mbar_wait(bar_full + 8 * s, (i / STAGES) & 1, abort_flag)) {
       alive = false;
@@ -150,14 +153,14 @@ attn_rows16_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     }
     const uint32_t k_base = base + s * STAGE_BYTES;
     const uint32_t v_base = k_base + TILE_BYTES;
-    const int tb = (tile_begin + i) * kTileTokens + warp * 16;   // first token of this warp's slice
+    const int tb = (tile_begin + i) * kTileTokens + cw * 16;     // first token of this warp's slice
     if (tb < kv_len) {
       if (tb + 16 > kv_len) {
         // rows past the end of the sequence hold whatever the page held: clear V there so that
         // a zero probability times a stale non-finite value cannot reach the accumulator
         uint8_t* vt = smem + s * STAGE_BYTES + TILE_BYTES;
         const int first = kv_len - (tile_begin + i) * kTileTokens;      // first invalid local row
-        for (int t = first + (lane >> 3); t < warp * 16 + 16; t += 4) {
+        for (int t = first + (lane >> 3); t < cw * 16 + 16; t += 4) {
 #pragma unroll
           for (int h = 0; h < D / 64; ++h)
             *reinterpret_cast<uint4*>(vt + h * (kTileTokens * 128) + t * 128 + (lane & 7) * 16) =
@@ -233,13 +236,14 @@ attn_rows16_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     if (lane == 0) mbar_arrive(bar_empty + 8 * s);
   }
 
-  // ------------------------------------------------------------ merge the 4 warps' partials
+  // ------------------------------------------------------------ merge the consumer warps' partials
   // (named barrier over the 128 consumer threads; the producer warp has no part in it)
-  asm volatile("bar.sync 1, 128;" ::: "memory");
+  asm volatile("bar.sync 1, %0;" ::"n"(128 * NG) : "memory");
   if (!alive || *abort_flag) return;   // a wait expired somewhere in this CTA: leave outputs alone
-  float* const o_sm = reinterpret_cast<float*>(smem);                  // [4][16][OPITCH]
-  float* const m_sm = o_sm + 4 * 16 * OPITCH;                          // [4][16]
-  float* const l_sm = m_sm + 64;                                       // [4][16]
+  constexpr int NW = 4 * NG;                                           // consumer warps
+  float* const o_sm = reinterpret_cast<float*>(smem);                  // [NW][16][OPITCH]
+  float* const m_sm = o_sm + NW * 16 * OPITCH;                         // [NW][16]
+  float* const l_sm = m_sm + NW * 16;                                  // [NW][16]
   l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
   l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
   l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
@@ -258,15 +262,17 @@ attn_rows16_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
       l_sm[warp * 16 + row1] = l1;
     }
   }
-  asm volatile("bar.sync 1, 128;" ::: "memory");
+  asm volatile("bar.sync 1, %0;" ::"n"(128 * NG) : "memory");
   const int item = lb * p.n_kv_heads + g;
-  for (int idx = tid; idx < p.rows * D; idx += 128) {
+  for (int idx = tid; idx < p.rows * D; idx += 128 * NG) {
     const int r = idx / D, c = idx - r * D;
-    float M = fmaxf(fmaxf(m_sm[r], m_sm[16 + r]), fmaxf(m_sm[32 + r], m_sm[48 + r]));
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) M = fmaxf(M, m_sm[w * 16 + r]);
     float num = 0.f, den = 0.f;
     if (M != -INFINITY) {
 #pragma unroll
-      for (int w = 0; w < 4; ++w) {
+      for (int w = 0; w < NW; ++w) {
         const float f = fast_exp2(m_sm[w * 16 + r] - M);
         den += l_sm[w * 16 + r] * f;
         num += o_sm[(w * 16 + r) * OPITCH + c] * f;
@@ -290,19 +296,19 @@ attn_rows16_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
   // ------------------------------------------------------------ merge of the item's splits
   // The CTA that brings an item's last partial merges them all, in split order (so the result
   // does not depend on which CTA that is):  out = sum_s w_s o_s / sum_s w_s,  w_s = 2^(lse_s - max).
-  int* const last_sm = reinterpret_cast<int*>(l_sm + 64);
+  int* const last_sm = reinterpret_cast<int*>(l_sm + NW * 16);
   __threadfence();
-  asm volatile("bar.sync 1, 128;" ::: "memory");
+  asm volatile("bar.sync 1, %0;" ::"n"(128 * NG) : "memory");
   if (tid == 0) {
     const int old = atomicAdd(p.ws_cnt + item, 1);
     __threadfence();
     *last_sm = old == p.n_splits - 1;
   }
-  asm volatile("bar.sync 1, 128;" ::: "memory");
+  asm volatile("bar.sync 1, %0;" ::"n"(128 * NG) : "memory");
   if (!*last_sm) return;
   const float* lse_base = p.ws_lse + (size_t)item * p.n_splits * p.rows;
   const float* o_base = p.ws_o + (size_t)item * p.n_splits * p.rows * D;
-  for (int idx = tid; idx < p.rows * (D / 4); idx += 128) {
+  for (int idx = tid; idx < p.rows * (D / 4); idx += 128 * NG) {
     const int r = idx / (D / 4), c4 = idx - r * (D / 4);
     float M = -INFINITY;
 #pragma unroll 4
@@ -400,16 +406,27 @@ int32_t attn_tc_launch(const specvlm_kv_t* kv, const void* q, int32_t batch, int
                        float sm_scale, void* out, float* lse, void* ws, size_t ws_bytes, int32_t* d_status,
                        cudaStream_t st, const int32_t* tree_parents);
 
+template <int D, int STAGES, int NG>
+static int32_t launch_rows16_s(const CUtensorMap& tk, const CUtensorMap& tv, const AttnParams& p,
+                               dim3 grid, cudaStream_t st) {
+  constexpr int SMEM = STAGES * 2 * kTileTokens * D * 2 + 1024 + 16 * STAGES + 16;
+  auto kern = attn_rows16_kernel<D, STAGES, NG>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
+    return SPECVLM_ERR_CUDA;
+  kern<<<grid, 32 * (4 * NG + 1), SMEM, st>>>(tk, tv, p);
+  return launch_status();
+}
+
+// Ring depth: 3 stages let two CTAs share an SM; a launch with no more CTAs than SMs would leave
+// every SM with one CTA and 96 KB of copies in flight, too little to cover the HBM latency, so it
+// takes 6 stages and two consumer groups instead.
 template <int D>
 static int32_t launch_rows16(const CUtensorMap& tk, const CUtensorMap& tv, const AttnParams& p,
                              dim3 grid, cudaStream_t st) {
-  constexpr int STAGES = 3;
-  constexpr int SMEM = STAGES * 2 * kTileTokens * D * 2 + 1024 + 16 * STAGES + 16;
-  auto kern = attn_rows16_kernel<D, STAGES>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
-    return SPECVLM_ERR_CUDA;
-  kern<<<grid, 160, SMEM, st>>>(tk, tv, p);
-  return launch_status();
+  const int64_t ctas = (int64_t)grid.x * grid.y * grid.z;
+  constexpr int kDeep = D == 128 ? 6 : 12;
+  return ctas <= sm_count() ? launch_rows16_s<D, kDeep, 2>(tk, tv, p, grid, st)
+                            : launch_rows16_s<D, 3, 1>(tk, tv, p, grid, st);
 }
 
 static int32_t attn_common(const specvlm_kv_t* kv, const void* q, int32_t batch, int32_t n_q_heads,
