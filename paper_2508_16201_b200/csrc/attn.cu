@@ -357,17 +357,23 @@ static int choose_splits(int max_seq_len, int64_t items) {
   if (forced > 0) {
     best = forced;
   } else {
-    // All CTAs of a launch stream the same number of tiles, `per`, plus a fixed start-up / epilogue
-    // cost of about two tiles, and run in ceil(CTAs / resident slots) rounds.  Splitting also costs
-    // the counter reset before the launch and the merge at its end: about eight tile times,
-    // measured on the 755-token draft cache, where not splitting wins.
-    const int64_t slots = (int64_t)sm_count() * 2;
+    // Unit: the time one group of four warps needs for a tile, about 0.5 us.  A launch whose CTAs
+    // fit one per SM runs the two-group kernel (half that per tile); otherwise two CTAs share an
+    // SM and the launch runs in rounds over the resident slots.  Every CTA adds a start-up /
+    // epilogue cost of two to three tiles; splitting adds the counter reset before the launch and
+    // the merge at its end (about eight tiles, measured); and no launch beats the time HBM needs
+    // for the bytes (about 95 tiles of 32 KB per unit).  With these figures neither the 755-token
+    // nor the 6400-token draft cache of the 28-layer draft is split, which is what measures best.
+    const int64_t sms = sm_count(), slots = 2 * sms;
+    const double hbm_floor = (double)items * n_tiles / 95.0;
     double best_cost = 1e300;
     for (int s = 1; s <= 64 && s <= n_tiles; ++s) {
       const int per = (n_tiles + s - 1) / s;
       if ((s - 1) * per >= n_tiles) continue;            // would leave an empty split
-      const double rounds = (double)((items * s + slots - 1) / slots);
-      const double cost = rounds * (per + 2.0) + (s > 1 ? 8.0 : 0.0);
+      const int64_t ctas = items * s;
+      double cost = ctas <= sms ? 0.5 * per + 3.0 : (double)((ctas + slots - 1) / slots) * (per + 2.0);
+      if (cost < hbm_floor) cost = hbm_floor;
+      if (s > 1) cost += 8.0;
       if (cost < best_cost - 1e-9) {
         best_cost = cost;
         best = s;
