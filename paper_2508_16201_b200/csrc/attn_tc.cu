@@ -133,7 +133,7 @@ template <int D, int M>
 struct TcCfg {
   static constexpr int SUB_BYTES = kTileTokens * D * 2;         // one 64-token K (or V) sub-tile
   static constexpr int NKP = D == 128 ? 2 : 3;                  // K ring: pair slots (128 tokens)
-  static constexpr int NVP = D == 128 ? (M == 64 ? 3 : 1) : 3;  // V ring: pair slots
+  static constexpr int NVP = D == 128 ? (M == 64 ? 3 : 2) : 3;  // V ring: pair slots
   static constexpr int NQ = (D == 128 && M == 128) ? 1 : 2;     // query buffers
   static constexpr int Q_BYTES = M * D * 2;                     // A operand of S = Q K^T
   static constexpr int P_BYTES = M * kBigTokens * 2;            // A operand of O += P V
@@ -146,8 +146,8 @@ struct TcCfg {
   static constexpr int SM_BAR = 0;
   static constexpr int SM_MISC = SM_BAR + 8 * N_BARS;
   static constexpr int SM_PREFIX = SM_MISC + 32;
-  static constexpr int SM_STATS = SM_PREFIX + (kSchedMaxBatch + 1) * 4;     // [2 segments][2 groups][M rows] float2
-  static constexpr int SMALL_USED = SM_STATS + 2 * 2 * M * 8;
+  static constexpr int SM_STATS = SM_PREFIX + (kSchedMaxBatch + 1) * 4;     // [2 groups][M rows] float2
+  static constexpr int SMALL_USED = SM_STATS + 2 * M * 8;
   static constexpr int SMALL = (SMALL_USED + 1023) / 1024 * 1024;
   static constexpr int kMaxSmem = 232448;                       // 227 KB
   // a spare KB for a base that is not 1024-byte aligned, where there is room for it
@@ -666,9 +666,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       const bool complete = sg.tile0 == 0 && sg.n_tiles == sg.item_tiles;
       const int lb = sg.layer * p.batch + sg.b;
       const int slot = partial_slot(cta, T0, sg.item_begin);
-      // statistics slots alternate between segments: a group may reach its next write while the
-      // other one still reads this segment's values
-      float2* const seg_stats = stats + (seg_idx & 1) * 2 * M;
+      // a group may get here while the other one still reads the previous segment's statistics:
+      // wait until both have left that epilogue (the barrier the PV issuer waits on as well)
+      float2* const seg_stats = stats;
+      if (seg_idx >= 1) SM_WAIT(bar_o_empty, (seg_idx - 1) & 1);
 #pragma unroll
       for (int h = 0; h < NH; ++h) {
         if (h >= nh) break;
