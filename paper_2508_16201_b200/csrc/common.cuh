@@ -141,6 +141,60 @@ __device__ __forceinline__ float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Packed pairs of fp32 (sm_100 issues an f32x2 operation on two values in one slot).
+__device__ __forceinline__ uint64_t f2_pack(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t f2_sub(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// 2^t for a pair of arguments t <= 0 on the FMA and integer pipes, leaving the special-function
+// unit to other elements: t = n + f with n = round(t) and |f| <= 1/2 (adding 1.5 * 2^23 leaves n in
+// the low mantissa bits), 2^f by a degree-4 polynomial (least-maximum relative error 2.7e-6 on
+// [-1/2, 1/2], fitted for this file), and n added to the exponent field.  Arguments below -125 give
+// 2^-125 instead of 0.
+__device__ __forceinline__ uint64_t f2_exp2_poly(uint64_t t2) {
+  float a, b;
+  f2_unpack(t2, a, b);
+  t2 = f2_pack(fmaxf(a, -125.f), fmaxf(b, -125.f));
+  const uint64_t magic = f2_pack(12582912.f, 12582912.f);
+  const uint64_t r2 = f2_add(t2, magic);
+  const uint64_t f2 = f2_sub(t2, f2_sub(r2, magic));
+  uint64_t p = f2_fma(f2_pack(0.009569965302944183f, 0.009569965302944183f), f2,
+                      f2_pack(0.05591750890016556f, 0.05591750890016556f));
+  p = f2_fma(p, f2, f2_pack(0.240247443318367f, 0.240247443318367f));
+  p = f2_fma(p, f2, f2_pack(0.6931218504905701f, 0.6931218504905701f));
+  p = f2_fma(p, f2, f2_pack(0.9999992847442627f, 0.9999992847442627f));
+  float p0, p1, r0, r1;
+  f2_unpack(p, p0, p1);
+  f2_unpack(r2, r0, r1);
+  p0 = __int_as_float(__float_as_int(p0) + (__float_as_int(r0) << 23));
+  p1 = __int_as_float(__float_as_int(p1) + (__float_as_int(r1) << 23));
+  return f2_pack(p0, p1);
+}
+__device__ __forceinline__ uint64_t f2_exp2_sfu(uint64_t t2) {
+  float a, b;
+  f2_unpack(t2, a, b);
+  return f2_pack(fast_exp2(a), fast_exp2(b));
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&t);

@@ -460,6 +460,20 @@ scores_colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
   }
 }
 
+#ifndef SPECVLM_POLY_LSE
+#define SPECVLM_POLY_LSE 2
+#endif
+#ifndef SPECVLM_POLY_COLSUM
+#define SPECVLM_POLY_COLSUM 0
+#endif
+// Of every 8 pairs of logits, this many take their exponential on the FMA pipe (f2_exp2_poly)
+// instead of the special-function unit, which both rating passes nearly saturate.  Measured: the
+// polynomial costs about as many FMA-pipe cycles per value as the unit it relieves (8), so it only
+// pays where issue slots are left over: 2 of 8 in pass 1 (-3 %); none in pass 2, whose four
+// epilogue groups already keep the unit busy (every share made it slower).
+constexpr int kPolyOf8Lse = SPECVLM_POLY_LSE;
+constexpr int kPolyOf8Colsum = SPECVLM_POLY_COLSUM;
+
 // ---------------------------------------------------------------------------------------------
 // Pass 2 on the 5th-generation tensor cores.  CTA = (block of 128 video keys, layer), looping over
 // the layer's KV heads and the sequence's row tiles as above, but
@@ -470,17 +484,23 @@ scores_colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
 // tile's epilogue).  With the keys on the TMEM lanes, an epilogue thread owns one key: it reads
 // its 128 row values with tcgen05.ld and adds up 2^(s - lse_row) in a single register for the
 // whole layer -- the column sum needs no cross-thread reduction at all.
-// Warps: 0 = TMA producer, 1 = TMEM allocation + MMA issue, 2..5 and 6..9 = two epilogue groups
-// (one TMEM lane quadrant per warp) that take alternate tiles, each on its own accumulator
-// buffer, so that one group's exponentials run while the other waits for its TMEM load.
+// Warps: 0 = TMA producer, 1 = TMEM allocation + MMA issue, then kColsumGroups epilogue groups of
+// four warps (one TMEM lane quadrant per warp) that take the tiles round-robin, each on its own
+// accumulator buffer: four warps per scheduler keep the special-function unit busy while others
+// wait for a TMEM load, a barrier or the row statistics.
 // ---------------------------------------------------------------------------------------------
+constexpr int kColsumGroups = 4;
+constexpr int kColsumThreads = 64 + 128 * kColsumGroups;
+
 template <int D, int STAGES>
-__global__ void __launch_bounds__(320, 1)
+__global__ void __launch_bounds__(kColsumThreads, 1)
 scores_colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
                         const __grid_constant__ ScoreParams p) {
   constexpr int TILE_BYTES = kKeyTile * D * 2;
   constexpr int KSTEPS = D / 16;
-  constexpr uint32_t kTmemCols = 256;
+  constexpr int NG = kColsumGroups;
+  constexpr uint32_t kTmemCols = 128 * NG;
+  static_assert(kTmemCols == 256 || kTmemCols == 512, "tensor memory is allocated in powers of two");
   constexpr uint32_t kIdesc = umma_idesc_bf16(128, 128, false, false);
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -493,12 +513,12 @@ scores_colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
   const uint32_t bar_qempty = bar_qfull + 8 * STAGES;
   const uint32_t bar_kfull = bar_qempty + 8 * STAGES;            // [2]
   const uint32_t bar_kempty = bar_kfull + 16;                    // [2]
-  const uint32_t bar_tfull = bar_kempty + 16;                    // [2]
-  const uint32_t bar_tempty = bar_tfull + 16;                    // [2]
-  uint8_t* const tail = smem + kTail + 16 * STAGES + 64;
+  const uint32_t bar_tfull = bar_kempty + 16;                    // [NG]
+  const uint32_t bar_tempty = bar_tfull + 8 * NG;                // [NG]
+  uint8_t* const tail = smem + kTail + 16 * STAGES + 32 + 16 * NG;
   volatile int* const abort_flag = reinterpret_cast<volatile int*>(tail);
   volatile uint32_t* const tmem_slot = reinterpret_cast<volatile uint32_t*>(tail + 8);
-  float* const lse_sm = reinterpret_cast<float*>(tail + 16);     // [2][128], log2 units
+  float* const lse_sm = reinterpret_cast<float*>(tail + 16);     // [NG groups][2][128]: -lse in log2 units
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int b = find_seq(p, blockIdx.x);
@@ -518,6 +538,8 @@ scores_colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_kfull + 8 * i, 1);
       mbar_init(bar_kempty + 8 * i, 1);
+    }
+    for (int i = 0; i < NG; ++i) {
       mbar_init(bar_tfull + 8 * i, 1);
       mbar_init(bar_tempty + 8 * i, 4);
     }
@@ -575,9 +597,9 @@ scores_colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
         const int kb = u & 1;
         ok = mbar_wait(bar_kfull + 8 * kb, (u >> 1) & 1, abort_flag);
         for (int t = 0; t < n_qt && ok; ++t, ++it) {
-          const int s = it % STAGES, buf = it & 1;
+          const int s = it % STAGES, buf = it % NG;
           ok = mbar_wait(bar_qfull + 8 * s, (it / STAGES) & 1, abort_flag);
-          if (ok && it >= 2) ok = mbar_wait(bar_tempty + 8 * buf, ((it >> 1) - 1) & 1, abort_flag);
+          if (ok && it >= NG) ok = mbar_wait(bar_tempty + 8 * buf, ((it / NG) - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
           const uint32_t a0 = k_sm + kb * TILE_BYTES, b0 = q_sm + s * TILE_BYTES;
@@ -597,82 +619,90 @@ scores_colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
       if (!ok && p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
     }
   } else {
-    // ---------------------------------------------------------------- epilogue: 2 groups x 4 warps, 128 keys
-    const int grp = (warp - 2) >> 2;            // tiles with (index & 1) == grp, accumulator buffer grp
+    // ---------------------------------------------------------------- epilogue: NG groups x 4 warps, 128 keys
+    const int grp = (warp - 2) >> 2;            // tiles with index % NG == grp, accumulator buffer grp
     const int quad = warp & 3;                  // TMEM lanes [32 * quad, 32 * quad + 32)
     const int key_l = quad * 32 + lane;         // this thread's key inside the block
     const int et = ((warp - 2) & 3) * 32 + lane;   // 0..127 inside the group: used to stage the row LSEs
-    float acc = 0.f;
+    float* const lse_g = lse_sm + grp * 256;    // this group's two staging buffers of 128 rows
+    // -lse (log2 units) of row `et` of tile `tile`; -inf for rows past the valid ones, whose
+    // exponentials then vanish
+    auto lse_fetch = [&](int tile) -> float {
+      if (tile >= n_tiles) return 0.f;
+      const int u = tile / n_qt, t = tile - u * n_qt;
+      const int rows_valid = min(p.qt, sq.n_text - t * p.qt) * p.group;
+      if (et >= rows_valid) return -INFINITY;
+      const int il = et / p.group, hg = et - il * p.group;
+      return -__ldg(p.lse + ((size_t)layer * p.sum_text + sq.text_off + t * p.qt + il) * p.n_q_heads + u * p.group + hg) *
+             kLog2e;
+    };
+    uint64_t acc2[4] = {0ull, 0ull, 0ull, 0ull};   // four chains of pairs for instruction-level parallelism
     bool alive = true;
-    int it = 0;
-    for (int u = 0; u < n_units; ++u) {
-      const float* lse_u = p.lse + ((size_t)layer * p.sum_text + sq.text_off) * p.n_q_heads + u * p.group;
-      for (int t = 0; t < n_qt; ++t, ++it) {
-        const int buf = it & 1;
-        if (buf != grp) continue;
-        const int rows_valid = min(p.qt, sq.n_text - t * p.qt) * p.group;
-        {
-          float v = 0.f;
-          if (et < rows_valid) {
-            const int il = et / p.group, hg = et - il * p.group;
-            v = __ldg(lse_u + (size_t)(t * p.qt + il) * p.n_q_heads + hg) * kLog2e;
-          }
-          lse_sm[buf * 128 + et] = v;
-        }
-        asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory");
-        if (alive && !mbar_wait(bar_tfull + 8 * buf, (it >> 1) & 1, abort_flag)) alive = false;
-        alive = __all_sync(0xffffffffu, alive); // warp-uniform: the TMEM loads below are warp-collective
-        if (!alive) continue;                   // keep taking part in the barrier above
-        tc_fence_after_sync();
-        const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * 128;
-        uint32_t v0[32], v1[32], v2[32], v3[32];
-        tmem_ld_x32(taddr, v0);
-        tmem_ld_x32(taddr + 32, v1);
-        tmem_ld_x32(taddr + 64, v2);
-        tmem_ld_x32(taddr + 96, v3);
+    float lv = lse_fetch(grp);
+    int n = 0;
+    for (int it = grp; it < n_tiles; it += NG, ++n) {
+      const int buf = grp;
+      float* const ls = lse_g + (n & 1) * 128;
+      ls[et] = lv;
+      // one barrier per tile: the buffer written here was last read two tiles ago, before the
+      // previous tile's barrier
+      asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory");
+      lv = lse_fetch(it + NG);                  // in flight during this tile's exponentials
+      if (alive && !mbar_wait(bar_tfull + 8 * buf, (it / NG) & 1, abort_flag)) alive = false;
+      alive = __all_sync(0xffffffffu, alive);   // warp-uniform: the TMEM loads below are warp-collective
+      if (!alive) continue;                     // keep taking part in the barrier above
+      tc_fence_after_sync();
+      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * 128;
+      const uint64_t sc2 = f2_pack(p.scale_log2, p.scale_log2);
+      uint32_t va[32], vb[32];                  // the load of chunk c + 1 flies while chunk c is summed
+      tmem_ld_x32(taddr, va);
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t(&v)[32] = (c & 1) ? vb : va;
         tmem_ld_wait();
-        tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);   // buffer free for the MMAs of tile it+2
-        const float* ls = lse_sm + buf * 128;
-        if (rows_valid == 128) {
-          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;    // four chains for instruction-level parallelism
-#pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            const float4 l0 = *reinterpret_cast<const float4*>(ls + j);
-            const float4 l1 = *reinterpret_cast<const float4*>(ls + 32 + j);
-            const float4 l2 = *reinterpret_cast<const float4*>(ls + 64 + j);
-            const float4 l3 = *reinterpret_cast<const float4*>(ls + 96 + j);
-            a0 += fast_exp2(__uint_as_float(v0[j]) * p.scale_log2 - l0.x) + fast_exp2(__uint_as_float(v0[j + 1]) * p.scale_log2 - l0.y) +
-                  fast_exp2(__uint_as_float(v0[j + 2]) * p.scale_log2 - l0.z) + fast_exp2(__uint_as_float(v0[j + 3]) * p.scale_log2 - l0.w);
-            a1 += fast_exp2(__uint_as_float(v1[j]) * p.scale_log2 - l1.x) + fast_exp2(__uint_as_float(v1[j + 1]) * p.scale_log2 - l1.y) +
-                  fast_exp2(__uint_as_float(v1[j + 2]) * p.scale_log2 - l1.z) + fast_exp2(__uint_as_float(v1[j + 3]) * p.scale_log2 - l1.w);
-            a2 += fast_exp2(__uint_as_float(v2[j]) * p.scale_log2 - l2.x) + fast_exp2(__uint_as_float(v2[j + 1]) * p.scale_log2 - l2.y) +
-                  fast_exp2(__uint_as_float(v2[j + 2]) * p.scale_log2 - l2.z) + fast_exp2(__uint_as_float(v2[j + 3]) * p.scale_log2 - l2.w);
-            a3 += fast_exp2(__uint_as_float(v3[j]) * p.scale_log2 - l3.x) + fast_exp2(__uint_as_float(v3[j + 1]) * p.scale_log2 - l3.y) +
-                  fast_exp2(__uint_as_float(v3[j + 2]) * p.scale_log2 - l3.z) + fast_exp2(__uint_as_float(v3[j + 3]) * p.scale_log2 - l3.w);
-          }
-          acc += (a0 + a1) + (a2 + a3);
+        if (c < 3) {
+          tmem_ld_x32(taddr + (c + 1) * 32, (c & 1) ? va : vb);
         } else {
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);   // buffer free for the MMAs of tile it + NG
+        }
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            if (j < rows_valid) acc += fast_exp2(__uint_as_float(v0[j]) * p.scale_log2 - ls[j]);
-            if (32 + j < rows_valid) acc += fast_exp2(__uint_as_float(v1[j]) * p.scale_log2 - ls[32 + j]);
-            if (64 + j < rows_valid) acc += fast_exp2(__uint_as_float(v2[j]) * p.scale_log2 - ls[64 + j]);
-            if (96 + j < rows_valid) acc += fast_exp2(__uint_as_float(v3[j]) * p.scale_log2 - ls[96 + j]);
-          }
+        for (int q = 0; q < 16; q += 2) {
+          const float4 l4 = *reinterpret_cast<const float4*>(ls + c * 32 + 2 * q);
+          const uint64_t ta = f2_fma(f2_pack(__uint_as_float(v[2 * q]), __uint_as_float(v[2 * q + 1])), sc2,
+                                     f2_pack(l4.x, l4.y));
+          const uint64_t tb = f2_fma(f2_pack(__uint_as_float(v[2 * q + 2]), __uint_as_float(v[2 * q + 3])), sc2,
+                                     f2_pack(l4.z, l4.w));
+          // kPolyOf8Colsum of every 8 pairs take the polynomial, spread so both kinds interleave
+          const bool pa = ((q & 7) * kPolyOf8Colsum) / 8 != (((q & 7) + 1) * kPolyOf8Colsum) / 8;
+          const bool pb = (((q + 1) & 7) * kPolyOf8Colsum) / 8 != ((((q + 1) & 7) + 1) * kPolyOf8Colsum) / 8;
+          acc2[q & 3] = f2_add(acc2[q & 3], pa ? f2_exp2_poly(ta) : f2_exp2_sfu(ta));
+          acc2[(q + 1) & 3] = f2_add(acc2[(q + 1) & 3], pb ? f2_exp2_poly(tb) : f2_exp2_sfu(tb));
         }
       }
     }
-    // the key's column sum = group 0's tiles + group 1's tiles (fixed order)
-    float* const acc_sm = lse_sm;               // [128]: the staging area is free after the last tile
-    asm volatile("bar.sync 3, 256;" ::: "memory");
-    if (grp == 1) acc_sm[key_l] = acc;
-    asm volatile("bar.sync 3, 256;" ::: "memory");
+    float acc;
+    {
+      float s0, s1, s2, s3, s4, s5, s6, s7;
+      f2_unpack(acc2[0], s0, s1);
+      f2_unpack(acc2[1], s2, s3);
+      f2_unpack(acc2[2], s4, s5);
+      f2_unpack(acc2[3], s6, s7);
+      acc = ((s0 + s1) + (s2 + s3)) + ((s4 + s5) + (s6 + s7));
+    }
+    // the key's column sum = the groups' sums added in group order (fixed)
+    float* const acc_sm = lse_sm;               // [NG - 1][128]: the staging area is free after the last tile
+    asm volatile("bar.sync %0, %1;" ::"r"(NG + 1), "r"(128 * NG) : "memory");
+    if (grp > 0) acc_sm[(grp - 1) * 128 + key_l] = acc;
+    asm volatile("bar.sync %0, %1;" ::"r"(NG + 1), "r"(128 * NG) : "memory");
     if (alive && !*abort_flag) {
       const int j = key0 + key_l - sq.video_start;           // video token index of this key
-      if (grp == 0 && j >= 0 && j < sq.n_video)
-        p.partial[(size_t)layer * p.sum_video + sq.score_off + j] = acc + acc_sm[key_l];
+      if (grp == 0 && j >= 0 && j < sq.n_video) {
+#pragma unroll
+        for (int g = 1; g < NG; ++g) acc += acc_sm[(g - 1) * 128 + key_l];
+        p.partial[(size_t)layer * p.sum_video + sq.score_off + j] = acc;
+      }
     } else if (p.d_status && et == 0) {
       *p.d_status = SPECVLM_ERR_TIMEOUT;
     }
@@ -825,37 +855,43 @@ scores_lse_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * 128;
       const int key0 = i * kKeyTile;
       const bool need_mask = key0 + kKeyTile > first_lim;
+      uint32_t va[32], vb[32];                    // the load of chunk c + 1 flies while chunk c is summed
+      tmem_ld_x32(taddr, va);
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
-        uint32_t v[32];
-        tmem_ld_x32(taddr + c * 32, v);
+        uint32_t(&v)[32] = (c & 1) ? vb : va;
         tmem_ld_wait();
-        if (c == 3) {
+        if (c < 3) {
+          tmem_ld_x32(taddr + (c + 1) * 32, (c & 1) ? va : vb);
+        } else {
           tc_fence_before_sync();
           __syncwarp();
           if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);   // buffer free for the MMAs of tile i + 2
         }
-        float x[32];
-        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
         if (need_mask) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            x[j] = key0 + c * 32 + j < lim ? __uint_as_float(v[j]) * p.scale_log2 : -INFINITY;
-            mx[j & 3] = fmaxf(mx[j & 3], x[j]);
-          }
-        } else {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            x[j] = __uint_as_float(v[j]) * p.scale_log2;
-            mx[j & 3] = fmaxf(mx[j & 3], x[j]);
-          }
+          for (int j = 0; j < 32; ++j)
+            if (key0 + c * 32 + j >= lim) v[j] = 0xff800000u;   // -inf: hidden by the causal rule
         }
-        const float mn = fmaxf(m, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])));
-        const float mu = mn == -INFINITY ? 0.f : mn;
-        float ps[4] = {0.f, 0.f, 0.f, 0.f};       // four chains for instruction-level parallelism
+        // the scale is positive, so the maximum of the raw products gives the maximum logit
+        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int j = 0; j < 32; ++j) ps[j & 3] += fast_exp2(x[j] - mu);
-        l = l * fast_exp2(m - mu) + ((ps[0] + ps[1]) + (ps[2] + ps[3]));
+        for (int j = 0; j < 32; j += 2) mx[(j >> 1) & 3] = fmaxf(mx[(j >> 1) & 3], fmaxf(__uint_as_float(v[j]), __uint_as_float(v[j + 1])));
+        const float mn = fmaxf(m, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2);
+        const float mu = mn == -INFINITY ? 0.f : mn;
+        const uint64_t sc2 = f2_pack(p.scale_log2, p.scale_log2), nmu2 = f2_pack(-mu, -mu);
+        uint64_t ps[2] = {0ull, 0ull};            // two chains of pairs
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+          const uint64_t t2 = f2_fma(f2_pack(__uint_as_float(v[2 * q]), __uint_as_float(v[2 * q + 1])), sc2, nmu2);
+          // kPolyOf8Lse of every 8 pairs take the polynomial, spread so both kinds interleave
+          const bool poly = ((q & 7) * kPolyOf8Lse) / 8 != (((q & 7) + 1) * kPolyOf8Lse) / 8;
+          ps[q & 1] = f2_add(ps[q & 1], poly ? f2_exp2_poly(t2) : f2_exp2_sfu(t2));
+        }
+        float s0, s1, s2, s3;
+        f2_unpack(ps[0], s0, s1);
+        f2_unpack(ps[1], s2, s3);
+        l = l * fast_exp2(m - mu) + ((s0 + s1) + (s2 + s3));
         m = mn;
       }
     }
@@ -1035,11 +1071,12 @@ static int32_t launch_colsum(ScoreSetup& su, float* scores, cudaStream_t st) {
     rc = launch_status();
   } else {
     constexpr int STAGES = 4;
-    constexpr int SMEM = (2 + STAGES) * kKeyTile * D * 2 + 1024 + 16 * STAGES + 64 + 16 + 2 * 128 * 4;
+    constexpr int SMEM = (2 + STAGES) * kKeyTile * D * 2 + 1024 + 16 * STAGES + 32 + 16 * kColsumGroups + 16 +
+                         kColsumGroups * 2 * 128 * 4;
     auto k = scores_colsum_tc_kernel<D, STAGES>;
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
       return SPECVLM_ERR_CUDA;
-    k<<<dim3((unsigned)su.n_key_blocks, (unsigned)su.kv.n_layers), 320, SMEM, st>>>(su.tk, su.tq, su.p2);
+    k<<<dim3((unsigned)su.n_key_blocks, (unsigned)su.kv.n_layers), kColsumThreads, SMEM, st>>>(su.tk, su.tq, su.p2);
     rc = launch_status();
   }
   if (rc != SPECVLM_OK) return rc;
