@@ -78,4 +78,33 @@ SPECVLM_HD int partial_slot(int c, int64_t cta_slice_begin, int64_t item_begin) 
   return cta_slice_begin >= item_begin ? 2 * c : 2 * c + 1;
 }
 
+// Walks a CTA's slice segment by segment, in flat order.  (Taking the item that the slice end cuts
+// first, so that the merges of cut items happen early, was measured slower: the partial results'
+// stores and fences then wait behind the full-rate K/V streams of the other CTAs.)
+struct SliceCursor {
+  int64_t f, end;
+  Segment sg;
+  int j;          // tile inside the current segment
+  int seg_idx;    // segments entered so far - 1
+  SPECVLM_HD void start(int64_t begin, int64_t end_, const int* prefix, int batch, int hkv) {
+    f = begin;
+    end = end_;
+    j = 0;
+    seg_idx = 0;
+    if (f < end) sg = segment_at(f, end, prefix, batch, hkv);
+  }
+  SPECVLM_HD bool done() const { return f >= end; }
+  SPECVLM_HD bool last_of_segment() const { return j == sg.n_tiles - 1; }
+  SPECVLM_HD void next_tile(const int* prefix, int batch, int hkv) {
+    ++f;
+    if (++j == sg.n_tiles) next_segment(prefix, batch, hkv);
+  }
+  SPECVLM_HD void next_segment(const int* prefix, int batch, int hkv) {
+    f = sg.item_begin + sg.tile0 + sg.n_tiles;
+    j = 0;
+    ++seg_idx;
+    if (f < end) sg = segment_at(f, end, prefix, batch, hkv);
+  }
+};
+
 }  // namespace specvlm

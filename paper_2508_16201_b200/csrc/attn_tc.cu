@@ -98,32 +98,6 @@ __device__ __forceinline__ float4 ldg_cg_f32x4(const float* p) {
   return v;
 }
 
-// Walks a CTA's slice segment by segment.
-struct SliceCursor {
-  int64_t f, end;
-  Segment sg;
-  int j;          // tile inside the current segment
-  int seg_idx;    // segments entered so far - 1
-  __device__ __forceinline__ void start(int64_t begin, int64_t end_, const int* prefix, int batch, int hkv) {
-    f = begin;
-    end = end_;
-    j = 0;
-    seg_idx = 0;
-    if (f < end) sg = segment_at(f, end, prefix, batch, hkv);
-  }
-  __device__ __forceinline__ bool last_of_segment() const { return j == sg.n_tiles - 1; }
-  __device__ __forceinline__ void next_tile(const int* prefix, int batch, int hkv) {
-    ++f;
-    if (++j == sg.n_tiles) next_segment(prefix, batch, hkv);
-  }
-  __device__ __forceinline__ void next_segment(const int* prefix, int batch, int hkv) {
-    f = sg.item_begin + sg.tile0 + sg.n_tiles;
-    j = 0;
-    ++seg_idx;
-    if (f < end) sg = segment_at(f, end, prefix, batch, hkv);
-  }
-};
-
 __device__ __forceinline__ int clamp_len(int n, int max_len) { return n < 0 ? 0 : (n > max_len ? max_len : n); }
 
 // Shared-memory plan.  A small region (barriers, flags, per-sequence tile counts, the softmax
@@ -297,7 +271,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       c.start(T0, T1, prefix, p.batch, hkv);
       bool ok = true;
       int i = 0;
-      while (c.f < T1 && ok) {
+      while (!c.done() && ok) {
         const Segment sg = c.sg;
         if (is_k) {
           // the item's query rows: a box of (64 channels) x (group heads) x (n_q tokens) per 64-channel block
@@ -486,7 +460,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     if (!ok) goto softmax_done;                                                     \
   } while (0)
 
-    while (c.f < T1) {
+    while (!c.done()) {
       const Segment sg = c.sg;
       const int seg_idx = c.seg_idx;
       const int kv_len = clamp_len(p.seq_lens[sg.b], p.max_seq_len);
@@ -774,35 +748,79 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         ++n_partial;
         if (*last_flag) {
           __threadfence();
-          for (int idx = st; idx < p.rows * (D / 4); idx += 256) {
-            const int r = idx / (D / 4), c4 = idx - r * (D / 4);
-            float mm = -INFINITY;
-            for (int cpart = c_first; cpart <= c_last; ++cpart) {
-              const int sl = partial_slot(cpart, slice_begin(cpart, n_active, total), sg.item_begin);
-              mm = fmaxf(mm, ldg_cg_f32(p.ws_lse + (size_t)sl * p.rows + r));
+          // Two output positions per thread and pass, the parts in chunks of kMergeChunk: every
+          // load of a chunk is issued before the first is used, so a pass costs one trip to the L2
+          // instead of one per part and value.  Parts are folded in slice order (fixed).
+          constexpr int kMergeChunk = 4;
+          const int n_parts = c_last - c_first + 1;
+          const int n_idx = p.rows * (D / 4);
+          for (int idx0 = st; idx0 < n_idx; idx0 += 512) {
+            int r[2], c4[2];
+            bool on[2];
+            float mm[2] = {-INFINITY, -INFINITY}, den[2] = {0.f, 0.f};
+            float4 acc[2] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f)};
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+              const int idx = idx0 + 256 * u;
+              on[u] = idx < n_idx;
+              r[u] = on[u] ? idx / (D / 4) : 0;
+              c4[u] = on[u] ? idx - r[u] * (D / 4) : 0;
             }
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            float den = 0.f;
-            if (mm != -INFINITY) {
-              for (int cpart = c_first; cpart <= c_last; ++cpart) {
-                const int sl = partial_slot(cpart, slice_begin(cpart, n_active, total), sg.item_begin);
-                const float w = fast_exp2(ldg_cg_f32(p.ws_lse + (size_t)sl * p.rows + r) - mm);
-                const float4 x = ldg_cg_f32x4(p.ws_o + ((size_t)sl * p.rows + r) * D + c4 * 4);
-                acc.x += w * x.x;
-                acc.y += w * x.y;
-                acc.z += w * x.z;
-                acc.w += w * x.w;
-                den += w;
+            for (int pc = 0; pc < n_parts; pc += kMergeChunk) {
+              float ls[2][kMergeChunk];
+              float4 x[2][kMergeChunk];
+#pragma unroll
+              for (int q = 0; q < kMergeChunk; ++q) {
+                const bool have = pc + q < n_parts;
+                const int cpart = c_first + pc + q;
+                const int sl = have ? partial_slot(cpart, slice_begin(cpart, n_active, total), sg.item_begin) : 0;
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                  if (have && on[u]) {
+                    ls[u][q] = ldg_cg_f32(p.ws_lse + (size_t)sl * p.rows + r[u]);
+                    x[u][q] = ldg_cg_f32x4(p.ws_o + ((size_t)sl * p.rows + r[u]) * D + c4[u] * 4);
+                  } else {
+                    ls[u][q] = -INFINITY;
+                    x[u][q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                  }
+                }
+              }
+#pragma unroll
+              for (int u = 0; u < 2; ++u) {
+                float m2 = mm[u];
+#pragma unroll
+                for (int q = 0; q < kMergeChunk; ++q) m2 = fmaxf(m2, ls[u][q]);
+                if (m2 == -INFINITY) continue;
+                const float sc = mm[u] == -INFINITY ? 0.f : fast_exp2(mm[u] - m2);
+                acc[u].x *= sc;
+                acc[u].y *= sc;
+                acc[u].z *= sc;
+                acc[u].w *= sc;
+                den[u] *= sc;
+#pragma unroll
+                for (int q = 0; q < kMergeChunk; ++q) {
+                  const float w = ls[u][q] == -INFINITY ? 0.f : fast_exp2(ls[u][q] - m2);
+                  acc[u].x += w * x[u][q].x;
+                  acc[u].y += w * x[u][q].y;
+                  acc[u].z += w * x[u][q].z;
+                  acc[u].w += w * x[u][q].w;
+                  den[u] += w;
+                }
+                mm[u] = m2;
               }
             }
-            const float invd = den > 0.f ? 1.f / den : 0.f;
-            const int t = r / p.group, hq = sg.g * p.group + (r - t * p.group);
-            const size_t orow = ((size_t)lb * p.n_q + t) * p.n_q_heads + hq;
-            uint2 packed;
-            packed.x = pack_bf16x2(acc.x * invd, acc.y * invd);
-            packed.y = pack_bf16x2(acc.z * invd, acc.w * invd);
-            *reinterpret_cast<uint2*>(p.out + orow * D + c4 * 4) = packed;
-            if (p.lse && c4 == 0) p.lse[orow] = den > 0.f ? (mm + log2f(den)) * kLn2 : -INFINITY;
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+              if (!on[u]) continue;
+              const float invd = den[u] > 0.f ? 1.f / den[u] : 0.f;
+              const int t = r[u] / p.group, hq = sg.g * p.group + (r[u] - t * p.group);
+              const size_t orow = ((size_t)lb * p.n_q + t) * p.n_q_heads + hq;
+              uint2 packed;
+              packed.x = pack_bf16x2(acc[u].x * invd, acc[u].y * invd);
+              packed.y = pack_bf16x2(acc[u].z * invd, acc[u].w * invd);
+              *reinterpret_cast<uint2*>(p.out + orow * D + c4[u] * 4) = packed;
+              if (p.lse && c4[u] == 0) p.lse[orow] = den[u] > 0.f ? (mm[u] + log2f(den[u])) * kLn2 : -INFINITY;
+            }
           }
         }
       }

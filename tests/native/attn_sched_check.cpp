@@ -54,6 +54,36 @@ static int check(const std::vector<int>& tiles, int n_layers, int hkv, int grid)
       f += s.n_tiles;
       ++nseg;
     }
+    // the kernel's cursor visits the same segments, each tile once, whether it steps by tile
+    // (producers, issuers) or by segment (softmax groups)
+    SliceCursor w;
+    w.start(t0, t1, prefix.data(), batch, hkv);
+    std::vector<char> seen((size_t)(t1 - t0), 0);
+    int wseg = 0;
+    while (!w.done()) {
+      const Segment s = w.sg;
+      if (w.seg_idx != wseg || w.j != 0) return 16;
+      const Segment lin = segment_at(s.item_begin + s.tile0, t1, prefix.data(), batch, hkv);
+      if (lin.item != s.item || lin.tile0 != s.tile0 || lin.n_tiles != s.n_tiles) return 17;   // a segment of the linear walk
+      for (int k = 0; k < s.n_tiles; ++k) {
+        const int64_t g = s.item_begin + s.tile0 + k;
+        if (g < t0 || g >= t1 || seen[(size_t)(g - t0)]) return 18;
+        seen[(size_t)(g - t0)] = 1;
+      }
+      // tile-wise stepping reaches the same next segment as segment-wise stepping
+      SliceCursor w2 = w;
+      for (int k = 0; k < s.n_tiles; ++k) {
+        if (w2.last_of_segment() != (k == s.n_tiles - 1)) return 19;
+        w2.next_tile(prefix.data(), batch, hkv);
+      }
+      w.next_segment(prefix.data(), batch, hkv);
+      if (w2.done() != w.done() || w2.seg_idx != w.seg_idx) return 20;
+      if (!w.done() && (w2.sg.item != w.sg.item || w2.sg.tile0 != w.sg.tile0 || w2.f != w.f)) return 21;
+      ++wseg;
+    }
+    if (wseg != nseg) return 22;
+    for (char v : seen)
+      if (!v) return 23;
   }
   for (int it = 0; it < n_items; ++it) {
     const int b = (it / hkv) % batch;
