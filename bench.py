@@ -366,9 +366,11 @@ def run_ours(args, rank, world):
     extra["select_random_us"] = timed(lambda: specvlm.select_baseline(specvlm.SEL_RANDOM, [w.n_frames[0]],
                                                                       w.tokens_per_frame, [path.kt], [0, path.kt],
                                                                       seed=1, device=device))
-    n_nodes = 128 // (w.t_q_heads // w.t_kv_heads)              # the widest tree one 128-row tile holds
-    n_tree = nv + nt + n_nodes
-    if n_tree <= inp["tcache"].max_seq_len + n_nodes:
+    # tree drafting: the widest tree one 128-row launch holds (16 nodes at 8 query heads per KV head),
+    # and a 26-node static tree (root + 25 candidates, the size of the static draft tree the paper
+    # adopts; its shape here is a binary heap, the paper's figure being unavailable): 208 rows, two launches
+    for n_nodes in (128 // (w.t_q_heads // w.t_kv_heads), 26):
+        n_tree = nv + nt + n_nodes
         tk = synth.randn_bf16((w.t_layers, 1, w.t_kv_heads, n_tree, D), device, 1, "treeK")
         tcache = specvlm.KvCache(tk, tk, torch.tensor([n_tree], dtype=torch.int32, device=device), n_tree)
         q_tree = synth.randn_bf16((w.t_layers, 1, n_nodes, w.t_q_heads, D), device, 1, "treeQ")
@@ -378,11 +380,13 @@ def run_ours(args, rank, world):
                            dtype=torch.uint8, device=device)
         us = timed(lambda: specvlm.verify_tree_attn(tcache, q_tree, parents, path.scale, out=o_tree, ws=ws_t), reps=5)
         extra["verify_tree_%d_nodes_us" % n_nodes] = us
-        extra["verify_tree_kv_gbs"] = 2 * n_tree * w.t_kv_heads * D * 2 * w.t_layers / (us * 1e-6) / 1e9
+        extra["verify_tree_%d_nodes_kv_gbs_per_pass" % n_nodes] = (
+            2 * n_tree * w.t_kv_heads * D * 2 * w.t_layers * ((n_nodes * (w.t_q_heads // w.t_kv_heads) + 127) // 128)
+            / (us * 1e-6) / 1e9)
         lg = torch.randn((1, n_nodes, w.vocab), device=device)
         toks = torch.zeros((1, n_nodes), dtype=torch.int32, device=device)
-        extra["accept_tree_us"] = timed(lambda: specvlm.accept_tree(lg, toks, parents))
-        del tk, tcache, q_tree, o_tree, lg
+        extra["accept_tree_%d_nodes_us" % n_nodes] = timed(lambda: specvlm.accept_tree(lg, toks, parents))
+        del tk, tcache, q_tree, o_tree, lg, ws_t
     new_kv = synth.randn_bf16((w.t_layers, 1, gamma + 1, w.t_kv_heads, D), device, 2, "newKV")
     lens_keep = inp["tcache"].seq_lens.clone()
 

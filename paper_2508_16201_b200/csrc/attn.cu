@@ -446,7 +446,6 @@ static int32_t attn_common(const specvlm_kv_t* kv, const void* q, int32_t batch,
   const int group = n_q_heads / kv->n_kv_heads;
   if (group > 16 || n_q > 9) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   const int rows = group * n_q;
-  if (rows > 128) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (rows > kRows16Max)
     return attn_tc_launch(kv, q, batch, n_q_heads, n_q, sm_scale, out, lse, ws, ws_bytes, d_status, st, nullptr);
@@ -511,7 +510,8 @@ extern "C" size_t specvlm_attn_workspace_bytes(const specvlm_kv_t* kv, int32_t b
       n_q_heads % kv->n_kv_heads != 0 || kv->n_layers < 1 || kv->max_seq_len < 1)
     return 0;
   const int rows = (n_q_heads / kv->n_kv_heads) * (gamma + 1);
-  if (rows > kRows16Max) return rows <= 128 && batch <= kSchedMaxBatch ? attn_tc_ws_bytes(kv, batch, rows) : 0;
+  if (n_q_heads / kv->n_kv_heads > 16 || gamma > 8) return 0;
+  if (rows > kRows16Max) return batch <= kSchedMaxBatch ? attn_tc_ws_bytes(kv, batch, rows) : 0;
   return rows16_ws_bytes(kv, batch, rows);
 }
 
@@ -538,7 +538,7 @@ extern "C" size_t specvlm_verify_tree_workspace_bytes(const specvlm_kv_t* kv, in
       kv->n_kv_heads < 1 || n_q_heads % kv->n_kv_heads != 0 || kv->n_layers < 1 || kv->max_seq_len < 1)
     return 0;
   const int rows = (n_q_heads / kv->n_kv_heads) * n_nodes;
-  if (rows > 128) return 0;
+  if (n_q_heads / kv->n_kv_heads > 16) return 0;
   return attn_tc_ws_bytes(kv, batch, rows) + attn_tc_tree_extra_bytes(batch, n_nodes);
 }
 
@@ -551,7 +551,7 @@ extern "C" int32_t specvlm_verify_tree_attn(const specvlm_kv_t* kv, const void* 
   if (!q || !out || !parents || n_q_heads < 1 || n_nodes < 1 || !(sm_scale > 0.f)) return SPECVLM_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(out) || n_q_heads % kv->n_kv_heads != 0) return SPECVLM_ERR_INVALID_ARG;
   const int group = n_q_heads / kv->n_kv_heads;
-  if (group > 16 || n_nodes > 32 || group * n_nodes > 128) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  if (group > 16 || n_nodes > 32) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   return attn_tc_launch(kv, q, batch, n_q_heads, n_nodes, sm_scale, out, lse_or_null, ws, ws_bytes, d_status,
                         static_cast<cudaStream_t>(stream), parents);
 }

@@ -33,16 +33,17 @@
 namespace specvlm {
 
 struct AttnTcParams {
-  __nv_bfloat16* out;         // [L][B][n_q][Hq][D]
-  float* lse;                 // [L][B][n_q][Hq] or null
+  __nv_bfloat16* out;         // [L][B][n_win][Hq][D]
+  float* lse;                 // [L][B][n_win][Hq] or null
   float* ws_o;                // partial results: [2 * grid][rows][D], normalised
   float* ws_lse;              // [2 * grid][rows], log2 units
   int32_t* ws_cnt;            // [items] arrival counters, zero at launch
   const int32_t* block_table; // [B][max_blocks] or null
   const int32_t* seq_lens;    // [B]
   int32_t* d_status;
-  const uint32_t* anc;        // [B][n_q] ancestor masks of a draft tree, or null: the window is a chain
+  const uint32_t* anc;        // [B][n_win] ancestor masks of a draft tree, or null: the window is a chain
   int32_t batch, n_layers, n_q, n_q_heads, n_kv_heads, group, rows;
+  int32_t n_win, q0;          // tokens of the whole window; first window token of this launch (n_q of them)
   int32_t max_blocks, block_tokens, max_seq_len;
   float scale_log2;           // sm_scale * log2(e)
 };
@@ -281,7 +282,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           mbar_arrive_expect_tx(bar_q_full + 8 * qb, (uint32_t)p.rows * 128u * (D / 64));
 #pragma unroll
           for (int h = 0; h < D / 64; ++h)
-            tma_load_5d(q_sm + qb * Q_BYTES + h * (M * 128), &tm_q, bar_q_full + 8 * qb, h * 64, 0, 0, sg.g,
+            tma_load_5d(q_sm + qb * Q_BYTES + h * (M * 128), &tm_q, bar_q_full + 8 * qb, h * 64, 0, p.q0, sg.g,
                         sg.layer * p.batch + sg.b, policy_q);
         }
         const int n_sub_seq = (clamp_len(p.seq_lens[sg.b], p.max_seq_len) + kTileTokens - 1) / kTileTokens;
@@ -442,7 +443,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         for (int idx = st; idx < p.rows * (D / 8); idx += 256) {
           const int r = idx / (D / 8), c8 = idx - r * (D / 8);
           const int t = r / p.group, h = g * p.group + (r - t * p.group);
-          const size_t orow = ((size_t)lb * p.n_q + t) * p.n_q_heads + h;
+          const size_t orow = ((size_t)lb * p.n_win + p.q0 + t) * p.n_q_heads + h;
           *reinterpret_cast<uint4*>(p.out + orow * D + c8 * 8) = make_uint4(0, 0, 0, 0);
           if (p.lse && c8 == 0) p.lse[orow] = -INFINITY;
         }
@@ -470,7 +471,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       // 0..t for a chain, the token's ancestors and itself for a tree.  Rows no item uses see nothing.
       // (A used row always has its own bit set, so a zero mask also marks an unused row.)
       // The chain keeps the equivalent limit form: key tok is visible to token t when tok < lim.
-      const int win0 = kv_len - p.n_q;
+      const int win0 = kv_len - p.n_win;
       uint32_t vis[NH][2];
       int lim[NH][2];
       float m_used[NH][2], l_sum[NH][2];
@@ -481,9 +482,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           const int r = row0(h) + lr + 8 * e;
           const int t = r / p.group;
           if constexpr (TREE) {
-            vis[h][e] = r < p.rows ? __ldg(p.anc + (size_t)sg.b * p.n_q + t) : 0u;
+            vis[h][e] = r < p.rows ? __ldg(p.anc + (size_t)sg.b * p.n_win + p.q0 + t) : 0u;
           } else {
-            lim[h][e] = r < p.rows ? win0 + t + 1 : 0;
+            lim[h][e] = r < p.rows ? win0 + p.q0 + t + 1 : 0;
           }
           m_used[h][e] = -INFINITY;
           l_sum[h][e] = 0.f;
@@ -706,7 +707,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               }
             if (complete) {
               const int t = r / p.group, hq = sg.g * p.group + (r - t * p.group);
-              const size_t orow = ((size_t)lb * p.n_q + t) * p.n_q_heads + hq;
+              const size_t orow = ((size_t)lb * p.n_win + p.q0 + t) * p.n_q_heads + hq;
               __nv_bfloat16* dst = p.out + orow * D + cc * 64 + lc;
 #pragma unroll
               for (int jj = 0; jj < 8; ++jj)
@@ -814,7 +815,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               if (!on[u]) continue;
               const float invd = den[u] > 0.f ? 1.f / den[u] : 0.f;
               const int t = r[u] / p.group, hq = sg.g * p.group + (r[u] - t * p.group);
-              const size_t orow = ((size_t)lb * p.n_q + t) * p.n_q_heads + hq;
+              const size_t orow = ((size_t)lb * p.n_win + p.q0 + t) * p.n_q_heads + hq;
               uint2 packed;
               packed.x = pack_bf16x2(acc[u].x * invd, acc[u].y * invd);
               packed.y = pack_bf16x2(acc[u].z * invd, acc[u].w * invd);
@@ -858,15 +859,15 @@ size_t attn_tc_ws_bytes(const specvlm_kv_t* kv, int32_t batch, int rows) {
 }
 
 // Queries as a 5-D tensor (channel, head in group, query token, KV head, layer * batch + sequence):
-// the box (64 channels, group, n_q, 1, 1) is one item's rows in the order r = t * group + head.
-static int32_t encode_q_map(CUtensorMap* map, const void* q, int D, int group, int n_q, int n_kv_heads,
+// the box (64 channels, group, n_q, 1, 1) at token q0 is one item's rows of a launch, r = t * group + head.
+static int32_t encode_q_map(CUtensorMap* map, const void* q, int D, int group, int n_win, int n_q, int n_kv_heads,
                             int64_t lb) {
   encode_tiled_fn enc = get_encode_tiled();
   if (!enc) return SPECVLM_ERR_CUDA;
   const int hq = group * n_kv_heads;
-  const cuuint64_t dims[5] = {(cuuint64_t)D, (cuuint64_t)group, (cuuint64_t)n_q, (cuuint64_t)n_kv_heads, (cuuint64_t)lb};
+  const cuuint64_t dims[5] = {(cuuint64_t)D, (cuuint64_t)group, (cuuint64_t)n_win, (cuuint64_t)n_kv_heads, (cuuint64_t)lb};
   const cuuint64_t strides[4] = {(cuuint64_t)D * 2, (cuuint64_t)hq * D * 2, (cuuint64_t)group * D * 2,
-                                 (cuuint64_t)n_q * hq * D * 2};
+                                 (cuuint64_t)n_win * hq * D * 2};
   const cuuint32_t box[5] = {64u, (cuuint32_t)group, (cuuint32_t)n_q, 1u, 1u};
   const cuuint32_t estr[5] = {1u, 1u, 1u, 1u, 1u};
   CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(q), dims, strides, box, estr,
@@ -925,7 +926,7 @@ int32_t attn_tc_launch(const specvlm_kv_t* kv, const void* q, int32_t batch, int
                        cudaStream_t st, const int32_t* tree_parents) {
   const int group = n_q_heads / kv->n_kv_heads;
   const int rows = group * n_q;
-  if (rows > 128 || batch > kSchedMaxBatch) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  if (group > 16 || batch > kSchedMaxBatch) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   const int64_t items = (int64_t)kv->n_layers * batch * kv->n_kv_heads;
   if (items > 0x3fffffff) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) return SPECVLM_ERR_INVALID_ARG;
@@ -934,34 +935,37 @@ int32_t attn_tc_launch(const specvlm_kv_t* kv, const void* q, int32_t batch, int
     return SPECVLM_ERR_WORKSPACE_TOO_SMALL;
   if (tree_parents && n_q > 32) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   const int grid = tc_grid(kv, batch);
+  // A window of more than 128 rows is cut into launches of equal numbers of query tokens, each of
+  // which streams the K/V once more: the accumulators of one launch fill the tensor memory.
+  const int n_launch = (rows + 127) / 128;
+  const int q_per = (n_q + n_launch - 1) / n_launch;
+  if (q_per * group > 128) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
 
-  CUtensorMap tk, tv, tq;
+  CUtensorMap tk, tv;
   int32_t rc = encode_kv_map(&tk, kv, kv->k, kTileTokens);
   if (rc != SPECVLM_OK) return rc;
   rc = encode_kv_map(&tv, kv, kv->v, kTileTokens);
-  if (rc != SPECVLM_OK) return rc;
-  rc = encode_q_map(&tq, q, kv->head_dim, group, n_q, kv->n_kv_heads, (int64_t)kv->n_layers * batch);
   if (rc != SPECVLM_OK) return rc;
 
   AttnTcParams p;
   p.out = static_cast<__nv_bfloat16*>(out);
   p.lse = lse;
+  const int rows_max = q_per * group;
   uint8_t* w = static_cast<uint8_t*>(ws);
   p.ws_o = reinterpret_cast<float*>(w);
-  w += round_up((size_t)2 * grid * rows * kv->head_dim * sizeof(float), 256);
+  w += round_up((size_t)2 * grid * rows_max * kv->head_dim * sizeof(float), 256);
   p.ws_lse = reinterpret_cast<float*>(w);
-  w += round_up((size_t)2 * grid * rows * sizeof(float), 256);
+  w += round_up((size_t)2 * grid * rows_max * sizeof(float), 256);
   p.ws_cnt = reinterpret_cast<int32_t*>(w);
   p.block_table = kv->block_table;
   p.seq_lens = kv->seq_lens;
   p.d_status = d_status;
   p.batch = batch;
   p.n_layers = kv->n_layers;
-  p.n_q = n_q;
+  p.n_win = n_q;
   p.n_q_heads = n_q_heads;
   p.n_kv_heads = kv->n_kv_heads;
   p.group = group;
-  p.rows = rows;
   p.max_blocks = kv->max_blocks;
   p.block_tokens = kv->block_tokens;
   p.max_seq_len = kv->max_seq_len;
@@ -976,10 +980,22 @@ int32_t attn_tc_launch(const specvlm_kv_t* kv, const void* q, int32_t batch, int
     p.anc = anc;
   }
 
-  if (cudaMemsetAsync(p.ws_cnt, 0, (size_t)items * sizeof(int32_t), st) != cudaSuccess) return SPECVLM_ERR_CUDA;
-  if (kv->head_dim == 128)
-    return rows <= 64 ? launch_tc<128, 64>(tk, tv, tq, p, grid, st) : launch_tc<128, 128>(tk, tv, tq, p, grid, st);
-  return rows <= 64 ? launch_tc<64, 64>(tk, tv, tq, p, grid, st) : launch_tc<64, 128>(tk, tv, tq, p, grid, st);
+  for (int q0 = 0; q0 < n_q; q0 += q_per) {
+    p.q0 = q0;
+    p.n_q = n_q - q0 < q_per ? n_q - q0 : q_per;
+    p.rows = p.n_q * group;
+    CUtensorMap tq;
+    rc = encode_q_map(&tq, q, kv->head_dim, group, n_q, p.n_q, kv->n_kv_heads, (int64_t)kv->n_layers * batch);
+    if (rc != SPECVLM_OK) return rc;
+    // the launches share the scratch memory: stream order keeps them apart
+    if (cudaMemsetAsync(p.ws_cnt, 0, (size_t)items * sizeof(int32_t), st) != cudaSuccess) return SPECVLM_ERR_CUDA;
+    if (kv->head_dim == 128)
+      rc = p.rows <= 64 ? launch_tc<128, 64>(tk, tv, tq, p, grid, st) : launch_tc<128, 128>(tk, tv, tq, p, grid, st);
+    else
+      rc = p.rows <= 64 ? launch_tc<64, 64>(tk, tv, tq, p, grid, st) : launch_tc<64, 128>(tk, tv, tq, p, grid, st);
+    if (rc != SPECVLM_OK) return rc;
+  }
+  return SPECVLM_OK;
 }
 
 }  // namespace specvlm

@@ -140,6 +140,13 @@ def test_verify_row_counts(Hq, Hkv, gamma, D, paged):
     _run_attn(1, Hq, Hkv, D, [421], gamma, paged=paged, seed=8, splits=3)
 
 
+@pytest.mark.parametrize("paged", [False, True])
+def test_verify_window_wider_than_one_launch(paged):
+    # group 16 with gamma 8: 144 rows, cut into two launches of 5 and 4 query tokens
+    _run_attn(2, 32, 2, 128, [300, 64 + 9, 9], 8, paged=paged, seed=11, poison=True)
+    _run_attn(1, 16, 1, 64, [200], 8, paged=paged, seed=12)
+
+
 def test_verify_window_crossing_tile_boundary():
     # the gamma+1 new tokens straddle a 64-token tile edge, and sit alone in the last tile
     for n in [64 + 3, 128, 128 + 6, 6]:
@@ -327,7 +334,7 @@ def test_gather_bit_exact(src_paged, dst_paged):
 
 
 # ------------------------------------------------------------------------------- scores
-def _scores_case(L, Hq, Hkv, D, n_frames, T, n_text, *, paged, seed, prefix=None, planted=50):
+def _scores_case(L, Hq, Hkv, D, n_frames, T, n_text, *, paged, seed, prefix=None, planted=50, scale_mul=1.0):
     from gpu_util import make_cache
     B = len(n_frames)
     prefix = prefix or [0] * B
@@ -349,7 +356,7 @@ def _scores_case(L, Hq, Hkv, D, n_frames, T, n_text, *, paged, seed, prefix=None
             synth.plant_salient_(kview, q[:, text_cu[b]:text_cu[b + 1]], sal)
         from gpu_util import host_view
         k_host = host_view(cache.k, None, seq_lens)
-    scale = 1.0 / math.sqrt(D)
+    scale = scale_mul / math.sqrt(D)
     text_start = [p + v for p, v in zip(prefix, nv)]
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     got = specvlm.stage1_scores(cache, q, text_cu, text_start, prefix, nv, video_cu, scale, d_status=status)
@@ -364,7 +371,7 @@ def _scores_case(L, Hq, Hkv, D, n_frames, T, n_text, *, paged, seed, prefix=None
         ref = oracle.stage1_scores(qh[:, text_cu[b]:text_cu[b + 1]], k_host[b], prefix[b], nv[b],
                                    text_start[b], scale)
         g = got[video_cu[b]:video_cu[b + 1]]
-        rel = np.abs(g - ref) / ref
+        rel = np.abs(g - ref) / np.maximum(ref, 1e-30)     # scores below fp32's range compare absolutely
         worst = max(worst, float(rel.max()))
     assert worst <= SCORE_TOL, f"scores rel err {worst}"
     return got
@@ -379,6 +386,15 @@ def test_scores_cfg1():
 def test_scores_group_sizes(Hq, Hkv, D):
     _scores_case(2, Hq, Hkv, D, [3], 100, [37], paged=False, seed=1)
     _scores_case(1, Hq, Hkv, D, [2], 77, [130], paged=True, seed=2, prefix=[9])
+
+
+def test_scores_sharp_softmax():
+    """Logits 12 times wider than usual: the smallest exponentials of a row lie more than 2^125 below
+    its maximum, where the polynomial exponential saturates and the special-function one flushes to
+    zero; neither may disturb a row's sum or a column's score."""
+    got = _scores_case(2, 16, 4, 128, [3], 100, [37], paged=False, seed=7, scale_mul=12.0)
+    assert np.isfinite(got).all() and (got >= 0).all() and got.sum() <= 1.0 + 1e-6
+    _scores_case(1, 8, 8, 64, [2], 130, [5], paged=True, seed=8, scale_mul=12.0)
 
 
 def test_scores_ragged_batch():
