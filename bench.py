@@ -623,6 +623,20 @@ def run_case(args):
         "gather": (lambda: path.gather_call(inp["dpruned"][0]), 4 * (w.k_total() + nt) * w.d_kv_heads * D * 2 * w.d_layers),
         "accept": (path.accept_call, (gamma + 1) * w.vocab * 4),
     }
+    if args.case == "verify_tree":
+        # a heap-shaped draft tree of --nodes nodes behind the prompt (128 rows per launch at most)
+        n_nodes = args.nodes
+        n_tree = nv + nt + n_nodes
+        tk = synth.randn_bf16((w.t_layers, 1, w.t_kv_heads, n_tree, D), device, 1, "treeK")
+        tcache = specvlm.KvCache(tk, tk, torch.tensor([n_tree], dtype=torch.int32, device=device), n_tree)
+        q_tree = synth.randn_bf16((w.t_layers, 1, n_nodes, w.t_q_heads, D), device, 1, "treeQ")
+        parents = torch.tensor([[-1] + [(t - 1) // 2 for t in range(1, n_nodes)]], dtype=torch.int32, device=device)
+        o_tree = torch.empty_like(q_tree)
+        ws_t = torch.empty(specvlm.lib().specvlm_verify_tree_workspace_bytes(ctypes_byref(tcache), 1, w.t_q_heads, n_nodes),
+                           dtype=torch.uint8, device=device)
+        passes = (n_nodes * (w.t_q_heads // w.t_kv_heads) + 127) // 128
+        calls["verify_tree"] = (lambda: specvlm.verify_tree_attn(tcache, q_tree, parents, path.scale, out=o_tree, ws=ws_t),
+                                passes * 2 * n_tree * w.t_kv_heads * D * 2 * w.t_layers)
     fn, nbytes = calls[args.case]
     ts = []
     for i in range(args.warmup + args.iters):
@@ -650,6 +664,7 @@ def main():
     ap.add_argument("--frames", type=int, default=0)
     ap.add_argument("--workload", type=int, default=2)
     ap.add_argument("--gamma", type=int, default=None)
+    ap.add_argument("--nodes", type=int, default=16, help="draft-tree nodes of --case verify_tree")
     ap.add_argument("--iters", type=int, default=10)
     ap.add_argument("--flush", action="store_true", help="write a 512 MB buffer before each launch")
     ap.add_argument("--gpus", type=int, default=1)

@@ -101,6 +101,69 @@ __device__ __forceinline__ float4 ldg_cg_f32x4(const float* p) {
 
 __device__ __forceinline__ int clamp_len(int n, int max_len) { return n < 0 ? 0 : (n > max_len ? max_len : n); }
 
+// Cold paths of the softmax loop, kept out of line: the loop's code has to stay small enough for
+// the instruction cache (with the mask logic inline the 128-row variant ran 25 % slower, although
+// only one or two tiles of an item ever need a mask).
+//
+// Tiles that overlap the window of new tokens: the invisible logits of this thread's two rows
+// (a 16-lane half of S: rows lr and lr + 8, columns 8j + lc + {0, 1} of each 64-column block) are
+// overwritten with -inf in tensor memory, so the loop itself knows no masks.  Visibility of key
+// `tok` for the row of query token t: every key before the window, and inside the window the
+// positions whose bit is set in the row's mask -- the token's ancestors and itself for a tree
+// (a0, a1 = the rows' masks), positions up to t for a chain (a0, a1 = the rows' limits `lim`:
+// key tok is visible when tok < lim).
+template <bool TREE>
+__device__ __noinline__ void mask_s_half(uint32_t saddr, int tile_tok0, int win0, int lc, uint32_t a0, uint32_t a1) {
+  const uint32_t a[2] = {a0, a1};
+#pragma unroll 1
+  for (int c = 0; c < 2; ++c) {
+    uint64_t mk[2];
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      if constexpr (TREE) {
+        // 128 visibility bits of the tile: the keys before the window, then the row's window mask
+        // at the window's offset in the tile
+        const int sh = win0 - tile_tok0;                       // tile column of window position 0
+        unsigned __int128 full = 0;
+        if (a[e]) {
+          if (sh > 0) full = sh >= 128 ? ~(unsigned __int128)0 : (((unsigned __int128)1 << sh) - 1);
+          const unsigned __int128 w = a[e];
+          full |= sh >= 0 ? (sh < 128 ? w << sh : (unsigned __int128)0)
+                          : (sh > -32 ? w >> (-sh) : (unsigned __int128)0);
+        }
+        mk[e] = (uint64_t)(full >> (64 * c)) >> lc;
+      } else {
+        const int n_vis = (int)a[e] - tile_tok0 - 64 * c;       // visible columns of the block
+        mk[e] = (n_vis <= 0 ? 0ull : (n_vis >= 64 ? ~0ull : ((1ull << n_vis) - 1ull))) >> lc;
+      }
+    }
+    uint32_t v[32];
+    tmem_ld_16x256b_x8(saddr + 64 * c, v);
+    tmem_ld_wait();
+#pragma unroll
+    for (int k = 0; k < 32; ++k)
+      if (!((mk[(k >> 1) & 1] >> ((k >> 2) * 8 + (k & 1))) & 1ull)) v[k] = 0xff800000u;   // -inf
+    tmem_st_16x256b_x8(saddr + 64 * c, v);
+  }
+  tmem_st_wait();
+}
+
+// A row maximum grew past the lazy-rescale threshold: the rows' O accumulators (16-lane half,
+// d columns from oaddr on) are multiplied by f0 (row lr) and f1 (row lr + 8) in tensor memory.
+template <int D>
+__device__ __noinline__ void rescale_o_half(uint32_t oaddr, float f0, float f1) {
+#pragma unroll 1
+  for (int cc = 0; cc < D / 64; ++cc) {
+    uint32_t o[32];
+    tmem_ld_16x256b_x8(oaddr + cc * 64, o);
+    tmem_ld_wait();
+#pragma unroll
+    for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * (((k >> 1) & 1) ? f1 : f0));
+    tmem_st_16x256b_x8(oaddr + cc * 64, o);
+  }
+  tmem_st_wait();
+}
+
 // Shared-memory plan.  A small region (barriers, flags, per-sequence tile counts, the softmax
 // groups' row statistics) sits at the start of the dynamic shared memory; the tile rings and the
 // operand tiles follow at the next 1024-byte boundary.
@@ -507,28 +570,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           // same (rolled) code: once for the row maxima, once for the probabilities.  That halves
           // the live registers and the code of the loop; a TMEM load costs far less than the spills.
           const uint32_t saddr = tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + C::COL_S + grp * kBigTokens;
-          // visibility of this thread's columns of chunk c, when the tile needs masking
-          auto chunk_mask = [&](int c, uint64_t (&mk)[2]) {
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-              if constexpr (TREE) {
-                // 128 visibility bits of the tile: the keys before the window, then the row's window
-                // mask at the window's offset in the tile
-                const int sh = win0 - tile_tok0;                       // tile column of window position 0
-                unsigned __int128 full = 0;
-                if (vis[h][e]) {
-                  if (sh > 0) full = sh >= 128 ? ~(unsigned __int128)0 : (((unsigned __int128)1 << sh) - 1);
-                  const unsigned __int128 w = vis[h][e];
-                  full |= sh >= 0 ? (sh < 128 ? w << sh : (unsigned __int128)0)
-                                  : (sh > -32 ? w >> (-sh) : (unsigned __int128)0);
-                }
-                mk[e] = (uint64_t)(full >> (64 * c)) >> lc;
-              } else {
-                const int n_vis = lim[h][e] - tile_tok0 - 64 * c;       // visible columns of the chunk
-                mk[e] = (n_vis <= 0 ? 0ull : (n_vis >= 64 ? ~0ull : ((1ull << n_vis) - 1ull))) >> lc;
-              }
-            }
-          };
+          if (__builtin_expect(need_mask, 0)) {
+            if constexpr (TREE) mask_s_half<true>(saddr, tile_tok0, win0, lc, vis[h][0], vis[h][1]);
+            else mask_s_half<false>(saddr, tile_tok0, win0, lc, (uint32_t)lim[h][0], (uint32_t)lim[h][1]);
+          }
           float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll 1
           for (int c = 0; c < 2; ++c) {
@@ -536,16 +581,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             tmem_ld_16x256b_x8(saddr + 64 * c, v);
             tmem_ld_wait();
             float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-            if (__builtin_expect(need_mask, 0)) {
-              uint64_t mk[2];
-              chunk_mask(c, mk);
 #pragma unroll
-              for (int k = 0; k < 32; ++k)
-                if ((mk[(k >> 1) & 1] >> ((k >> 2) * 8 + (k & 1))) & 1ull) mx[k & 3] = fmaxf(mx[k & 3], __uint_as_float(v[k]));
-            } else {
-#pragma unroll
-              for (int k = 0; k < 32; ++k) mx[k & 3] = fmaxf(mx[k & 3], __uint_as_float(v[k]));
-            }
+            for (int k = 0; k < 32; ++k) mx[k & 3] = fmaxf(mx[k & 3], __uint_as_float(v[k]));
             mx0 = fmaxf(mx0, fmaxf(mx[0], mx[1]));
             mx1 = fmaxf(mx1, fmaxf(mx[2], mx[3]));
           }
@@ -572,18 +609,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               l_sum[h][0] *= a0;
               l_sum[h][1] *= a1;
               tc_fence_after_sync();
-#pragma unroll 1
-              for (int cc = 0; cc < D / 64; ++cc) {
-                uint32_t o[32];
-                const uint32_t oaddr = tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + C::COL_O + grp * D + cc * 64;
-                tmem_ld_16x256b_x8(oaddr, o);
-                tmem_ld_wait();
-#pragma unroll
-                for (int k = 0; k < 32; ++k)
-                  o[k] = __float_as_uint(__uint_as_float(o[k]) * (((k >> 1) & 1) ? a1 : a0));
-                tmem_st_16x256b_x8(oaddr, o);
-              }
-              tmem_st_wait();
+              rescale_o_half<D>(tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + C::COL_O + grp * D, a0, a1);
               tc_fence_before_sync();
             }
           }
@@ -604,13 +630,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               tc_fence_before_sync();
               __syncwarp();
               if (lane == 0) mbar_arrive(bar_s_empty + 8 * grp);
-            }
-            if (__builtin_expect(need_mask, 0)) {
-              uint64_t mk[2];
-              chunk_mask(c, mk);
-#pragma unroll
-              for (int k = 0; k < 32; ++k)
-                if (!((mk[(k >> 1) & 1] >> ((k >> 2) * 8 + (k & 1))) & 1ull)) v[k] = 0xff800000u;   // -inf
             }
 #pragma unroll
             for (int jj = 0; jj < 8; ++jj) {
