@@ -563,16 +563,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           __syncwarp();
           if (lane == 0) mbar_arrive(bar_s_empty + 8 * grp);
         }
-#pragma unroll
-        for (int h = 0; h < NH; ++h) {
-          if (h >= nh) break;
+        // One copy of the code serves both 16-row halves of a warp (the 128-row variant): the loop is
+        // rolled, the current half's state sits at index 0 of its arrays, and the two halves' states
+        // change places after each half -- twice per tile, so every tile finds them as it left them.
+#pragma unroll 1
+        for (int h = 0; h < nh; ++h) {
           // The half's 16 rows x 128 columns are read from TMEM twice, 64 columns at a time, by the
           // same (rolled) code: once for the row maxima, once for the probabilities.  That halves
           // the live registers and the code of the loop; a TMEM load costs far less than the spills.
           const uint32_t saddr = tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + C::COL_S + grp * kBigTokens;
           if (__builtin_expect(need_mask, 0)) {
-            if constexpr (TREE) mask_s_half<true>(saddr, tile_tok0, win0, lc, vis[h][0], vis[h][1]);
-            else mask_s_half<false>(saddr, tile_tok0, win0, lc, (uint32_t)lim[h][0], (uint32_t)lim[h][1]);
+            if constexpr (TREE) mask_s_half<true>(saddr, tile_tok0, win0, lc, vis[0][0], vis[0][1]);
+            else mask_s_half<false>(saddr, tile_tok0, win0, lc, (uint32_t)lim[0][0], (uint32_t)lim[0][1]);
           }
           float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll 1
@@ -596,26 +598,26 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           if (h == 0 && i >= 2) SM_WAIT(bar_p_empty + 8 * grp, ((i >> 1) - 1) & 1);
           if (j < 2) {
             // the group's first tile of the item: O is overwritten by this tile's product
-            m_used[h][0] = mx0;
-            m_used[h][1] = mx1;
+            m_used[0][0] = mx0;
+            m_used[0][1] = mx1;
           } else {
-            const bool up0 = mx0 > m_used[h][0] + kRescaleThreshold, up1 = mx1 > m_used[h][1] + kRescaleThreshold;
+            const bool up0 = mx0 > m_used[0][0] + kRescaleThreshold, up1 = mx1 > m_used[0][1] + kRescaleThreshold;
             if (__builtin_expect(__any_sync(0xffffffffu, up0 || up1) != 0, 0)) {
               // raise the reference maximum of those rows and rescale their O rows in TMEM
-              const float a0 = up0 ? fast_exp2(m_used[h][0] - mx0) : 1.f;
-              const float a1 = up1 ? fast_exp2(m_used[h][1] - mx1) : 1.f;
-              if (up0) m_used[h][0] = mx0;
-              if (up1) m_used[h][1] = mx1;
-              l_sum[h][0] *= a0;
-              l_sum[h][1] *= a1;
+              const float a0 = up0 ? fast_exp2(m_used[0][0] - mx0) : 1.f;
+              const float a1 = up1 ? fast_exp2(m_used[0][1] - mx1) : 1.f;
+              if (up0) m_used[0][0] = mx0;
+              if (up1) m_used[0][1] = mx1;
+              l_sum[0][0] *= a0;
+              l_sum[0][1] *= a1;
               tc_fence_after_sync();
               rescale_o_half<D>(tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + C::COL_O + grp * D, a0, a1);
               tc_fence_before_sync();
             }
           }
           // probabilities: p = 2^(s * scale - m), with a row that sees nothing yet kept at zero
-          const float nmu0 = m_used[h][0] == -INFINITY ? 0.f : -m_used[h][0];
-          const float nmu1 = m_used[h][1] == -INFINITY ? 0.f : -m_used[h][1];
+          const float nmu0 = m_used[0][0] == -INFINITY ? 0.f : -m_used[0][0];
+          const float nmu1 = m_used[0][1] == -INFINITY ? 0.f : -m_used[0][1];
           float ps[4] = {0.f, 0.f, 0.f, 0.f};
           // rows of the A operand of O += P V: the item's rows
           const int m0 = row0(h) + lr, m1 = m0 + 8;
@@ -645,8 +647,27 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                            "r"(pack_bf16x2(p2, p3)) : "memory");
             }
           }
-          l_sum[h][0] += ps[0] + ps[1];
-          l_sum[h][1] += ps[2] + ps[3];
+          l_sum[0][0] += ps[0] + ps[1];
+          l_sum[0][1] += ps[2] + ps[3];
+          if (NH == 2 && nh == 2) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const float tm = m_used[0][e], tl = l_sum[0][e];
+              m_used[0][e] = m_used[NH - 1][e];
+              m_used[NH - 1][e] = tm;
+              l_sum[0][e] = l_sum[NH - 1][e];
+              l_sum[NH - 1][e] = tl;
+              if constexpr (TREE) {
+                const uint32_t tv = vis[0][e];
+                vis[0][e] = vis[NH - 1][e];
+                vis[NH - 1][e] = tv;
+              } else {
+                const int tv = lim[0][e];
+                lim[0][e] = lim[NH - 1][e];
+                lim[NH - 1][e] = tv;
+              }
+            }
+          }
         }
         if (nh == 0 && i >= 2) SM_WAIT(bar_p_empty + 8 * grp, ((i >> 1) - 1) & 1);
         fence_proxy_async();
