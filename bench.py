@@ -372,7 +372,8 @@ def run_ours(args, rank, world):
     for n_nodes in (128 // (w.t_q_heads // w.t_kv_heads), 26):
         n_tree = nv + nt + n_nodes
         tk = synth.randn_bf16((w.t_layers, 1, w.t_kv_heads, n_tree, D), device, 1, "treeK")
-        tcache = specvlm.KvCache(tk, tk, torch.tensor([n_tree], dtype=torch.int32, device=device), n_tree)
+        tv = synth.randn_bf16((w.t_layers, 1, w.t_kv_heads, n_tree, D), device, 1, "treeV")
+        tcache = specvlm.KvCache(tk, tv, torch.tensor([n_tree], dtype=torch.int32, device=device), n_tree)
         q_tree = synth.randn_bf16((w.t_layers, 1, n_nodes, w.t_q_heads, D), device, 1, "treeQ")
         parents = torch.tensor([[-1] + [(t - 1) // 2 for t in range(1, n_nodes)]], dtype=torch.int32, device=device)
         o_tree = torch.empty_like(q_tree)
@@ -386,7 +387,7 @@ def run_ours(args, rank, world):
         lg = torch.randn((1, n_nodes, w.vocab), device=device)
         toks = torch.zeros((1, n_nodes), dtype=torch.int32, device=device)
         extra["accept_tree_%d_nodes_us" % n_nodes] = timed(lambda: specvlm.accept_tree(lg, toks, parents))
-        del tk, tcache, q_tree, o_tree, lg, ws_t
+        del tk, tv, tcache, q_tree, o_tree, lg, ws_t
     new_kv = synth.randn_bf16((w.t_layers, 1, gamma + 1, w.t_kv_heads, D), device, 2, "newKV")
     lens_keep = inp["tcache"].seq_lens.clone()
 
@@ -628,7 +629,8 @@ def run_case(args):
         n_nodes = args.nodes
         n_tree = nv + nt + n_nodes
         tk = synth.randn_bf16((w.t_layers, 1, w.t_kv_heads, n_tree, D), device, 1, "treeK")
-        tcache = specvlm.KvCache(tk, tk, torch.tensor([n_tree], dtype=torch.int32, device=device), n_tree)
+        tv = synth.randn_bf16((w.t_layers, 1, w.t_kv_heads, n_tree, D), device, 1, "treeV")
+        tcache = specvlm.KvCache(tk, tv, torch.tensor([n_tree], dtype=torch.int32, device=device), n_tree)
         q_tree = synth.randn_bf16((w.t_layers, 1, n_nodes, w.t_q_heads, D), device, 1, "treeQ")
         parents = torch.tensor([[-1] + [(t - 1) // 2 for t in range(1, n_nodes)]], dtype=torch.int32, device=device)
         o_tree = torch.empty_like(q_tree)
