@@ -152,18 +152,47 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const __grid_con
           }
         }
         __syncthreads();
-        if (tid == 0) {
-          int d = 255;
-          unsigned long long acc = above;
-          int n = n_above;
-          for (; d > 0; --d) {
-            if (1000ull * (acc + mass[d]) >= target) break;
-            acc += mass[d];
-            n += hist[d];
+        // Scanning the digits from 255 down, the first one whose keys bring the mass up to the target
+        // (digit 0 if none does).  Warp 0 does it: lane l owns digits 8l .. 8l+7, a shuffle scan
+        // gives the mass and the count above each lane's digits, and the one lane whose digits
+        // contain the crossing walks its eight.
+        if (tid < 32) {
+          unsigned long long hm[8], sm = 0ull;
+          int hc[8], sc = 0;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            hm[i] = mass[8 * tid + i];
+            hc[i] = hist[8 * tid + i];
+            sm += hm[i];
+            sc += hc[i];
           }
-          misc[0] = d;
-          misc[1] = n;
-          mass[257] = acc;
+          unsigned long long am = sm;
+          int ac = sc;
+#pragma unroll
+          for (int off = 1; off < 32; off <<= 1) {
+            const unsigned long long vm = __shfl_down_sync(0xffffffffu, am, off);
+            const int vc = __shfl_down_sync(0xffffffffu, ac, off);
+            if (tid + off < 32) {
+              am += vm;
+              ac += vc;
+            }
+          }
+          unsigned long long acc = above + (am - sm);      // mass of the live keys with larger digits
+          int n = n_above + (ac - sc);
+          const bool crosses = 1000ull * acc < target && 1000ull * (acc + sm) >= target;
+          const unsigned any = __ballot_sync(0xffffffffu, crosses);
+          if (crosses || (any == 0u && tid == 0)) {
+            int d = 8 * tid + 7;
+#pragma unroll
+            for (int i = 7; i >= 0; --i, --d) {
+              if (d == 0 || 1000ull * (acc + hm[i]) >= target) break;
+              acc += hm[i];
+              n += hc[i];
+            }
+            misc[0] = d;
+            misc[1] = n;
+            mass[257] = acc;
+          }
         }
         __syncthreads();
         pfx |= static_cast<uint32_t>(misc[0]) << shift;
@@ -198,14 +227,34 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const __grid_con
         if (live && (tid & 31) == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
       }
       __syncthreads();
-      if (tid == 0) {
-        int acc = 0, d = 255;
-        for (; d > 0; --d) {
-          if (acc + hist[d] >= k_rem) break;
-          acc += hist[d];
+      // Scanning the digits from 255 down, the first one that brings the count up to k_rem (digit 0
+      // if none does): warp 0, lane l owning digits 8l .. 8l+7, as in the Top-P descent above.
+      if (tid < 32) {
+        int hc[8], sc = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          hc[i] = hist[8 * tid + i];
+          sc += hc[i];
         }
-        misc[0] = d;                   // digit of the k_rem-th largest live key
-        misc[1] = k_rem - acc;         // wanted among the keys with that digit
+        int ac = sc;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const int vc = __shfl_down_sync(0xffffffffu, ac, off);
+          if (tid + off < 32) ac += vc;
+        }
+        int acc = ac - sc;             // live keys with larger digits
+        const bool crosses = acc < k_rem && acc + sc >= k_rem;
+        const unsigned any = __ballot_sync(0xffffffffu, crosses);
+        if (crosses || (any == 0u && tid == 0)) {
+          int d = 8 * tid + 7;
+#pragma unroll
+          for (int i = 7; i >= 0; --i, --d) {
+            if (d == 0 || acc + hc[i] >= k_rem) break;
+            acc += hc[i];
+          }
+          misc[0] = d;                 // digit of the k_rem-th largest live key
+          misc[1] = k_rem - acc;       // wanted among the keys with that digit
+        }
       }
       __syncthreads();
       prefix |= static_cast<uint32_t>(misc[0]) << shift;
