@@ -300,19 +300,21 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const __grid_con
   }
   __syncthreads();
   // ---- 3. Stage II pick test, then compaction
-  const long long n_u = k_total - k1;
+  // All products below stay under 2^32: counts are at most n_v <= 57 344 tokens (the shared-memory
+  // limit), so 32-bit unsigned division is exact here -- and keeps this kernel's code small.
+  const uint32_t n_u = (uint32_t)(k_total - k1);
   int n_keep = 0;
   {
     int run = e;
     for (int j = j_lo; j < j_hi; ++j) {
       if (key[j] == 0u) {
         const int f = j / T;
-        const int c0 = cf[f], c1 = cf[f + 1];
-        const int c_f = c1 - c0;
-        const int rank = run - c0;
-        const int n_f = static_cast<int>((c1 * n_u) / m_total - (c0 * n_u) / m_total);
-        if (n_f > 0) {
-          const long long t = ((long long)rank * n_f + c_f - 1) / c_f;
+        const uint32_t c0 = (uint32_t)cf[f], c1 = (uint32_t)cf[f + 1];
+        const uint32_t c_f = c1 - c0;
+        const uint32_t rank = (uint32_t)run - c0;
+        const uint32_t n_f = (c1 * n_u) / (uint32_t)m_total - (c0 * n_u) / (uint32_t)m_total;
+        if (n_f > 0u) {
+          const uint32_t t = (rank * n_f + c_f - 1u) / c_f;
           if (t < n_f && (t * c_f) / n_f == rank) key[j] = 2u;
         }
         ++run;
