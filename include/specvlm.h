@@ -208,6 +208,9 @@ int32_t specvlm_gather_kv(const specvlm_kv_t* src, const int32_t* kept_idx, cons
  *   lse_or_null device fp32 [n_layers][batch][n_q][n_q_heads]: natural-log sum-exp of the logits
  *   ws          device scratch, specvlm_attn_workspace_bytes(kv, batch, n_q_heads, gamma)
  * fp32 softmax and accumulation; probabilities are rounded to bf16 before the PV product.
+ * Stream order: the decode kernel (windows of at most 16 rows) is launched with programmatic stream
+ * serialization; it may begin while the kernel before it on the stream is still running, and
+ * touches no global memory until that kernel's writes are complete and visible.
  * Supported: head_dim 64/128; group = n_q_heads/n_kv_heads in 1..16; 0 <= gamma <= 8;
  * batch <= 127 when group * (gamma+1) > 16.  A window of more than 128 rows (group * (gamma+1))
  * runs as several launches of at most 128 rows, each reading the cache once.

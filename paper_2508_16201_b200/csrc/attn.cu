@@ -43,12 +43,6 @@ attn_rows16_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
   const int split = blockIdx.x, g = blockIdx.y, lb = blockIdx.z;
   const int layer = lb / p.batch, b = lb - layer * p.batch;
 
-  int kv_len = p.seq_lens[b];
-  kv_len = kv_len < 0 ? 0 : (kv_len > p.max_seq_len ? p.max_seq_len : kv_len);
-  int tile_begin, tile_end;
-  split_range(kv_len, p.n_splits, split, tile_begin, tile_end);
-  const int n_my = tile_end - tile_begin;
-
   if (tid == 0) {
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(bar_full + 8 * s, 1);
@@ -57,6 +51,18 @@ attn_rows16_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     *abort_flag = 0;
     mbar_fence_init();
   }
+  // Programmatic dependent launch: the kernel is launched so that it may start while the kernel
+  // before it in the stream is still running.  Everything above touches no global memory; the
+  // wait below returns once that kernel's memory operations are complete and visible.  The kernel
+  // after this one may be scheduled as soon as every CTA here has got this far.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  int kv_len = p.seq_lens[b];
+  kv_len = kv_len < 0 ? 0 : (kv_len > p.max_seq_len ? p.max_seq_len : kv_len);
+  int tile_begin, tile_end;
+  split_range(kv_len, p.n_splits, split, tile_begin, tile_end);
+  const int n_my = tile_end - tile_begin;
   __syncthreads();
 
   if (warp == 4 * NG) {
@@ -419,7 +425,18 @@ static int32_t launch_rows16_s(const CUtensorMap& tk, const CUtensorMap& tv, con
   auto kern = attn_rows16_kernel<D, STAGES, NG>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
     return SPECVLM_ERR_CUDA;
-  kern<<<grid, 32 * (4 * NG + 1), SMEM, st>>>(tk, tv, p);
+  // launched with programmatic stream serialization: see the kernel's griddepcontrol.wait
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(32 * (4 * NG + 1), 1, 1);
+  cfg.dynamicSmemBytes = SMEM;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, kern, tk, tv, p) != cudaSuccess) return SPECVLM_ERR_CUDA;
   return launch_status();
 }
 
