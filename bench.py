@@ -49,9 +49,9 @@ def measured_peaks():
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
 # summarised under profiles/; None where no capture of that launch exists.  Each capture ran a
 # subset of the layers (the capture-size rule) and is scaled to the layers one launch processes:
-# traffic is proportional to the layers streamed.  verify: 215.8 MB for 8 of 80 layers; rating
-# passes: 156.4 MB and 153.1 MB for 10 of 80 layers.
-NCU_TRAFFIC_BYTES = {"verify": 215.8e6 * 10, "decode": None, "scores_colsum": 153.1e6 * 8, "scores_lse": 156.4e6 * 8}
+# traffic is proportional to the layers streamed.  verify: 216.0 MB for 8 of 80 layers; rating
+# passes: 156.5 MB and 153.2 MB for 10 of 80 layers; decode: 43.5 MB, captured whole.
+NCU_TRAFFIC_BYTES = {"verify": 216.0e6 * 10, "decode": 43.5e6, "scores_colsum": 153.2e6 * 8, "scores_lse": 156.5e6 * 8}
 
 
 class ClockSampler:
