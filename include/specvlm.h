@@ -340,6 +340,15 @@ int32_t specvlm_accept_noalloc(const float* target_logits, const int32_t* draft_
                                int32_t gamma, int32_t vocab, int32_t* accept_len,
                                int32_t* next_token, int32_t* target_argmax_or_null, void* stream);
 
+/*
+ * Diagnostic for tests; the paper has no counterpart.  Launches a kernel on `stream` that fills
+ * the shared memory of the SMs with NaN bit patterns (0xffffffff words).  Shared memory keeps its
+ * contents from one kernel to the next, so a kernel that reads a word it never wrote usually
+ * sees something harmless and a test passes by luck; after this call it sees NaNs.  Computes
+ * nothing, allocates nothing, touches no global memory.
+ */
+int32_t specvlm_debug_poison_shared_memory(void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -546,6 +546,20 @@ scores_colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
     *abort_flag = 0;
     mbar_fence_init();
   }
+  {
+    // A row tile holds qt * group rows; the TMA box never writes the rows after them, and whatever
+    // the shared memory held there would reach every key's sum through the product (a NaN times a
+    // vanishing weight is still a NaN).  They are cleared once: row r of a tile is the 128 bytes at
+    // r * 128 of each 64-channel block, whatever the swizzle does inside a row.
+    const int rows_used = p.qt * p.group;
+    const int n16 = (kKeyTile - rows_used) * 8;                    // 16-byte units per block
+    for (int i = tid; i < STAGES * (D / 64) * n16; i += blockDim.x) {
+      const int blk = i / n16, u = i - blk * n16;
+      *reinterpret_cast<uint4*>(smem + 2 * TILE_BYTES + blk * (kKeyTile * 128) + rows_used * 128 + u * 16) =
+          make_uint4(0u, 0u, 0u, 0u);
+    }
+    fence_proxy_async();                                           // the MMAs read it through the async proxy
+  }
   if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
   tc_fence_before_sync();
   __syncthreads();

@@ -53,7 +53,7 @@ EXPORTS = [
     "specvlm_accept_workspace_bytes", "specvlm_accept", "specvlm_accept_noalloc",
     "specvlm_append_kv", "specvlm_rollback_kv",
     "specvlm_verify_tree_workspace_bytes", "specvlm_verify_tree_attn", "specvlm_accept_tree",
-    "specvlm_compact_tree_kv",
+    "specvlm_compact_tree_kv", "specvlm_debug_poison_shared_memory",
 ]
 
 
@@ -88,6 +88,8 @@ def lib():
         L.specvlm_select_top_p.restype = c_int32
         L.specvlm_select_top_p.argtypes = [c_void_p, i32p, i32p, c_int32, i32p, i32p, i32p, c_int32, c_void_p,
                                            c_void_p, c_void_p, c_void_p]
+        L.specvlm_debug_poison_shared_memory.restype = c_int32
+        L.specvlm_debug_poison_shared_memory.argtypes = [c_void_p]
         L.specvlm_verify_tree_workspace_bytes.restype = c_size_t
         L.specvlm_verify_tree_workspace_bytes.argtypes = [kvp, c_int32, c_int32, c_int32]
         L.specvlm_verify_tree_attn.restype = c_int32
@@ -387,6 +389,11 @@ def accept_tree(target_logits: torch.Tensor, node_tokens: torch.Tensor, parents:
                                    _ptr(path), _ptr(g), _ptr(ws), ws.numel(), _stream())
     _check(rc, "specvlm_accept_tree")
     return n, nxt, path, g
+
+
+def debug_poison_shared_memory() -> None:
+    """Fills the SMs' shared memory with NaN bit patterns (test diagnostic)."""
+    _check(lib().specvlm_debug_poison_shared_memory(_stream()), "specvlm_debug_poison_shared_memory")
 
 
 def compact_tree_kv(kv: KvCache, path: torch.Tensor, accept_len: torch.Tensor,

@@ -24,3 +24,14 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _poisoned_shared_memory(request):
+    """Before every GPU test the SMs' shared memory is filled with NaN bit patterns: a kernel that
+    reads a shared-memory word it never wrote then fails its parity check every time, instead of
+    passing whenever the previous kernel happened to leave something harmless there."""
+    if "gpu" in request.keywords:
+        from paper_2508_16201_b200 import specvlm
+        specvlm.debug_poison_shared_memory()
+    yield

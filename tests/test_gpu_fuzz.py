@@ -1,0 +1,120 @@
+"""Seeded random shapes through the attention, rating and selection entry points, against the
+oracle.  The hand-picked cases of the other GPU tests aim at known edges; these sweep combinations
+nobody thought of (group size x window rows x ragged lengths x paging x layer count), which is
+where a flat work partition or a tile-edge mask would break.  Every case is small enough for the
+fp64 oracle; the draws are fixed by the seed in the test id."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import make_cache
+from helpers import bits, f64, row_rel_err
+from paper_2508_16201_b200 import specvlm, synth
+from test_gpu_parity import ATTN_TOL, _run_attn, _scores_case
+
+pytestmark = pytest.mark.gpu
+
+GROUPS = [(4, 4), (8, 2), (28, 4), (40, 8), (64, 8), (16, 1), (12, 2)]     # (query heads, KV heads)
+
+
+def _lens(rng, batch, lo, hi, n_q):
+    """ragged lengths; now and then a sequence that holds the window only, or sits on a tile edge"""
+    out = []
+    for _ in range(batch):
+        r = rng.random()
+        if r < 0.1:
+            out.append(n_q)
+        elif r < 0.25:
+            out.append(int(rng.integers(1, 5)) * 64 + int(rng.integers(0, 2)) * n_q)
+        else:
+            out.append(int(rng.integers(max(lo, n_q), hi)))
+    return out
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_fuzz_chain_attention(seed):
+    rng = np.random.default_rng(1000 + seed)
+    Hq, Hkv = GROUPS[int(rng.integers(0, len(GROUPS)))]
+    D = 64 if rng.random() < 0.3 else 128
+    gamma = int(rng.integers(0, 9))
+    L = int(rng.integers(1, 4))
+    batch = int(rng.integers(1, 6))
+    lens = _lens(rng, batch, 1, 700, gamma + 1)
+    _run_attn(L, Hq, Hkv, D, lens, gamma, paged=bool(rng.integers(0, 2)), seed=2000 + seed, poison=True)
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_fuzz_tree_attention(seed):
+    rng = np.random.default_rng(3000 + seed)
+    Hq, Hkv = GROUPS[int(rng.integers(0, len(GROUPS)))]
+    D = 64 if rng.random() < 0.3 else 128
+    n_nodes = int(rng.integers(1, 33))
+    L = int(rng.integers(1, 3))
+    batch = int(rng.integers(1, 5))
+    lens = _lens(rng, batch, 1, 500, n_nodes)
+    paged = bool(rng.integers(0, 2))
+    cache, k_host, v_host = make_cache(L, Hkv, D, lens, paged=paged, seed=4000 + seed, poison_tail=True)
+    parents = [[-1] + [int(rng.integers(0, t)) for t in range(1, n_nodes)] for _ in range(batch)]
+    par = torch.tensor(parents, dtype=torch.int32, device="cuda")
+    q = synth.randn_bf16((L, batch, n_nodes, Hq, D), "cuda", 4000 + seed, "Qt")
+    scale = 1.0 / math.sqrt(D)
+    lse = torch.empty((L, batch, n_nodes, Hq), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = specvlm.verify_tree_attn(cache, q, par, scale, lse=lse, d_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    got, qh = f64(out), bits(q)
+    assert np.isfinite(got).all()
+    worst = 0.0
+    for l in range(L):
+        for b in range(batch):
+            ref, ref_lse = oracle.attention_tree(qh[l, b], k_host[b][l], v_host[b][l], lens[b], parents[b], scale)
+            worst = max(worst, row_rel_err(got[l, b], ref))
+            np.testing.assert_allclose(lse[l, b].cpu().numpy(), ref_lse, rtol=0, atol=2e-3)
+    assert worst <= ATTN_TOL, f"row rel err {worst}"
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_fuzz_scores(seed):
+    rng = np.random.default_rng(5000 + seed)
+    Hq, Hkv = GROUPS[int(rng.integers(0, len(GROUPS)))]
+    D = 64 if rng.random() < 0.3 else 128
+    batch = int(rng.integers(1, 4))
+    T = int(rng.integers(20, 200))
+    n_frames = [int(rng.integers(1, 5)) for _ in range(batch)]
+    n_text = [int(rng.integers(1, 150)) for _ in range(batch)]
+    prefix = [int(rng.integers(0, 80)) for _ in range(batch)]
+    paged = bool(rng.integers(0, 2))
+    _scores_case(int(rng.integers(1, 3)), Hq, Hkv, D, n_frames, T, n_text, paged=paged, seed=6000 + seed,
+                 prefix=prefix)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_fuzz_select(seed):
+    """Stage I + II on random score vectors with planted ties; fixed count and Top-P count."""
+    rng = np.random.default_rng(7000 + seed)
+    batch = int(rng.integers(1, 5))
+    T = int(rng.integers(3, 300))
+    frames = [int(rng.integers(1, 12)) for _ in range(batch)]
+    nv = [f * T for f in frames]
+    cu = np.concatenate([[0], np.cumsum(nv)]).astype(int).tolist()
+    scores = rng.random(cu[-1]).astype(np.float32) ** 6          # long-tailed
+    scores[rng.integers(0, cu[-1], size=cu[-1] // 5)] = scores[rng.integers(0, cu[-1])]   # ties
+    kt = [int(rng.integers(0, n + 1)) for n in nv]
+    k1 = [int(rng.integers(0, k + 1)) for k in kt]
+    kept_cu = np.concatenate([[0], np.cumsum(kt)]).astype(int).tolist()
+    sc_d = torch.from_numpy(scores).cuda()
+    got = specvlm.select(sc_d, cu, frames, T, k1, kt, kept_cu).cpu().numpy()
+    for b in range(batch):
+        ref = oracle.select(scores[cu[b]:cu[b + 1]], frames[b], T, k1[b], kt[b])
+        assert np.array_equal(got[kept_cu[b]:kept_cu[b + 1]], ref), f"sequence {b}"
+    lam = [int(rng.integers(0, 1001)) for _ in range(batch)]
+    got_p, k1_p = specvlm.select_top_p(sc_d, cu, frames, T, lam, kt, kept_cu)
+    got_p, k1_p = got_p.cpu().numpy(), k1_p.cpu().numpy()
+    for b in range(batch):
+        ref, ref_k1 = oracle.select_top_p(scores[cu[b]:cu[b + 1]], frames[b], T, lam[b], kt[b])
+        assert int(k1_p[b]) == ref_k1
+        assert np.array_equal(got_p[kept_cu[b]:kept_cu[b + 1]], ref), f"top-p sequence {b}"
