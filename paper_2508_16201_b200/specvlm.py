@@ -198,8 +198,16 @@ class KvCache:
         return self.k.shape[4]
 
 
+# When set (the GPU tests set it), scratch buffers that this binding allocates are filled with 0xff
+# bytes (NaN as fp32, -1 as int32) first: no call may depend on what its workspace held before.
+debug_fill_workspaces = False
+
+
 def _ws(nbytes: int, device) -> torch.Tensor:
-    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+    ws = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+    if debug_fill_workspaces:
+        ws.fill_(0xFF)
+    return ws
 
 
 # ---------------------------------------------------------------------------------- attention

@@ -34,4 +34,5 @@ def _poisoned_shared_memory(request):
     if "gpu" in request.keywords:
         from paper_2508_16201_b200 import specvlm
         specvlm.debug_poison_shared_memory()
+        specvlm.debug_fill_workspaces = True          # scratch buffers start as 0xff bytes, too
     yield
