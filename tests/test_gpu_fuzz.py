@@ -124,3 +124,85 @@ def test_fuzz_select(seed):
         ref, ref_k1 = oracle.select_top_p(scores[cu[b]:cu[b + 1]], frames[b], T, lam[b], kt[b])
         assert int(k1_p[b]) == ref_k1
         assert np.array_equal(got_p[kept_cu[b]:kept_cu[b + 1]], ref), f"top-p sequence {b}"
+
+
+@pytest.mark.parametrize("seed", range(6 * SCALE))
+def test_fuzz_gather(seed):
+    from gpu_util import host_view
+    rng = np.random.default_rng(8000 + seed)
+    L, H = int(rng.integers(1, 4)), int(rng.integers(1, 5))
+    D = 64 if rng.random() < 0.3 else 128
+    batch = int(rng.integers(1, 5))
+    video_start = [int(rng.integers(0, 40)) for _ in range(batch)]
+    video_len = [int(rng.integers(1, 600)) for _ in range(batch)]
+    n_text = [int(rng.integers(1, 90)) for _ in range(batch)]
+    src_len = [a + b + c for a, b, c in zip(video_start, video_len, n_text)]
+    kept, kept_cu = [], [0]
+    for nv in video_len:
+        kk = np.sort(rng.choice(nv, int(rng.integers(0, nv + 1)), replace=False)).astype(np.int32)
+        kept.append(kk)
+        kept_cu.append(kept_cu[-1] + len(kk))
+    dst_len = [s - v + len(k) for s, v, k in zip(src_len, video_len, kept)]
+    src, sk, sv = make_cache(L, H, D, src_len, paged=bool(rng.integers(0, 2)), seed=8100 + seed)
+    dst, _, _ = make_cache(L, H, D, dst_len, paged=bool(rng.integers(0, 2)), seed=8200 + seed)
+    kept_all = np.concatenate(kept) if kept_cu[-1] else np.zeros(1, dtype=np.int32)
+    specvlm.gather_kv(src, torch.from_numpy(kept_all).cuda(), kept_cu, video_start, video_len, src_len, dst)
+    torch.cuda.synchronize()
+    dk = host_view(dst.k, dst.block_table, dst_len)
+    dv = host_view(dst.v, dst.block_table, dst_len)
+    for b in range(batch):
+        rk = oracle.gather_kv(sk[b], kept[b], video_start[b], video_len[b], src_len[b])
+        rv = oracle.gather_kv(sv[b], kept[b], video_start[b], video_len[b], src_len[b])
+        n = rk.shape[2]
+        assert np.array_equal(dk[b][:, :, :n], rk) and np.array_equal(dv[b][:, :, :n], rv), f"sequence {b}"
+
+
+@pytest.mark.parametrize("seed", range(6 * SCALE))
+def test_fuzz_accept_chain_and_tree(seed):
+    rng = np.random.default_rng(9000 + seed)
+    batch, gamma = int(rng.integers(1, 9)), int(rng.integers(0, 9))
+    vocab = int(rng.choice([7, 1000, 4099, 32000, 152064]))
+    g = torch.Generator().manual_seed(9000 + seed)
+    logits = torch.randn((batch, gamma + 1, vocab), generator=g)
+    if rng.random() < 0.5:                                   # exact ties: the lowest index wins
+        logits = torch.round(logits * 2) / 2
+    lg = logits.numpy()
+    am = lg.argmax(2)
+    drafts = np.where(rng.random((batch, gamma)) < 0.7, am[:, :gamma], rng.integers(0, vocab, (batch, gamma))).astype(np.int32)
+    n, nxt, gmax = specvlm.accept(logits.cuda(), torch.from_numpy(drafts).cuda().contiguous(), want_argmax=True)
+    torch.cuda.synchronize()
+    for b in range(batch):
+        rn, rnext = oracle.accept_fast(lg[b], drafts[b])[:2]
+        assert (int(n[b]), int(nxt[b])) == (int(rn), int(rnext)), f"sequence {b}"
+    assert np.array_equal(gmax.cpu().numpy(), am)
+    # the same logits as a tree: node t's parent is a random earlier node
+    n_nodes = gamma + 1
+    parents = [[-1] + [int(rng.integers(0, t)) for t in range(1, n_nodes)] for _ in range(batch)]
+    tokens = [[0] + [int(am[b, parents[b][t]]) if rng.random() < 0.7 else int(rng.integers(0, vocab))
+                     for t in range(1, n_nodes)] for b in range(batch)]
+    tn, tnxt, path, _ = specvlm.accept_tree(logits.cuda(), torch.tensor(tokens, dtype=torch.int32, device="cuda"),
+                                            torch.tensor(parents, dtype=torch.int32, device="cuda"))
+    torch.cuda.synchronize()
+    for b in range(batch):
+        rn, rnext, rpath = oracle.accept_tree(lg[b], tokens[b], parents[b])
+        assert (int(tn[b]), int(tnxt[b])) == (rn, rnext), f"tree sequence {b}"
+        assert path[b].cpu().tolist() == rpath + [-1] * (n_nodes - rn)
+
+
+@pytest.mark.parametrize("seed", range(4 * SCALE))
+def test_fuzz_baseline_selectors(seed):
+    rng = np.random.default_rng(9500 + seed)
+    batch = int(rng.integers(1, 5))
+    T = int(rng.integers(1, 300))
+    frames = [int(rng.integers(1, 40)) for _ in range(batch)]
+    kts = [int(rng.integers(0, f * T + 1)) for f in frames]
+    kept_cu = np.concatenate([[0], np.cumsum(kts)]).astype(int).tolist()
+    sd = int(rng.integers(0, 2**62))
+    for mode in (specvlm.SEL_WINDOW_FRONT, specvlm.SEL_WINDOW_MIDDLE, specvlm.SEL_WINDOW_END, specvlm.SEL_FRAMES,
+                 specvlm.SEL_RANDOM):
+        kept, kept_n = specvlm.select_baseline(mode, frames, T, kts, kept_cu, seed=sd)
+        kept, kept_n = kept.cpu().numpy(), kept_n.cpu().numpy()
+        for b, F in enumerate(frames):
+            ref = oracle.select_baseline(mode, F, T, kts[b], seed=sd, b=b)
+            assert int(kept_n[b]) == len(ref), f"mode {mode} sequence {b}"
+            assert np.array_equal(kept[kept_cu[b]:kept_cu[b] + len(ref)], ref), f"mode {mode} sequence {b}"
