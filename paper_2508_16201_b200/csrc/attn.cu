@@ -269,31 +269,50 @@ attn_rows16_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     }
   }
   asm volatile("bar.sync 1, %0;" ::"n"(128 * NG) : "memory");
-  const int item = lb * p.n_kv_heads + g;
-  for (int idx = tid; idx < p.rows * D; idx += 128 * NG) {
-    const int r = idx / D, c = idx - r * D;
+  // The weights of the NW partials are the same for every channel of a row: one thread per
+  // (warp, row) turns its (max, sum) into the weight 2^(m - M) / den in place, thread (0, row)
+  // also leaves the row's log2-sum-exp in l_sm.
+  if (tid < NW * 16) {
+    const int w_me = tid >> 4, r = tid & 15;
     float M = -INFINITY;
 #pragma unroll
     for (int w = 0; w < NW; ++w) M = fmaxf(M, m_sm[w * 16 + r]);
-    float num = 0.f, den = 0.f;
+    float den = 0.f;
     if (M != -INFINITY) {
 #pragma unroll
-      for (int w = 0; w < NW; ++w) {
-        const float f = fast_exp2(m_sm[w * 16 + r] - M);
-        den += l_sm[w * 16 + r] * f;
-        num += o_sm[(w * 16 + r) * OPITCH + c] * f;
-      }
+      for (int w = 0; w < NW; ++w) den += l_sm[w * 16 + r] * fast_exp2(m_sm[w * 16 + r] - M);
     }
-    const float val = den > 0.f ? num / den : 0.f;
-    const float lse2 = den > 0.f ? M + log2f(den) : -INFINITY;
+    const float wt = den > 0.f ? fast_exp2(m_sm[tid] - M) / den : 0.f;
+    asm volatile("bar.sync 2, %0;" ::"n"(NW * 16) : "memory");        // every (max, sum) has been read
+    m_sm[tid] = wt;
+    if (w_me == 0) l_sm[r] = den > 0.f ? M + log2f(den) : -INFINITY;
+  }
+  asm volatile("bar.sync 1, %0;" ::"n"(128 * NG) : "memory");
+  const int item = lb * p.n_kv_heads + g;
+  for (int idx = tid; idx < p.rows * (D / 4); idx += 128 * NG) {
+    const int r = idx / (D / 4), c = (idx - r * (D / 4)) * 4;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int w = 0; w < NW; ++w) {
+      const float f = m_sm[w * 16 + r];
+      const float4 x = *reinterpret_cast<const float4*>(o_sm + (w * 16 + r) * OPITCH + c);
+      acc.x += x.x * f;
+      acc.y += x.y * f;
+      acc.z += x.z * f;
+      acc.w += x.w * f;
+    }
+    const float lse2 = l_sm[r];
     if (p.n_splits == 1) {
       const int t = r / p.group, h = g * p.group + (r - t * p.group);
       const size_t orow = ((size_t)lb * p.n_q + t) * p.n_q_heads + h;
-      p.out[orow * D + c] = __float2bfloat16_rn(val);
+      uint2 packed;
+      packed.x = pack_bf16x2(acc.x, acc.y);
+      packed.y = pack_bf16x2(acc.z, acc.w);
+      *reinterpret_cast<uint2*>(p.out + orow * D + c) = packed;
       if (p.lse && c == 0) p.lse[orow] = lse2 * kLn2;
     } else {
       const size_t prow = ((size_t)item * p.n_splits + split) * p.rows + r;
-      p.ws_o[prow * D + c] = val;
+      *reinterpret_cast<float4*>(p.ws_o + prow * D + c) = acc;
       if (c == 0) p.ws_lse[prow] = lse2;
     }
   }
