@@ -55,6 +55,10 @@ attn_rows16_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
   // before it in the stream is still running.  Everything above touches no global memory; the
   // wait below returns once that kernel's memory operations are complete and visible.  The kernel
   // after this one may be scheduled as soon as every CTA here has got this far.
+  if (tid == 32 * 4 * NG) {              // the producer's lane: descriptors are kernel parameters
+    tma_prefetch_desc(&tm_k);
+    tma_prefetch_desc(&tm_v);
+  }
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
@@ -68,8 +72,6 @@ attn_rows16_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
   if (warp == 4 * NG) {
     // ------------------------------------------------------------------ producer
     if (lane == 0 && n_my > 0) {
-      tma_prefetch_desc(&tm_k);
-      tma_prefetch_desc(&tm_v);
       const uint64_t policy = l2_policy_evict_first();
       const int tiles_per_block = p.block_tokens / kTileTokens;   // used only when paged
       int issued = 0;
