@@ -59,24 +59,44 @@ attn_rows16_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     tma_prefetch_desc(&tm_k);
     tma_prefetch_desc(&tm_v);
   }
+  __syncthreads();                       // the barriers are initialised
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  // The first tile of an unsplit, contiguous cache sits at a known place whatever the sequence's
+  // length (rows past the cache's end are zero-filled by the copy): the producer asks for it
+  // before the length has even been read, which takes a global-memory round trip off the start.
+  const bool spec = p.n_splits == 1 && p.block_table == nullptr;
+  if (spec && tid == 32 * 4 * NG) {
+    const uint64_t policy = l2_policy_evict_first();
+    mbar_arrive_expect_tx(bar_full, STAGE_BYTES);
+#pragma unroll
+    for (int h = 0; h < D / 64; ++h) {
+      tma_load_5d(base + h * (kTileTokens * 128), &tm_k, bar_full, h * 64, 0, g, b, layer, policy);
+      tma_load_5d(base + TILE_BYTES + h * (kTileTokens * 128), &tm_v, bar_full, h * 64, 0, g, b, layer, policy);
+    }
+  }
 
   int kv_len = p.seq_lens[b];
   kv_len = kv_len < 0 ? 0 : (kv_len > p.max_seq_len ? p.max_seq_len : kv_len);
   int tile_begin, tile_end;
   split_range(kv_len, p.n_splits, split, tile_begin, tile_end);
   const int n_my = tile_end - tile_begin;
-  __syncthreads();
 
   if (warp == 4 * NG) {
     // ------------------------------------------------------------------ producer
+    if (lane == 0 && n_my == 0 && spec) {
+      // an empty sequence: nobody will consume the tile asked for above; stay until it has landed
+      const uint64_t t0 = global_timer_ns();
+      while (!mbar_try_wait(bar_full, 0) && global_timer_ns() - t0 < kWaitLimitNs) {
+      }
+    }
     if (lane == 0 && n_my > 0) {
       const uint64_t policy = l2_policy_evict_first();
       const int tiles_per_block = p.block_tokens / kTileTokens;   // used only when paged
-      int issued = 0;
+      int issued = spec ? 1 : 0;
       bool ok = true;
-      for (int i = 0; i < n_my && ok; ++i) {
+      for (int i = issued; i < n_my && ok; ++i) {
         const int s = i % STAGES;
         if (i >= STAGES) ok = mbar_wait(bar_empty + 8 * s, ((i / STAGES) - 1) & 1, abort_flag);
         if (!ok) break;
