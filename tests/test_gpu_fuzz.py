@@ -206,3 +206,63 @@ def test_fuzz_baseline_selectors(seed):
             ref = oracle.select_baseline(mode, F, T, kts[b], seed=sd, b=b)
             assert int(kept_n[b]) == len(ref), f"mode {mode} sequence {b}"
             assert np.array_equal(kept[kept_cu[b]:kept_cu[b] + len(ref)], ref), f"mode {mode} sequence {b}"
+
+
+@pytest.mark.parametrize("seed", range(6 * SCALE))
+def test_fuzz_cache_append_rollback_compact(seed):
+    """append -> rollback lengths, and tree compaction along a random accepted path, bit for bit."""
+    from gpu_util import host_view
+    rng = np.random.default_rng(9800 + seed)
+    L, H = int(rng.integers(1, 4)), int(rng.integers(1, 5))
+    D = 64 if rng.random() < 0.3 else 128
+    batch = int(rng.integers(1, 5))
+    paged = bool(rng.integers(0, 2))
+    n_new = int(rng.integers(1, 10))
+    lens = [int(rng.integers(0, 300)) for _ in range(batch)]
+    cap = [n + n_new for n in lens]
+    cache, k_host, v_host = make_cache(L, H, D, cap, paged=paged, seed=9900 + seed)
+    cache.seq_lens.copy_(torch.tensor(lens, dtype=torch.int32))
+    new_k = synth.randn_bf16((L, batch, n_new, H, D), "cuda", 9900 + seed, "nk")
+    new_v = synth.randn_bf16((L, batch, n_new, H, D), "cuda", 9900 + seed, "nv")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    specvlm.append_kv(cache, new_k, new_v, d_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and cache.seq_lens.cpu().tolist() == cap
+    gk = host_view(cache.k, cache.block_table, cap)
+    gv = host_view(cache.v, cache.block_table, cap)
+    for b in range(batch):
+        rk, _ = oracle.append_kv(k_host[b], bits(new_k[:, b]), lens[b])
+        rv, _ = oracle.append_kv(v_host[b], bits(new_v[:, b]), lens[b])
+        assert np.array_equal(gk[b], rk) and np.array_equal(gv[b], rv), f"append, sequence {b}"
+        k_host[b], v_host[b] = rk, rv
+    # the n_new rows as a draft tree's window: keep a random root-to-node path
+    n_nodes = n_new
+    paths = []
+    for b in range(batch):
+        parents = [-1] + [int(rng.integers(0, t)) for t in range(1, n_nodes)]
+        node = int(rng.integers(0, n_nodes))
+        chain = []
+        while node > 0:
+            chain.append(node)
+            node = parents[node]
+        paths.append(chain[::-1])
+    path_d = torch.tensor([p + [-1] * (n_nodes - len(p)) for p in paths], dtype=torch.int32, device="cuda")
+    n_acc = torch.tensor([len(p) for p in paths], dtype=torch.int32, device="cuda")
+    specvlm.compact_tree_kv(cache, path_d, n_acc, d_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    new_lens = cache.seq_lens.cpu().tolist()
+    gk = host_view(cache.k, cache.block_table, new_lens)
+    gv = host_view(cache.v, cache.block_table, new_lens)
+    for b in range(batch):
+        rk, nl = oracle.compact_tree_kv(k_host[b], cap[b], n_nodes, paths[b])
+        rv, _ = oracle.compact_tree_kv(v_host[b], cap[b], n_nodes, paths[b])
+        assert new_lens[b] == nl
+        assert np.array_equal(gk[b], rk[:, :, :nl]) and np.array_equal(gv[b], rv[:, :, :nl]), f"compaction, sequence {b}"
+    # chain rollback arithmetic on fresh lengths
+    gamma = n_new - 1
+    acc = [int(rng.integers(0, gamma + 1)) for _ in range(batch)]
+    lens_d = torch.tensor(cap, dtype=torch.int32, device="cuda")
+    specvlm.rollback_kv(lens_d, torch.tensor(acc, dtype=torch.int32, device="cuda"), gamma)
+    torch.cuda.synchronize()
+    assert lens_d.cpu().tolist() == [oracle.rollback_len(cap[b], gamma, acc[b]) for b in range(batch)]
