@@ -170,3 +170,27 @@ def test_gather_cfg2_all_28_layers():
     for name, s_t, d_t in (("K", sk, dk), ("V", sv, dv)):
         ref = oracle.gather_kv(bits(s_t[:, 0]), kept_np, 0, nv, nv + nt)
         assert np.array_equal(bits(d_t[:, 0]), ref), name
+
+
+def test_scores_cfg3_shapes_sampled_layer():
+    """Token rating at workload 3's per-layer size (5 query heads per KV head: 25 queries x 5 heads
+    fill 125 of a tile's 128 rows; 23 040 video + 256 text tokens), 3 of 64 layers, one of them
+    rated by the oracle."""
+    w = synth.workload(3)
+    D, nv, nt, L = w.head_dim, w.n_video(), w.n_text[0], 3
+    scale = 1.0 / math.sqrt(D)
+    k = synth.randn_bf16((L, 1, w.t_kv_heads, nv + nt, D), "cuda", 131, "tK")
+    q = synth.randn_bf16((L, nt, w.t_q_heads, D), "cuda", 131, "Qtext")
+    synth.plant_salient_(k[:, 0, :, :nv, :], q, synth.salient_set(nv, w.planted_permille, 131))
+    lens = torch.tensor([nv + nt], dtype=torch.int32, device="cuda")
+    args = ([0, nt], [nv], [0], [nv], [0, nv], scale)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    full = specvlm.stage1_scores(specvlm.KvCache(k, k, lens, nv + nt), q, *args, d_status=status).double()
+    one = specvlm.stage1_scores(specvlm.KvCache(k[1:2], k[1:2], lens, nv + nt), q[1:2], *args, d_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ref = oracle.stage1_scores(bits(q[1:2]), bits(k[1:2, 0]), 0, nv, nv, scale)
+    got = one.cpu().numpy().astype(np.float64)
+    rel = float((np.abs(got - ref) / ref).max())
+    assert rel <= SCORE_TOL, f"scores rel err {rel}"
+    assert np.isfinite(full.cpu().numpy()).all() and float(full.sum()) <= 1.0 and float(full.min()) >= 0.0
