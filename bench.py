@@ -618,6 +618,9 @@ def run_case(args):
         w = dataclasses.replace(w, n_frames=(args.frames,))
     device = torch.device("cuda", 0)
     torch.cuda.set_device(0)
+    if w.batch > 1:
+        run_case_batched(args, w, device)
+        return
     inp = build_inputs(w, device, n_copies=1)
     path = Path(w, inp, device)
     path.row_lse_call(); path.scores_call(); path.select_call()
@@ -670,6 +673,54 @@ def run_case(args):
                       "median_us": round(med * 1e3, 2), "min_us": round(min(ts) * 1e3, 2),
                       "gbs": round(nbytes / (med * 1e-3) / 1e9, 1) if nbytes else None,
                       "env": {k: v for k, v in os.environ.items() if k.startswith("SPECVLM_")}}))
+
+
+def run_case_batched(args, w, device):
+    """The attention calls on a batched workload: ragged sequences in 64-token pages scattered over a
+    pool (the rating / selection / gather cases time one sequence at a time and are not offered here)."""
+    import torch
+    from paper_2508_16201_b200 import specvlm, synth
+    D, B, gamma = w.head_dim, w.batch, w.gamma
+    scale = 1.0 / math.sqrt(D)
+
+    def paged(n_layers, n_kv_heads, lens, tag):
+        need = [(n + 63) // 64 for n in lens]
+        pool, max_blocks = sum(need) + 3, max(need) + 1
+        table = synth.page_table(B, max_blocks, pool, need, 0, device)
+        k = synth.randn_bf16((n_layers, pool, n_kv_heads, 64, D), device, 0, tag + "K")
+        v = synth.randn_bf16((n_layers, pool, n_kv_heads, 64, D), device, 0, tag + "V")
+        cache = specvlm.KvCache(k, v, torch.tensor(lens, dtype=torch.int32, device=device), max(lens), table)
+        return cache, 2 * sum(lens) * n_kv_heads * D * 2 * n_layers
+
+    if args.case == "verify":
+        cache, nbytes = paged(w.t_layers, w.t_kv_heads, [w.seq_len(b) + gamma + 1 for b in range(B)], "t")
+        q = synth.randn_bf16((w.t_layers, B, gamma + 1, w.t_q_heads, D), device, 0, "Qv")
+        out = torch.empty_like(q)
+        ws = torch.empty(max(256, specvlm.attn_workspace_bytes(cache, B, w.t_q_heads, gamma)), dtype=torch.uint8, device=device)
+        fn = lambda: specvlm.verify_attn(cache, q, gamma, scale, out=out, ws=ws)
+    elif args.case in ("decode", "decode_unpruned"):
+        lens = [(w.k_total(b) + w.n_text[b]) if args.case == "decode" else w.seq_len(b) for b in range(B)]
+        cache, nbytes = paged(w.d_layers, w.d_kv_heads, lens, "d")
+        q = synth.randn_bf16((w.d_layers, B, w.d_q_heads, D), device, 0, "Qd")
+        out = torch.empty_like(q)
+        ws = torch.empty(max(256, specvlm.attn_workspace_bytes(cache, B, w.d_q_heads, 0)), dtype=torch.uint8, device=device)
+        fn = lambda: specvlm.draft_decode_attn(cache, q, scale, out=out, ws=ws)
+    else:
+        raise SystemExit("--case %s is timed one sequence at a time: use a batch-1 workload" % args.case)
+    status = torch.zeros(1, dtype=torch.int32, device=device)
+    ts = []
+    for i in range(args.warmup + args.iters):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        torch.cuda.synchronize()
+        if i >= args.warmup:
+            ts.append(a.elapsed_time(b))
+    med = statistics.median(ts)
+    print(json.dumps({"case": args.case, "workload": w.name, "batch": B, "paged": True, "gamma": gamma,
+                      "median_us": round(med * 1e3, 2), "min_us": round(min(ts) * 1e3, 2),
+                      "gbs": round(nbytes / (med * 1e-3) / 1e9, 1)}))
 
 
 def main():
