@@ -480,10 +480,11 @@ constexpr int kPolyOf8Colsum = SPECVLM_POLY_COLSUM;
 //   D[key][row] = K_block (A: 128 keys x d, K-major) * Q_tile^T (B: 128 rows x d, K-major)
 // is one chain of tcgen05.mma instructions (M = N = 128, K = 16 each) issued by a single thread,
 // with both operands read straight from the 128-byte-swizzled tiles the TMA wrote and the fp32
-// accumulator in tensor memory (two 128-column buffers, so the next tile's MMAs overlap this
-// tile's epilogue).  With the keys on the TMEM lanes, an epilogue thread owns one key: it reads
-// its 128 row values with tcgen05.ld and adds up 2^(s - lse_row) in a single register for the
-// whole layer -- the column sum needs no cross-thread reduction at all.
+// accumulator in tensor memory (one 128-column buffer per epilogue group, so the MMAs of the next
+// tiles overlap the epilogues of the current ones).  With the keys on the TMEM lanes, an epilogue
+// thread owns one key: it reads its 128 row values with tcgen05.ld and adds up 2^(s - lse_row) in
+// registers for the whole layer -- the column sum needs no cross-thread reduction inside a group;
+// the groups' sums meet once, at the end, in a fixed order.
 // Warps: 0 = TMA producer, 1 = TMEM allocation + MMA issue, then kColsumGroups epilogue groups of
 // four warps (one TMEM lane quadrant per warp) that take the tiles round-robin, each on its own
 // accumulator buffer: four warps per scheduler keep the special-function unit busy while others
