@@ -1,5 +1,7 @@
 // Streaming softmax attention over a bf16 K/V cache on the 5th-generation tensor cores of sm_100a:
-// draft decode attention (1 query token) and (gamma+1)-query verification attention.
+// (gamma+1)-query verification attention and tree verification, i.e. windows of 17 to 128 rows per
+// KV head and launch (wider windows run as several launches; up to 16 rows run on the kernel of
+// attn.cu).
 //
 // One persistent CTA per SM streams a contiguous slice of the flat (layer, sequence, KV head, tile)
 // list (attn_sched.h), so the cache is read exactly once, every SM moves the same number of bytes
