@@ -113,6 +113,25 @@ int32_t specvlm_stage1_scores(const specvlm_kv_t* target_kv, const void* q_text,
                               const int32_t* video_cu, int32_t batch, int32_t n_q_heads,
                               float sm_scale, const float* row_lse_or_null, float* scores, void* ws,
                               size_t ws_bytes, int32_t* d_status, void* stream);
+/*
+ * The same rating, a range of layers at a time (Eq. 5 averages over the layers, so their
+ * contributions can be gathered as the verifier's prefill produces them, or as their queries arrive
+ * from the host).  All arguments describe the whole problem, exactly as for specvlm_stage1_scores
+ * (target_kv and q_text cover all n_layers layers); this call rates layers layer_begin ..
+ * layer_end-1 and leaves each layer's unnormalised column sums in `ws`.  With finish != 0 it then
+ * adds up the sums of ALL layers, in layer order, and writes `scores`: the result is bit-identical to
+ * one call of specvlm_stage1_scores, provided every layer has been rated by some earlier call (or
+ * this one) with the same `ws`, whose contents must be left alone in between.  An empty range with
+ * finish != 0 only reduces.  row_lse_or_null, when given, is the full [n_layers][sum_text][n_q_heads]
+ * array; only the range's rows are read.
+ */
+int32_t specvlm_stage1_scores_layers(const specvlm_kv_t* target_kv, const void* q_text,
+                                     const int32_t* text_cu, const int32_t* text_start,
+                                     const int32_t* video_start, const int32_t* video_len,
+                                     const int32_t* video_cu, int32_t batch, int32_t n_q_heads,
+                                     float sm_scale, const float* row_lse_or_null, float* scores, void* ws,
+                                     size_t ws_bytes, int32_t layer_begin, int32_t layer_end, int32_t finish,
+                                     int32_t* d_status, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Steps 1b + 2 -- two-stage selection (Section 4.2).

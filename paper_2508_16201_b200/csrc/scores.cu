@@ -30,6 +30,7 @@ struct ScoreParams {
   const int32_t* block_table;
   int32_t* d_status;
   int32_t batch, n_layers, n_q_heads, n_kv_heads, group, qt, sum_text, sum_video;
+  int32_t layer0;                      // first layer of this launch (the grid covers a range of layers)
   int32_t max_blocks, block_tokens;
   float scale_log2;
   ScoreSeq seq[kScoresMaxBatch];
@@ -91,7 +92,7 @@ scores_lse_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   const int b = find_seq(p, blockIdx.x);
   const ScoreSeq sq = p.seq[b];
   const int qtile = blockIdx.x - sq.tile_off;
-  const int g = blockIdx.y, layer = blockIdx.z;
+  const int g = blockIdx.y, layer = blockIdx.z + p.layer0;
   const int i_first = qtile * p.qt;
   const int n_i = min(p.qt, sq.n_text - i_first);               // queries in this tile
   const int rows_valid = n_i * p.group;
@@ -290,7 +291,7 @@ scores_colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
   const int b = find_seq(p, blockIdx.x);
   const ScoreSeq sq = p.seq[b];
   const int kblock = blockIdx.x - sq.tile_off;
-  const int layer = blockIdx.y;
+  const int layer = blockIdx.y + p.layer0;
   // key blocks start on a page boundary at or before the first video token, so that a 64-token
   // TMA box never straddles two cache pages; columns outside the video range are dropped
   const int key0 = (sq.video_start / 64) * 64 + kblock * kKeyTile;   // absolute position of column 0
@@ -525,7 +526,7 @@ scores_colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
   const int b = find_seq(p, blockIdx.x);
   const ScoreSeq sq = p.seq[b];
   const int kblock = blockIdx.x - sq.tile_off;
-  const int layer = blockIdx.y;
+  const int layer = blockIdx.y + p.layer0;
   const int key0 = (sq.video_start / 64) * 64 + kblock * kKeyTile;
   const int n_qt = (sq.n_text + p.qt - 1) / p.qt;
   const int n_units = p.n_kv_heads;
@@ -773,7 +774,7 @@ scores_lse_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
   const int b = find_seq(p, blockIdx.x);
   const ScoreSeq sq = p.seq[b];
   const int qtile = blockIdx.x - sq.tile_off;
-  const int g = blockIdx.y, layer = blockIdx.z;
+  const int g = blockIdx.y, layer = blockIdx.z + p.layer0;
   const int i_first = qtile * p.qt;
   const int n_i = min(p.qt, sq.n_text - i_first);               // queries in this tile
   const int rows_valid = n_i * p.group;
@@ -952,6 +953,8 @@ static void ws_layout(int n_layers, int n_q_heads, int64_t sum_text, int64_t sum
 }
 
 struct ScoreSetup {
+  int layer_begin = 0, layer_count = 0;   // the layers this call rates
+  bool finish = true;                      // reduce the per-layer partial sums into the scores
   specvlm_kv_t kv;
   ScoreParams p1, p2;          // pass-1 (row tiles) and pass-2 (key blocks) CTA tables
   CUtensorMap tk, tq;
@@ -1001,6 +1004,7 @@ static int32_t setup_scores(const specvlm_kv_t* target_kv, const void* q_text, c
   p.d_status = d_status;
   p.batch = batch;
   p.n_layers = kv.n_layers;
+  p.layer0 = 0;
   p.n_q_heads = n_q_heads;
   p.n_kv_heads = kv.n_kv_heads;
   p.group = group;
@@ -1010,6 +1014,9 @@ static int32_t setup_scores(const specvlm_kv_t* target_kv, const void* q_text, c
   p.block_tokens = kv.block_tokens;
   p.scale_log2 = sm_scale * kLog2e;
   su.p2 = p;
+  su.layer_begin = 0;
+  su.layer_count = kv.n_layers;
+  su.finish = true;
   su.n_row_tiles = su.n_key_blocks = 0;
   for (int b = 0; b < batch; ++b) {
     const int nt = text_cu[b + 1] - text_cu[b];
@@ -1053,7 +1060,7 @@ static bool scores_legacy_mma() {
 
 template <int D>
 static int32_t launch_lse(ScoreSetup& su, cudaStream_t st) {
-  const dim3 grid((unsigned)su.n_row_tiles, (unsigned)su.kv.n_kv_heads, (unsigned)su.kv.n_layers);
+  const dim3 grid((unsigned)su.n_row_tiles, (unsigned)su.kv.n_kv_heads, (unsigned)su.layer_count);
   if (scores_legacy_mma()) {
     constexpr int STAGES = 4;
     constexpr int SMEM = STAGES * kKeyTile * D * 2 + 1024 + 16 * STAGES + 16 + 2 * 128 * 2 * 4;
@@ -1082,7 +1089,7 @@ static int32_t launch_colsum(ScoreSetup& su, float* scores, cudaStream_t st) {
     auto k = scores_colsum_kernel<D, STAGES>;
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
       return SPECVLM_ERR_CUDA;
-    k<<<dim3((unsigned)su.n_key_blocks, (unsigned)su.kv.n_layers), 288, SMEM, st>>>(su.tk, su.tq, su.p2);
+    k<<<dim3((unsigned)su.n_key_blocks, (unsigned)su.layer_count), 288, SMEM, st>>>(su.tk, su.tq, su.p2);
     rc = launch_status();
   } else {
     constexpr int STAGES = 4;
@@ -1091,10 +1098,10 @@ static int32_t launch_colsum(ScoreSetup& su, float* scores, cudaStream_t st) {
     auto k = scores_colsum_tc_kernel<D, STAGES>;
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
       return SPECVLM_ERR_CUDA;
-    k<<<dim3((unsigned)su.n_key_blocks, (unsigned)su.kv.n_layers), kColsumThreads, SMEM, st>>>(su.tk, su.tq, su.p2);
+    k<<<dim3((unsigned)su.n_key_blocks, (unsigned)su.layer_count), kColsumThreads, SMEM, st>>>(su.tk, su.tq, su.p2);
     rc = launch_status();
   }
-  if (rc != SPECVLM_OK) return rc;
+  if (rc != SPECVLM_OK || !su.finish) return rc;
   scores_finish_kernel<<<(unsigned)((su.p2.sum_video + 255) / 256), 256, 0, st>>>(su.p2, scores);
   return launch_status();
 }
@@ -1128,23 +1135,35 @@ extern "C" int32_t specvlm_stage1_row_lse(const specvlm_kv_t* target_kv, const v
   return su.kv.head_dim == 128 ? launch_lse<128>(su, st) : launch_lse<64>(su, st);
 }
 
-extern "C" int32_t specvlm_stage1_scores(const specvlm_kv_t* target_kv, const void* q_text,
-                                         const int32_t* text_cu, const int32_t* text_start,
-                                         const int32_t* video_start, const int32_t* video_len,
-                                         const int32_t* video_cu, int32_t batch, int32_t n_q_heads,
-                                         float sm_scale, const float* row_lse_or_null, float* scores,
-                                         void* ws, size_t ws_bytes, int32_t* d_status, void* stream) {
+static int32_t stage1_scores_range(const specvlm_kv_t* target_kv, const void* q_text, const int32_t* text_cu,
+                                   const int32_t* text_start, const int32_t* video_start,
+                                   const int32_t* video_len, const int32_t* video_cu, int32_t batch,
+                                   int32_t n_q_heads, float sm_scale, const float* row_lse_or_null, float* scores,
+                                   void* ws, size_t ws_bytes, int32_t layer_begin, int32_t layer_end, bool finish,
+                                   int32_t* d_status, void* stream) {
   if (!video_start || !video_len || !video_cu || !scores || !ws) return SPECVLM_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(ws) & 255u) return SPECVLM_ERR_INVALID_ARG;
   ScoreSetup su;
   int32_t rc = setup_scores(target_kv, q_text, text_cu, text_start, video_start, video_len, video_cu, batch,
                             n_q_heads, sm_scale, d_status, su);
   if (rc != SPECVLM_OK) return rc;
+  if (layer_begin < 0 || layer_end > su.kv.n_layers || layer_begin > layer_end) return SPECVLM_ERR_INVALID_ARG;
   size_t lse_bytes, partial_bytes;
   ws_layout(su.kv.n_layers, n_q_heads, su.p1.sum_text, su.p1.sum_video, lse_bytes, partial_bytes);
   if (ws_bytes < lse_bytes + partial_bytes) return SPECVLM_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool d128 = su.kv.head_dim == 128;
+  su.layer_begin = layer_begin;
+  su.layer_count = layer_end - layer_begin;
+  su.finish = finish;
+  su.p1.layer0 = su.p2.layer0 = layer_begin;
+  su.p2.partial = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + lse_bytes);
+  if (su.layer_count == 0) {
+    // nothing to rate: only the final reduction, if asked for
+    if (!finish) return SPECVLM_OK;
+    scores_finish_kernel<<<(unsigned)((su.p2.sum_video + 255) / 256), 256, 0, st>>>(su.p2, scores);
+    return launch_status();
+  }
   if (row_lse_or_null) {
     su.p2.lse = const_cast<float*>(row_lse_or_null);
   } else {
@@ -1152,6 +1171,29 @@ extern "C" int32_t specvlm_stage1_scores(const specvlm_kv_t* target_kv, const vo
     rc = d128 ? launch_lse<128>(su, st) : launch_lse<64>(su, st);
     if (rc != SPECVLM_OK) return rc;
   }
-  su.p2.partial = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + lse_bytes);
   return d128 ? launch_colsum<128>(su, scores, st) : launch_colsum<64>(su, scores, st);
+}
+
+extern "C" int32_t specvlm_stage1_scores(const specvlm_kv_t* target_kv, const void* q_text,
+                                         const int32_t* text_cu, const int32_t* text_start,
+                                         const int32_t* video_start, const int32_t* video_len,
+                                         const int32_t* video_cu, int32_t batch, int32_t n_q_heads,
+                                         float sm_scale, const float* row_lse_or_null, float* scores,
+                                         void* ws, size_t ws_bytes, int32_t* d_status, void* stream) {
+  if (!target_kv) return SPECVLM_ERR_INVALID_ARG;
+  return stage1_scores_range(target_kv, q_text, text_cu, text_start, video_start, video_len, video_cu, batch,
+                             n_q_heads, sm_scale, row_lse_or_null, scores, ws, ws_bytes, 0, target_kv->n_layers, true,
+                             d_status, stream);
+}
+
+extern "C" int32_t specvlm_stage1_scores_layers(const specvlm_kv_t* target_kv, const void* q_text,
+                                                const int32_t* text_cu, const int32_t* text_start,
+                                                const int32_t* video_start, const int32_t* video_len,
+                                                const int32_t* video_cu, int32_t batch, int32_t n_q_heads,
+                                                float sm_scale, const float* row_lse_or_null, float* scores,
+                                                void* ws, size_t ws_bytes, int32_t layer_begin, int32_t layer_end,
+                                                int32_t finish, int32_t* d_status, void* stream) {
+  return stage1_scores_range(target_kv, q_text, text_cu, text_start, video_start, video_len, video_cu, batch,
+                             n_q_heads, sm_scale, row_lse_or_null, scores, ws, ws_bytes, layer_begin, layer_end,
+                             finish != 0, d_status, stream);
 }

@@ -48,6 +48,7 @@ _lib = None
 EXPORTS = [
     "specvlm_version", "specvlm_status_string",
     "specvlm_stage1_scores_workspace_bytes", "specvlm_stage1_row_lse", "specvlm_stage1_scores",
+    "specvlm_stage1_scores_layers",
     "specvlm_select", "specvlm_select_top_p", "specvlm_select_baseline", "specvlm_gather_kv",
     "specvlm_attn_workspace_bytes", "specvlm_draft_decode_attn", "specvlm_verify_attn",
     "specvlm_accept_workspace_bytes", "specvlm_accept", "specvlm_accept_noalloc",
@@ -76,6 +77,10 @@ def lib():
         L.specvlm_stage1_scores.argtypes = [kvp, c_void_p, i32p, i32p, i32p, i32p, i32p, c_int32, c_int32,
                                             c_float, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p,
                                             c_void_p]
+        L.specvlm_stage1_scores_layers.restype = c_int32
+        L.specvlm_stage1_scores_layers.argtypes = [kvp, c_void_p, i32p, i32p, i32p, i32p, i32p, c_int32, c_int32,
+                                                   c_float, c_void_p, c_void_p, c_void_p, c_size_t, c_int32,
+                                                   c_int32, c_int32, c_void_p, c_void_p]
         L.specvlm_stage1_row_lse.restype = c_int32
         L.specvlm_stage1_row_lse.argtypes = [kvp, c_void_p, i32p, i32p, c_int32, c_int32, c_float, c_void_p,
                                              c_void_p, c_void_p]
@@ -285,6 +290,25 @@ def stage1_scores(kv: KvCache, q_text: torch.Tensor, text_cu, text_start, video_
                                      float(sm_scale), _ptr(row_lse), _ptr(scores), _ptr(ws), ws.numel(),
                                      _ptr(d_status), _stream())
     _check(rc, "specvlm_stage1_scores")
+    return scores
+
+
+def stage1_scores_layers(kv: KvCache, q_text: torch.Tensor, text_cu, text_start, video_start, video_len,
+                         video_cu, sm_scale: float, scores: torch.Tensor, ws: torch.Tensor, layer_begin: int,
+                         layer_end: int, finish: bool, d_status: torch.Tensor | None = None,
+                         row_lse: torch.Tensor | None = None) -> torch.Tensor:
+    """Rates layers [layer_begin, layer_end) of the problem that ``kv`` and ``q_text`` describe as a
+    whole; with ``finish`` the sums of all layers (left in ``ws`` by this and earlier calls) become
+    ``scores``.  ``ws`` and ``scores`` are the caller's, kept across the calls."""
+    L, n_text_all, Hq, D = q_text.shape
+    batch = len(video_len)
+    assert q_text.is_contiguous() and q_text.dtype == torch.bfloat16 and n_text_all == text_cu[-1]
+    rc = lib().specvlm_stage1_scores_layers(byref(kv.struct), _ptr(q_text), _i32(text_cu), _i32(text_start),
+                                            _i32(video_start), _i32(video_len), _i32(video_cu), batch, Hq,
+                                            float(sm_scale), _ptr(row_lse), _ptr(scores), _ptr(ws), ws.numel(),
+                                            int(layer_begin), int(layer_end), 1 if finish else 0,
+                                            _ptr(d_status), _stream())
+    _check(rc, "specvlm_stage1_scores_layers")
     return scores
 
 

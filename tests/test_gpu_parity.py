@@ -397,6 +397,36 @@ def test_scores_sharp_softmax():
     _scores_case(1, 8, 8, 64, [2], 130, [5], paged=True, seed=8, scale_mul=12.0)
 
 
+def test_scores_by_layer_ranges_equal_one_call():
+    """Rating the layers in ranges (uneven ones, an empty one, the reduction on its own) gives the
+    bits of the single call: each layer's sums land in the workspace, the last call adds them in
+    layer order."""
+    from gpu_util import make_cache
+    L, Hq, Hkv, D, nv, nt, prefix = 5, 40, 8, 128, 300, 37, 3
+    cache, _, _ = make_cache(L, Hkv, D, [prefix + nv + nt], paged=True, seed=20)
+    q = synth.randn_bf16((L, nt, Hq, D), "cuda", 20, "Qtext")
+    args = ([0, nt], [prefix + nv], [prefix], [nv], [0, nv], 1.0 / math.sqrt(D))
+    whole = specvlm.stage1_scores(cache, q, *args)
+    for cuts in ([0, 2, 2, 3, 5], [0, 5], [0, 1, 2, 3, 4, 5]):
+        ws = torch.full((specvlm.stage1_scores_workspace_bytes(cache, [0, nt], [nv], Hq),), 0xFF, dtype=torch.uint8,
+                        device="cuda")
+        out = torch.full((nv,), float("nan"), device="cuda")
+        for a, b in zip(cuts[:-1], cuts[1:]):
+            specvlm.stage1_scores_layers(cache, q, *args, out, ws, a, b, finish=False)
+        specvlm.stage1_scores_layers(cache, q, *args, out, ws, L, L, finish=True)
+        torch.cuda.synchronize()
+        assert torch.equal(out, whole), cuts
+    # the last range may finish by itself
+    ws = torch.zeros((specvlm.stage1_scores_workspace_bytes(cache, [0, nt], [nv], Hq),), dtype=torch.uint8, device="cuda")
+    out = torch.empty((nv,), device="cuda")
+    specvlm.stage1_scores_layers(cache, q, *args, out, ws, 0, 3, finish=False)
+    specvlm.stage1_scores_layers(cache, q, *args, out, ws, 3, 5, finish=True)
+    torch.cuda.synchronize()
+    assert torch.equal(out, whole)
+    with pytest.raises(specvlm.SpecvlmError):
+        specvlm.stage1_scores_layers(cache, q, *args, out, ws, 4, 6, finish=False)
+
+
 def test_scores_ragged_batch():
     _scores_case(2, 16, 4, 128, [2, 5, 1], 64, [64, 17, 200], paged=True, seed=3)
     _scores_case(2, 16, 4, 128, [2, 5, 1], 50, [64, 17, 200], paged=False, seed=4, prefix=[0, 3, 70])
