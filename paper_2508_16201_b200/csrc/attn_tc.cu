@@ -53,7 +53,12 @@ struct AttnTcParams {
 constexpr float kRescaleThreshold = 8.f;   // log2 units
 constexpr int kBigTokens = 2 * kTileTokens;          // tokens per MMA tile
 constexpr int kTcThreads = 384;
-constexpr int kRegsLight = 96, kRegsSoftmax = 200;   // 128 * 96 + 256 * 200 <= 64 K registers
+// setmaxnreg moves registers between the warps of a CTA inside the pool the CTA got at launch
+// (threads x registers per thread as compiled: 384 x 168), and an increase blocks until the pool
+// has them -- for ever, if the requests add up to more than the pool.  The launch code checks the
+// sum against the compiled kernel's pool and refuses to launch otherwise.
+constexpr int kRegsLight = 96, kRegsSoftmax = 200;
+constexpr int kRegsNeeded = 128 * kRegsLight + 256 * kRegsSoftmax;
 
 template <int N> __device__ __forceinline__ void setmaxnreg_dec() {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
@@ -925,6 +930,9 @@ static int32_t launch_tc_t(const CUtensorMap& tk, const CUtensorMap& tv, const C
   auto kern = attn_tc_kernel<D, M, TREE>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::TOTAL) != cudaSuccess)
     return SPECVLM_ERR_CUDA;
+  cudaFuncAttributes fa;
+  if (cudaFuncGetAttributes(&fa, kern) != cudaSuccess) return SPECVLM_ERR_CUDA;
+  if (fa.numRegs * kTcThreads < kRegsNeeded) return SPECVLM_ERR_CUDA;   // setmaxnreg could never be satisfied
   kern<<<grid, kTcThreads, C::TOTAL, st>>>(tk, tv, tq, p);
   return launch_status();
 }
