@@ -1,5 +1,6 @@
 // Host-side helpers: argument validation of specvlm_kv_t, tensor-map encoding, launch checks.
 #pragma once
+#include <atomic>
 
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -41,7 +42,9 @@ typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_
                                     CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 inline encode_tiled_fn get_encode_tiled() {
-  static encode_tiled_fn fn = nullptr;     // resolved once per process; a pure function pointer
+  // resolved once per process; a pure function pointer (threads that race here store the same value)
+  static std::atomic<encode_tiled_fn> cached{nullptr};
+  encode_tiled_fn fn = cached.load(std::memory_order_acquire);
   if (!fn) {
     void* p = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -49,6 +52,7 @@ inline encode_tiled_fn get_encode_tiled() {
         qres != cudaDriverEntryPointSuccess)
       return nullptr;
     fn = reinterpret_cast<encode_tiled_fn>(p);
+    cached.store(fn, std::memory_order_release);
   }
   return fn;
 }
@@ -78,12 +82,15 @@ inline int32_t launch_status() {
 }
 
 inline int sm_count() {
-  static int n = 0;
+  // one process drives one GPU; the count of the first device seen is kept
+  static std::atomic<int> cached{0};
+  int n = cached.load(std::memory_order_relaxed);
   if (!n) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
       n = 148;
+    cached.store(n, std::memory_order_relaxed);
   }
   return n;
 }
