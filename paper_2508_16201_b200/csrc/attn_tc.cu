@@ -535,7 +535,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       const Segment sg = c.sg;
       const int seg_idx = c.seg_idx;
       const int kv_len = clamp_len(p.seq_lens[sg.b], p.max_seq_len);
-      const int n_sub_seq = (kv_len + kTileTokens - 1) / kTileTokens;
       // Visibility of key `tok` for a row of query token t: every key before the window of the n_q
       // new tokens, and inside the window the positions whose bit is set in the row's mask -- bits
       // 0..t for a chain, the token's ancestors and itself for a tree.  Rows no item uses see nothing.
