@@ -30,7 +30,6 @@ struct ScoreParams {
   const int32_t* block_table;
   int32_t* d_status;
   int32_t batch, n_layers, n_q_heads, n_kv_heads, group, qt, sum_text, sum_video;
-  int32_t layer0;                      // first layer of this launch (the grid covers a range of layers)
   int32_t max_blocks, block_tokens;
   float scale_log2;
   ScoreSeq seq[kScoresMaxBatch];
@@ -92,7 +91,7 @@ scores_lse_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   const int b = find_seq(p, blockIdx.x);
   const ScoreSeq sq = p.seq[b];
   const int qtile = blockIdx.x - sq.tile_off;
-  const int g = blockIdx.y, layer = blockIdx.z + p.layer0;
+  const int g = blockIdx.y, layer = blockIdx.z;
   const int i_first = qtile * p.qt;
   const int n_i = min(p.qt, sq.n_text - i_first);               // queries in this tile
   const int rows_valid = n_i * p.group;
@@ -291,7 +290,7 @@ scores_colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
   const int b = find_seq(p, blockIdx.x);
   const ScoreSeq sq = p.seq[b];
   const int kblock = blockIdx.x - sq.tile_off;
-  const int layer = blockIdx.y + p.layer0;
+  const int layer = blockIdx.y;
   // key blocks start on a page boundary at or before the first video token, so that a 64-token
   // TMA box never straddles two cache pages; columns outside the video range are dropped
   const int key0 = (sq.video_start / 64) * 64 + kblock * kKeyTile;   // absolute position of column 0
@@ -526,7 +525,7 @@ scores_colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
   const int b = find_seq(p, blockIdx.x);
   const ScoreSeq sq = p.seq[b];
   const int kblock = blockIdx.x - sq.tile_off;
-  const int layer = blockIdx.y + p.layer0;
+  const int layer = blockIdx.y;
   const int key0 = (sq.video_start / 64) * 64 + kblock * kKeyTile;
   const int n_qt = (sq.n_text + p.qt - 1) / p.qt;
   const int n_units = p.n_kv_heads;
@@ -774,7 +773,7 @@ scores_lse_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
   const int b = find_seq(p, blockIdx.x);
   const ScoreSeq sq = p.seq[b];
   const int qtile = blockIdx.x - sq.tile_off;
-  const int g = blockIdx.y, layer = blockIdx.z + p.layer0;
+  const int g = blockIdx.y, layer = blockIdx.z;
   const int i_first = qtile * p.qt;
   const int n_i = min(p.qt, sq.n_text - i_first);               // queries in this tile
   const int rows_valid = n_i * p.group;
@@ -965,10 +964,12 @@ struct ScoreSetup {
 static int32_t setup_scores(const specvlm_kv_t* target_kv, const void* q_text, const int32_t* text_cu,
                             const int32_t* text_start, const int32_t* video_start, const int32_t* video_len,
                             const int32_t* video_cu, int32_t batch, int32_t n_q_heads, float sm_scale,
-                            int32_t* d_status, ScoreSetup& su) {
+                            int32_t* d_status, ScoreSetup& su, int32_t layer_begin = 0, int32_t layer_end = -1) {
   if (!target_kv) return SPECVLM_ERR_INVALID_ARG;
   su.kv = *target_kv;
   specvlm_kv_t& kv = su.kv;
+  if (layer_end < 0) layer_end = kv.n_layers;
+  if (layer_begin < 0 || layer_end > kv.n_layers || layer_begin > layer_end) return SPECVLM_ERR_INVALID_ARG;
   static const int32_t dummy = 0;
   if (!kv.seq_lens) kv.seq_lens = &dummy;             // lengths come from text_start / text_cu here
   int32_t rc = validate_kv(&kv, batch, false);
@@ -1004,7 +1005,6 @@ static int32_t setup_scores(const specvlm_kv_t* target_kv, const void* q_text, c
   p.d_status = d_status;
   p.batch = batch;
   p.n_layers = kv.n_layers;
-  p.layer0 = 0;
   p.n_q_heads = n_q_heads;
   p.n_kv_heads = kv.n_kv_heads;
   p.group = group;
@@ -1014,8 +1014,8 @@ static int32_t setup_scores(const specvlm_kv_t* target_kv, const void* q_text, c
   p.block_tokens = kv.block_tokens;
   p.scale_log2 = sm_scale * kLog2e;
   su.p2 = p;
-  su.layer_begin = 0;
-  su.layer_count = kv.n_layers;
+  su.layer_begin = layer_begin;
+  su.layer_count = layer_end - layer_begin;
   su.finish = true;
   su.n_row_tiles = su.n_key_blocks = 0;
   for (int b = 0; b < batch; ++b) {
@@ -1035,18 +1035,27 @@ static int32_t setup_scores(const specvlm_kv_t* target_kv, const void* q_text, c
     su.n_key_blocks += (s.video_start % 64 + s.n_video + kKeyTile - 1) / kKeyTile;
   }
 
-  rc = encode_kv_map(&su.tk, &kv, kv.k, 64);
+  // The kernels count layers from 0 (one code for a range and for the whole problem): the K map, the
+  // Q map and the query pointer start at the range's first layer; the callers offset the row
+  // statistics and the partial sums the same way.
+  specvlm_kv_t kv_range = kv;
+  kv_range.n_layers = su.layer_count > 0 ? su.layer_count : 1;
+  void* const k_range = static_cast<uint8_t*>(kv.k) + (size_t)layer_begin * kv.stride_layer * 2;
+  rc = encode_kv_map(&su.tk, &kv_range, k_range, 64);
   if (rc != SPECVLM_OK) return rc;
   encode_tiled_fn enc = get_encode_tiled();
   if (!enc) return SPECVLM_ERR_CUDA;
   const int D = kv.head_dim;
   const cuuint64_t dims[5] = {(cuuint64_t)D, (cuuint64_t)group, (cuuint64_t)kv.n_kv_heads,
-                              (cuuint64_t)p.sum_text, (cuuint64_t)kv.n_layers};
+                              (cuuint64_t)p.sum_text, (cuuint64_t)kv_range.n_layers};
   const cuuint64_t strides[4] = {(cuuint64_t)D * 2, (cuuint64_t)group * D * 2, (cuuint64_t)n_q_heads * D * 2,
                                  (cuuint64_t)p.sum_text * n_q_heads * D * 2};
   const cuuint32_t box[5] = {64u, (cuuint32_t)group, 1u, (cuuint32_t)p.qt, 1u};
   const cuuint32_t estr[5] = {1u, 1u, 1u, 1u, 1u};
-  if (enc(&su.tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(q_text), dims, strides, box, estr,
+  const __nv_bfloat16* const q_range =
+      static_cast<const __nv_bfloat16*>(q_text) + (size_t)layer_begin * p.sum_text * n_q_heads * D;
+  su.p1.q = su.p2.q = q_range;
+  if (enc(&su.tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<__nv_bfloat16*>(q_range), dims, strides, box, estr,
           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return SPECVLM_ERR_CUDA;
@@ -1101,9 +1110,8 @@ static int32_t launch_colsum(ScoreSetup& su, float* scores, cudaStream_t st) {
     k<<<dim3((unsigned)su.n_key_blocks, (unsigned)su.layer_count), kColsumThreads, SMEM, st>>>(su.tk, su.tq, su.p2);
     rc = launch_status();
   }
-  if (rc != SPECVLM_OK || !su.finish) return rc;
-  scores_finish_kernel<<<(unsigned)((su.p2.sum_video + 255) / 256), 256, 0, st>>>(su.p2, scores);
-  return launch_status();
+  (void)scores;
+  return rc;
 }
 
 }  // namespace specvlm
@@ -1145,33 +1153,35 @@ static int32_t stage1_scores_range(const specvlm_kv_t* target_kv, const void* q_
   if (reinterpret_cast<uintptr_t>(ws) & 255u) return SPECVLM_ERR_INVALID_ARG;
   ScoreSetup su;
   int32_t rc = setup_scores(target_kv, q_text, text_cu, text_start, video_start, video_len, video_cu, batch,
-                            n_q_heads, sm_scale, d_status, su);
+                            n_q_heads, sm_scale, d_status, su, layer_begin, layer_end);
   if (rc != SPECVLM_OK) return rc;
-  if (layer_begin < 0 || layer_end > su.kv.n_layers || layer_begin > layer_end) return SPECVLM_ERR_INVALID_ARG;
   size_t lse_bytes, partial_bytes;
   ws_layout(su.kv.n_layers, n_q_heads, su.p1.sum_text, su.p1.sum_video, lse_bytes, partial_bytes);
   if (ws_bytes < lse_bytes + partial_bytes) return SPECVLM_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool d128 = su.kv.head_dim == 128;
-  su.layer_begin = layer_begin;
-  su.layer_count = layer_end - layer_begin;
-  su.finish = finish;
-  su.p1.layer0 = su.p2.layer0 = layer_begin;
-  su.p2.partial = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + lse_bytes);
-  if (su.layer_count == 0) {
-    // nothing to rate: only the final reduction, if asked for
-    if (!finish) return SPECVLM_OK;
-    scores_finish_kernel<<<(unsigned)((su.p2.sum_video + 255) / 256), 256, 0, st>>>(su.p2, scores);
-    return launch_status();
-  }
-  if (row_lse_or_null) {
-    su.p2.lse = const_cast<float*>(row_lse_or_null);
-  } else {
-    su.p1.lse = su.p2.lse = static_cast<float*>(ws);
-    rc = d128 ? launch_lse<128>(su, st) : launch_lse<64>(su, st);
+  su.finish = false;                       // the reduction below runs over all layers, not the range
+  float* const partial_all = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + lse_bytes);
+  if (su.layer_count > 0) {
+    // the range's slices of the row statistics and of the per-layer partial sums
+    const size_t lse_off = (size_t)layer_begin * su.p1.sum_text * n_q_heads;
+    if (row_lse_or_null) {
+      su.p2.lse = const_cast<float*>(row_lse_or_null) + lse_off;
+    } else {
+      su.p1.lse = su.p2.lse = static_cast<float*>(ws) + lse_off;
+      rc = d128 ? launch_lse<128>(su, st) : launch_lse<64>(su, st);
+      if (rc != SPECVLM_OK) return rc;
+    }
+    su.p2.partial = partial_all + (size_t)layer_begin * su.p1.sum_video;
+    rc = d128 ? launch_colsum<128>(su, scores, st) : launch_colsum<64>(su, scores, st);
     if (rc != SPECVLM_OK) return rc;
   }
-  return d128 ? launch_colsum<128>(su, scores, st) : launch_colsum<64>(su, scores, st);
+  if (!finish) return SPECVLM_OK;
+  ScoreParams pf = su.p2;                  // all layers' partial sums, in layer order
+  pf.partial = partial_all;
+  pf.n_layers = su.kv.n_layers;
+  scores_finish_kernel<<<(unsigned)((pf.sum_video + 255) / 256), 256, 0, st>>>(pf, scores);
+  return launch_status();
 }
 
 extern "C" int32_t specvlm_stage1_scores(const specvlm_kv_t* target_kv, const void* q_text,
