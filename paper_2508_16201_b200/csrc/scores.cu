@@ -640,20 +640,33 @@ scores_colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
     const int key_l = quad * 32 + lane;         // this thread's key inside the block
     const int et = ((warp - 2) & 3) * 32 + lane;   // 0..127 inside the group: used to stage the row LSEs
     float* const lse_g = lse_sm + grp * 256;    // this group's two staging buffers of 128 rows
-    // -lse (log2 units) of row `et` of tile `tile`; -inf for rows past the valid ones, whose
-    // exponentials then vanish
-    auto lse_fetch = [&](int tile) -> float {
-      if (tile >= n_tiles) return 0.f;
-      const int u = tile / n_qt, t = tile - u * n_qt;
-      const int rows_valid = min(p.qt, sq.n_text - t * p.qt) * p.group;
-      if (et >= rows_valid) return -INFINITY;
-      const int il = et / p.group, hg = et - il * p.group;
-      return -__ldg(p.lse + ((size_t)layer * p.sum_text + sq.text_off + t * p.qt + il) * p.n_q_heads + u * p.group + hg) *
-             kLog2e;
+    // -lse (log2 units) of row `et` of the tile (KV head fu, row tile ft); -inf for rows past the valid
+    // ones, whose exponentials then vanish.  (fu, ft) walk this group's tiles ahead of the loop
+    // below: no division per tile, and the address is two multiply-adds off a fixed base.
+    const int il = et / p.group, hg = et - il * p.group;
+    const float* const lse_row =
+        p.lse + ((size_t)layer * p.sum_text + sq.text_off + il) * p.n_q_heads + hg;
+    int fu = 0, ft = grp;                       // the tile the next lse_fetch() is for
+    while (ft >= n_qt) {
+      ft -= n_qt;
+      ++fu;
+    }
+    auto lse_fetch = [&]() -> float {
+      float v = 0.f;
+      if (fu < n_units) {
+        const int rows_valid = min(p.qt, sq.n_text - ft * p.qt) * p.group;
+        v = et < rows_valid ? -__ldg(lse_row + (size_t)(ft * p.qt) * p.n_q_heads + fu * p.group) * kLog2e : -INFINITY;
+      }
+      ft += NG;                                 // this group's next tile
+      while (ft >= n_qt) {
+        ft -= n_qt;
+        ++fu;
+      }
+      return v;
     };
     uint64_t acc2[4] = {0ull, 0ull, 0ull, 0ull};   // four chains of pairs for instruction-level parallelism
     bool alive = true;
-    float lv = lse_fetch(grp);
+    float lv = lse_fetch();
     int n = 0;
     for (int it = grp; it < n_tiles; it += NG, ++n) {
       const int buf = grp;
@@ -662,7 +675,7 @@ scores_colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
       // one barrier per tile: the buffer written here was last read two tiles ago, before the
       // previous tile's barrier
       asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory");
-      lv = lse_fetch(it + NG);                  // in flight during this tile's exponentials
+      lv = lse_fetch();                         // the next tile's: in flight during this tile's exponentials
       if (alive && !mbar_wait(bar_tfull + 8 * buf, (it / NG) & 1, abort_flag)) alive = false;
       alive = __all_sync(0xffffffffu, alive);   // warp-uniform: the TMEM loads below are warp-collective
       if (!alive) continue;                     // keep taking part in the barrier above
