@@ -68,3 +68,16 @@ def test_host_validation_without_gpu():
     rc = L.specvlm_accept(0x1000, 0x1000, 1, 4, 1024, 0x1000, 0x1000, None, 0x1000, 8, None)
     assert rc == specvlm.ERR_WORKSPACE_TOO_SMALL
     assert L.specvlm_accept_workspace_bytes(1, 4, 1024) >= 5 * 8
+    # rating a range of layers: a range outside the cache's layers is refused before anything runs
+    kv.head_dim = 128
+    kv.stride_token = 128
+    kv.stride_head = kv.stride_block = kv.stride_layer = 128 * 128
+    kv.n_layers = 4
+    common = (ctypes.byref(kv), 0x1000, i32(0, 8), i32(64), i32(0), i32(64), i32(0, 64), 1, 4, 0.1, None, 0x1000,
+              0x1000, 1 << 30)
+    assert L.specvlm_stage1_scores_layers(*common, 3, 5, 0, None, None) == specvlm.ERR_INVALID_ARG
+    assert L.specvlm_stage1_scores_layers(*common, 2, 1, 0, None, None) == specvlm.ERR_INVALID_ARG
+    # tree verification: more nodes than the ancestor masks hold
+    rc = L.specvlm_verify_tree_attn(ctypes.byref(kv), 0x1000, 0x1000, 1, 4, 33, 0.1, 0x1000, None, 0x1000, 1 << 30,
+                                    None, None)
+    assert rc == specvlm.ERR_UNSUPPORTED_SHAPE
