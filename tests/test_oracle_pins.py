@@ -5,6 +5,7 @@ import os
 
 import numpy as np
 import pytest
+import scipy.special
 import torch
 
 import oracle
@@ -90,7 +91,9 @@ def test_scores_invariants_and_library():
     G = M[..., vs:vs + nv]
     ref = G.mean(dim=(0, 1, 2)).numpy()
     np.testing.assert_allclose(a, ref, rtol=1e-11)
-    np.testing.assert_allclose(lse, torch.logsumexp(s, dim=-1).numpy(), rtol=1e-12)
+    # (scipy's routine: torch.logsumexp's first call in a process now and then returns one thread's
+    # block of rows 4e-10 off, and the exact values when called again)
+    np.testing.assert_allclose(lse, scipy.special.logsumexp(s.numpy(), axis=-1), rtol=1e-12)
     # the other reading (softmax over video keys only) is a different function
     a2 = oracle.stage1_scores(bits(q), bits(k), vs, nv, vs + nv, scale, video_only=True)
     np.testing.assert_allclose(a2.sum(), 1.0, rtol=1e-12)
