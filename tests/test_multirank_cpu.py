@@ -3,6 +3,7 @@ is an independent replica of the path; step time = the slowest rank's; value = a
 over that time) and its reference arm's rule that only rank 0 prints."""
 import json
 import os
+import socket
 import subprocess
 import sys
 import textwrap
@@ -10,8 +11,14 @@ import textwrap
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
-def _run_ranks(code, world=2, port=29541):
-    procs = []
+def _free_port():
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _run_ranks(code, world=2):
+    procs, port = [], _free_port()
     for r in range(world):
         env = dict(os.environ, RANK=str(r), WORLD_SIZE=str(world), LOCAL_RANK=str(r), MASTER_ADDR="127.0.0.1",
                    MASTER_PORT=str(port), PYTHONPATH=ROOT)
