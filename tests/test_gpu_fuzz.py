@@ -20,6 +20,14 @@ pytestmark = pytest.mark.gpu
 
 # SPECVLM_FUZZ_SCALE=10 runs ten times as many draws (a bug hunt, not the regular suite)
 SCALE = int(os.environ.get("SPECVLM_FUZZ_SCALE", "1"))
+# SPECVLM_FUZZ_FIRST=100000 starts the seeds elsewhere: another set of draws
+FIRST = int(os.environ.get("SPECVLM_FUZZ_FIRST", "0"))
+
+
+def _seeds(n):
+    return range(FIRST, FIRST + n * SCALE)
+
+
 GROUPS = [(4, 4), (8, 2), (28, 4), (40, 8), (64, 8), (16, 1), (12, 2)]     # (query heads, KV heads)
 
 
@@ -37,7 +45,7 @@ def _lens(rng, batch, lo, hi, n_q):
     return out
 
 
-@pytest.mark.parametrize("seed", range(24 * SCALE))
+@pytest.mark.parametrize("seed", _seeds(24))
 def test_fuzz_chain_attention(seed):
     rng = np.random.default_rng(1000 + seed)
     Hq, Hkv = GROUPS[int(rng.integers(0, len(GROUPS)))]
@@ -52,7 +60,7 @@ def test_fuzz_chain_attention(seed):
     _run_attn(L, Hq, Hkv, D, lens, gamma, paged=bool(rng.integers(0, 2)), seed=2000 + seed, poison=True)
 
 
-@pytest.mark.parametrize("seed", range(16 * SCALE))
+@pytest.mark.parametrize("seed", _seeds(16))
 def test_fuzz_tree_attention(seed):
     rng = np.random.default_rng(3000 + seed)
     Hq, Hkv = GROUPS[int(rng.integers(0, len(GROUPS)))]
@@ -83,7 +91,7 @@ def test_fuzz_tree_attention(seed):
     assert worst <= ATTN_TOL, f"row rel err {worst}"
 
 
-@pytest.mark.parametrize("seed", range(6 * SCALE))
+@pytest.mark.parametrize("seed", _seeds(6))
 def test_fuzz_scores(seed):
     rng = np.random.default_rng(5000 + seed)
     Hq, Hkv = GROUPS[int(rng.integers(0, len(GROUPS)))]
@@ -98,7 +106,7 @@ def test_fuzz_scores(seed):
                  prefix=prefix)
 
 
-@pytest.mark.parametrize("seed", range(6 * SCALE))
+@pytest.mark.parametrize("seed", _seeds(6))
 def test_fuzz_select(seed):
     """Stage I + II on random score vectors with planted ties; fixed count and Top-P count."""
     rng = np.random.default_rng(7000 + seed)
@@ -126,7 +134,7 @@ def test_fuzz_select(seed):
         assert np.array_equal(got_p[kept_cu[b]:kept_cu[b + 1]], ref), f"top-p sequence {b}"
 
 
-@pytest.mark.parametrize("seed", range(6 * SCALE))
+@pytest.mark.parametrize("seed", _seeds(6))
 def test_fuzz_gather(seed):
     from gpu_util import host_view
     rng = np.random.default_rng(8000 + seed)
@@ -157,7 +165,7 @@ def test_fuzz_gather(seed):
         assert np.array_equal(dk[b][:, :, :n], rk) and np.array_equal(dv[b][:, :, :n], rv), f"sequence {b}"
 
 
-@pytest.mark.parametrize("seed", range(6 * SCALE))
+@pytest.mark.parametrize("seed", _seeds(6))
 def test_fuzz_accept_chain_and_tree(seed):
     rng = np.random.default_rng(9000 + seed)
     batch, gamma = int(rng.integers(1, 9)), int(rng.integers(0, 9))
@@ -189,7 +197,7 @@ def test_fuzz_accept_chain_and_tree(seed):
         assert path[b].cpu().tolist() == rpath + [-1] * (n_nodes - rn)
 
 
-@pytest.mark.parametrize("seed", range(4 * SCALE))
+@pytest.mark.parametrize("seed", _seeds(4))
 def test_fuzz_baseline_selectors(seed):
     rng = np.random.default_rng(9500 + seed)
     batch = int(rng.integers(1, 5))
@@ -208,7 +216,7 @@ def test_fuzz_baseline_selectors(seed):
             assert np.array_equal(kept[kept_cu[b]:kept_cu[b] + len(ref)], ref), f"mode {mode} sequence {b}"
 
 
-@pytest.mark.parametrize("seed", range(6 * SCALE))
+@pytest.mark.parametrize("seed", _seeds(6))
 def test_fuzz_cache_append_rollback_compact(seed):
     """append -> rollback lengths, and tree compaction along a random accepted path, bit for bit."""
     from gpu_util import host_view
