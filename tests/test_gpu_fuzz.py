@@ -106,6 +106,34 @@ def test_fuzz_scores(seed):
                  prefix=prefix)
 
 
+@pytest.mark.parametrize("seed", _seeds(4))
+def test_fuzz_scores_by_layer_ranges(seed):
+    """random cuts of the layers (empty ranges included) give the bits of the single call"""
+    rng = np.random.default_rng(5500 + seed)
+    Hq, Hkv = GROUPS[int(rng.integers(0, len(GROUPS)))]
+    D = 64 if rng.random() < 0.3 else 128
+    L = int(rng.integers(2, 7))
+    batch = int(rng.integers(1, 4))
+    nv = [int(rng.integers(20, 400)) for _ in range(batch)]
+    nt = [int(rng.integers(1, 100)) for _ in range(batch)]
+    prefix = [int(rng.integers(0, 40)) for _ in range(batch)]
+    cache, _, _ = make_cache(L, Hkv, D, [p + v + t for p, v, t in zip(prefix, nv, nt)],
+                             paged=bool(rng.integers(0, 2)), seed=5600 + seed)
+    text_cu = [0] + np.cumsum(nt).tolist()
+    video_cu = [0] + np.cumsum(nv).tolist()
+    q = synth.randn_bf16((L, text_cu[-1], Hq, D), "cuda", 5600 + seed, "Qtext")
+    args = (text_cu, [p + v for p, v in zip(prefix, nv)], prefix, nv, video_cu, 1.0 / math.sqrt(D))
+    whole = specvlm.stage1_scores(cache, q, *args)
+    cuts = [0] + sorted(int(c) for c in rng.integers(0, L + 1, size=int(rng.integers(0, 4)))) + [L]
+    ws = torch.full((specvlm.stage1_scores_workspace_bytes(cache, text_cu, nv, Hq),), 0xFF, dtype=torch.uint8,
+                    device="cuda")
+    out = torch.full((video_cu[-1],), float("nan"), device="cuda")
+    for i, (a, b) in enumerate(zip(cuts[:-1], cuts[1:])):
+        specvlm.stage1_scores_layers(cache, q, *args, out, ws, a, b, finish=(i == len(cuts) - 2))
+    torch.cuda.synchronize()
+    assert torch.equal(out, whole), cuts
+
+
 @pytest.mark.parametrize("seed", _seeds(6))
 def test_fuzz_select(seed):
     """Stage I + II on random score vectors with planted ties; fixed count and Top-P count."""
