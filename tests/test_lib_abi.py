@@ -81,3 +81,21 @@ def test_host_validation_without_gpu():
     rc = L.specvlm_verify_tree_attn(ctypes.byref(kv), 0x1000, 0x1000, 1, 4, 33, 0.1, 0x1000, None, 0x1000, 1 << 30,
                                     None, None)
     assert rc == specvlm.ERR_UNSUPPORTED_SHAPE
+
+
+def test_missing_library_raises_and_package_is_oracle_free(monkeypatch, tmp_path):
+    """No fallback: with the library file absent every call through the binding raises; and the
+    package's sources neither import nor include anything of the oracle."""
+    monkeypatch.setattr(specvlm, "_lib", None)
+    monkeypatch.setattr(specvlm, "LIB_PATH", str(tmp_path / "libspecvlm.so"))
+    with pytest.raises(RuntimeError, match="missing"):
+        specvlm.lib()
+    with pytest.raises(RuntimeError, match="missing"):
+        specvlm.accept_workspace_bytes(1, 4, 1024)
+    pkg = os.path.dirname(specvlm.__file__)
+    for root, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h", ".cpp")):
+                with open(os.path.join(root, f)) as fh:
+                    src = fh.read()
+                assert not re.search(r"^\s*(import|from)\s+oracle|#include[^\n]*oracle|oracle[./]", src, re.M), f
