@@ -64,421 +64,17 @@ __device__ __forceinline__ void load_key_tile(const CUtensorMap* tm_k, const Sco
                   policy);
   }
 }
-// byte offset of (row r of a 128-row tile, 16-byte chunk c16); halves of 64 channels are 16 KB apart
-template <int D>
-__device__ __forceinline__ uint32_t tile128_offset(int r, int c16) {
-  return static_cast<uint32_t>((c16 >> 3) * (kKeyTile * 128) + r * 128 + (((c16 & 7) ^ (r & 7)) << 4));
-}
 
-// ---------------------------------------------------------------------------------------------
-// Pass 1.  CTA = (row tile, KV head, layer).  8 compute warps = 4 (32 rows each) x 2 (64 of the
-// tile's 128 keys each); warp 8 streams K tiles.  Q fragments stay in registers.
-// ---------------------------------------------------------------------------------------------
-template <int D, int STAGES>
-__global__ void __launch_bounds__(288, 1)
-scores_lse_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ ScoreParams p) {
-  constexpr int TILE_BYTES = kKeyTile * D * 2;
-  constexpr int KSTEPS = D / 16;
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t raw_addr = smem_u32(smem_raw);
-  const uint32_t base = (raw_addr + 1023u) & ~1023u;
-  uint8_t* const smem = smem_raw + (base - raw_addr);
-  const uint32_t bar_full = base + STAGES * TILE_BYTES;
-  const uint32_t bar_empty = bar_full + 8 * STAGES;
-  volatile int* const abort_flag =
-      reinterpret_cast<volatile int*>(smem + STAGES * TILE_BYTES + 16 * STAGES);
-  float* const red = reinterpret_cast<float*>(smem + STAGES * TILE_BYTES + 16 * STAGES + 16);  // [2][128][2]
-
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int b = find_seq(p, blockIdx.x);
-  const ScoreSeq sq = p.seq[b];
-  const int qtile = blockIdx.x - sq.tile_off;
-  const int g = blockIdx.y, layer = blockIdx.z;
-  const int i_first = qtile * p.qt;
-  const int n_i = min(p.qt, sq.n_text - i_first);               // queries in this tile
-  const int rows_valid = n_i * p.group;
-  const int key_end = sq.text_start + i_first + n_i;            // keys [0, key_end) are needed
-  const int n_kt = (key_end + kKeyTile - 1) / kKeyTile;
-
-  if (tid == 0) {
-    for (int s = 0; s < STAGES; ++s) {
-      mbar_init(bar_full + 8 * s, 1);
-      mbar_init(bar_empty + 8 * s, 8);
-    }
-    *abort_flag = 0;
-    mbar_fence_init();
-  }
-  __syncthreads();
-
-  if (warp == 8) {
-    if (lane == 0) {
-      tma_prefetch_desc(&tm_k);
-      const uint64_t policy = l2_policy_evict_last();           // K is re-read by the other row tiles
-      int issued = 0;
-      bool ok = true;
-      for (int i = 0; i < n_kt; ++i) {
-        const int s = i % STAGES;
-        if (i >= STAGES) ok = mbar_wait(bar_empty + 8 * s, ((i / STAGES) - 1) & 1, abort_flag);
-        if (!ok) break;
-        mbar_arrive_expect_tx(bar_full + 8 * s, TILE_BYTES);
-        load_key_tile<D>(&tm_k, p, b, g, layer, i * kKeyTile, base + s * TILE_BYTES, bar_full + 8 * s,
-                         policy);
-        issued = i + 1;
-      }
-      if (!ok) {
-        if (p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
-        for (int i = issued > STAGES ? issued - STAGES : 0; i < issued; ++i) {
-          const uint64_t t0 = global_timer_ns();
-          while (!mbar_try_wait(bar_full + 8 * (i % STAGES), (i / STAGES) & 1) &&
-                 global_timer_ns() - t0 < kWaitLimitNs) {
-          }
-        }
-      }
-    }
-    return;
-  }
-
-  const int wm = warp >> 1, wn = warp & 1;        // 4 row groups x 2 key halves
-  const int col = (lane & 3) * 2;
-  // the four rows this thread holds: mt*16 + (lane>>2) + {0, 8}
-  uint32_t qf[2][KSTEPS][4];
-  int lim[2][2];
-#pragma unroll
-  for (int mt = 0; mt < 2; ++mt) {
-#pragma unroll
-    for (int hf = 0; hf < 2; ++hf) {
-      const int r = wm * 32 + mt * 16 + (lane >> 2) + hf * 8;
-      const __nv_bfloat16* qp = nullptr;
-      lim[mt][hf] = 0;
-      if (r < rows_valid) {
-        const int il = r / p.group, hg = r - il * p.group;
-        qp = p.q + (((size_t)layer * p.sum_text + sq.text_off + i_first + il) * p.n_q_heads +
-                    g * p.group + hg) * D;
-        lim[mt][hf] = sq.text_start + i_first + il + 1;
-      }
-#pragma unroll
-      for (int ks = 0; ks < KSTEPS; ++ks) {
-        qf[mt][ks][hf] = qp ? *reinterpret_cast<const uint32_t*>(qp + ks * 16 + col) : 0u;
-        qf[mt][ks][2 + hf] = qp ? *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8 + col) : 0u;
-      }
-    }
-  }
-  float m[2][2], l[2][2];
-#pragma unroll
-  for (int mt = 0; mt < 2; ++mt) m[mt][0] = m[mt][1] = -INFINITY, l[mt][0] = l[mt][1] = 0.f;
-
-  const int mi = lane >> 3, r8 = lane & 7;
-  bool alive = true;
-  for (int i = 0; i < n_kt; ++i) {
-    const int s = i % STAGES;
-    if (!mbar_wait(bar_full + 8 * s, (i / STAGES) & 1, abort_flag)) {
-      alive = false;
-      break;
-    }
-    const uint32_t k_base = base + s * TILE_BYTES;
-    const int key0 = i * kKeyTile + wn * 64;
-    if (key0 < key_end) {
-      float sc[2][8][4];
-#pragma unroll
-      for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt) sc[mt][nt][0] = sc[mt][nt][1] = sc[mt][nt][2] = sc[mt][nt][3] = 0.f;
-#pragma unroll
-      for (int ks = 0; ks < KSTEPS; ++ks) {
-#pragma unroll
-        for (int np = 0; np < 4; ++np) {       // 16 keys per ldmatrix.x4
-          uint32_t b0, b1, b2, b3;
-          const int kr = wn * 64 + np * 16 + (mi >> 1) * 8 + r8;
-          ldmatrix_x4(k_base + tile128_offset<D>(kr, 2 * ks + (mi & 1)), b0, b1, b2, b3);
-#pragma unroll
-          for (int mt = 0; mt < 2; ++mt) {
-            mma_bf16_16816(sc[mt][2 * np], qf[mt][ks], b0, b1);
-            mma_bf16_16816(sc[mt][2 * np + 1], qf[mt][ks], b2, b3);
-          }
-        }
-      }
-      const bool need_mask = key0 + 64 > sq.text_start + i_first + 1;   // tile reaches past the first limit
-#pragma unroll
-      for (int mt = 0; mt < 2; ++mt) {
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-          float mx = -INFINITY;
-#pragma unroll
-          for (int nt = 0; nt < 8; ++nt) {
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-              float v = sc[mt][nt][hf * 2 + e] * p.scale_log2;
-              if (need_mask && key0 + nt * 8 + col + e >= lim[mt][hf]) v = -INFINITY;
-              sc[mt][nt][hf * 2 + e] = v;
-              mx = fmaxf(mx, v);
-            }
-          }
-          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-          const float mn = fmaxf(m[mt][hf], mx);
-          const float mu = mn == -INFINITY ? 0.f : mn;
-          float ps = 0.f;
-#pragma unroll
-          for (int nt = 0; nt < 8; ++nt) ps += fast_exp2(sc[mt][nt][hf * 2] - mu) + fast_exp2(sc[mt][nt][hf * 2 + 1] - mu);
-          l[mt][hf] = l[mt][hf] * fast_exp2(m[mt][hf] - mu) + ps;
-          m[mt][hf] = mn;
-        }
-      }
-    }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(bar_empty + 8 * s);
-  }
-  // combine the quad's partial sums, then the two key halves
-#pragma unroll
-  for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-    for (int hf = 0; hf < 2; ++hf) {
-      l[mt][hf] += __shfl_xor_sync(0xffffffffu, l[mt][hf], 1);
-      l[mt][hf] += __shfl_xor_sync(0xffffffffu, l[mt][hf], 2);
-    }
-  if ((lane & 3) == 0) {
-#pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {
-        const int r = wm * 32 + mt * 16 + (lane >> 2) + hf * 8;
-        red[(wn * 128 + r) * 2] = m[mt][hf];
-        red[(wn * 128 + r) * 2 + 1] = l[mt][hf];
-      }
-  }
-  asm volatile("bar.sync 1, 256;" ::: "memory");
-  if (!alive || *abort_flag) {
-    if (tid == 0 && p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
-    return;
-  }
-  if (tid < rows_valid) {
-    const float ma = red[tid * 2], la = red[tid * 2 + 1];
-    const float mb = red[(128 + tid) * 2], lb2 = red[(128 + tid) * 2 + 1];
-    const float M = fmaxf(ma, mb);
-    const float L = la * fast_exp2(ma - M) + lb2 * fast_exp2(mb - M);
-    const int il = tid / p.group, hg = tid - il * p.group;
-    p.lse[((size_t)layer * p.sum_text + sq.text_off + i_first + il) * p.n_q_heads + g * p.group + hg] =
-        (M + log2f(L)) * kLn2;
-  }
-}
-
-// ---------------------------------------------------------------------------------------------
-// Pass 2.  CTA = (block of 128 video keys, layer); it loops over the layer's KV heads and, for
-// each, over all row tiles of the sequence.  8 compute warps = 2 (64 rows each) x 4 (32 keys
-// each); a warp keeps its K fragments in registers for the whole head and its 8 column sums in
-// registers for the whole layer.  Warp 8 streams the K block of each head and the Q row tiles.
-// ---------------------------------------------------------------------------------------------
-template <int D, int STAGES>
-__global__ void __launch_bounds__(288, 1)
-scores_colsum_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q,
-                     const __grid_constant__ ScoreParams p) {
-  constexpr int TILE_BYTES = kKeyTile * D * 2;     // K block and Q tile alike (128 rows)
-  constexpr int KSTEPS = D / 16;
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t raw_addr = smem_u32(smem_raw);
-  const uint32_t base = (raw_addr + 1023u) & ~1023u;
-  uint8_t* const smem = smem_raw + (base - raw_addr);
-  const uint32_t k_sm = base;                                    // K block
-  const uint32_t q_sm = base + TILE_BYTES;                       // Q ring
-  const uint32_t bar_qfull = base + (STAGES + 1) * TILE_BYTES;
-  const uint32_t bar_qempty = bar_qfull + 8 * STAGES;
-  const uint32_t bar_kfull = bar_qempty + 8 * STAGES;
-  const uint32_t bar_kempty = bar_kfull + 8;
-  uint8_t* const tail = smem + (STAGES + 1) * TILE_BYTES + 16 * STAGES + 16;
-  volatile int* const abort_flag = reinterpret_cast<volatile int*>(tail);
-  float* const red = reinterpret_cast<float*>(tail + 16);        // [128] column sums of row half 1
-
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int b = find_seq(p, blockIdx.x);
-  const ScoreSeq sq = p.seq[b];
-  const int kblock = blockIdx.x - sq.tile_off;
-  const int layer = blockIdx.y;
-  // key blocks start on a page boundary at or before the first video token, so that a 64-token
-  // TMA box never straddles two cache pages; columns outside the video range are dropped
-  const int key0 = (sq.video_start / 64) * 64 + kblock * kKeyTile;   // absolute position of column 0
-  const int n_qt = (sq.n_text + p.qt - 1) / p.qt;
-  const int n_units = p.n_kv_heads;
-
-  if (tid == 0) {
-    for (int s = 0; s < STAGES; ++s) {
-      mbar_init(bar_qfull + 8 * s, 1);
-      mbar_init(bar_qempty + 8 * s, 8);
-    }
-    mbar_init(bar_kfull, 1);
-    mbar_init(bar_kempty, 8);
-    *abort_flag = 0;
-    mbar_fence_init();
-  }
-  __syncthreads();
-
-  if (warp == 8) {
-    if (lane == 0) {
-      tma_prefetch_desc(&tm_k);
-      tma_prefetch_desc(&tm_q);
-      const uint64_t pol_k = l2_policy_evict_first();
-      const uint64_t pol_q = l2_policy_evict_last();             // Q is re-read by every key block
-      bool ok = true;
-      int qi = 0;                                                 // running Q-tile counter
-      for (int u = 0; u < n_units && ok; ++u) {
-        if (u > 0) ok = mbar_wait(bar_kempty, (u - 1) & 1, abort_flag);
-        if (!ok) break;
-        mbar_arrive_expect_tx(bar_kfull, TILE_BYTES);
-        load_key_tile<D>(&tm_k, p, b, u, layer, key0, k_sm, bar_kfull, pol_k);
-        for (int t = 0; t < n_qt && ok; ++t, ++qi) {
-          const int s = qi % STAGES;
-          if (qi >= STAGES) ok = mbar_wait(bar_qempty + 8 * s, ((qi / STAGES) - 1) & 1, abort_flag);
-          if (!ok) break;
-          // box = (64 channels, group heads, 1 KV head, QT queries, 1 layer); rows land in the
-          // order r = query * group + head.  When group does not divide 128 the box has fewer
-          // than 128 rows; the barrier expects exactly the box bytes.
-          mbar_arrive_expect_tx(bar_qfull + 8 * s, (D / 64) * p.qt * p.group * 128);
-#pragma unroll
-          for (int h = 0; h < D / 64; ++h)
-            tma_load_5d(q_sm + s * TILE_BYTES + h * (kKeyTile * 128), &tm_q, bar_qfull + 8 * s, h * 64, 0,
-                        u, sq.text_off + t * p.qt, layer, pol_q);
-        }
-      }
-      if (!ok) {
-        // a wait expired: report, then stay until the copies already issued have landed
-        if (p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
-        const uint64_t t0 = global_timer_ns();
-        for (int i = qi > STAGES ? qi - STAGES : 0; i < qi; ++i)
-          while (!mbar_try_wait(bar_qfull + 8 * (i % STAGES), (i / STAGES) & 1) &&
-                 global_timer_ns() - t0 < kWaitLimitNs) {
-          }
-      }
-    }
-    return;
-  }
-
-  const int wm = warp >> 2, wn = warp & 3;          // 2 row halves x 4 key quarters
-  const int col = (lane & 3) * 2;
-  const int mi = lane >> 3, r8 = lane & 7;
-  float colsum[4][2];
-#pragma unroll
-  for (int nt = 0; nt < 4; ++nt) colsum[nt][0] = colsum[nt][1] = 0.f;
-
-  bool alive = true;
-  int qi = 0;
-  for (int u = 0; u < n_units && alive; ++u) {
-    if (!mbar_wait(bar_kfull, u & 1, abort_flag)) {
-      alive = false;
-      break;
-    }
-    uint32_t kf[KSTEPS][4][2];                      // B fragments: 4 n-tiles of 8 keys
-#pragma unroll
-    for (int ks = 0; ks < KSTEPS; ++ks) {
-#pragma unroll
-      for (int np = 0; np < 2; ++np) {
-        const int kr = wn * 32 + np * 16 + (mi >> 1) * 8 + r8;
-        ldmatrix_x4(k_sm + tile128_offset<D>(kr, 2 * ks + (mi & 1)), kf[ks][2 * np][0], kf[ks][2 * np][1],
-                    kf[ks][2 * np + 1][0], kf[ks][2 * np + 1][1]);
-      }
-    }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(bar_kempty);
-    const float* lse_u = p.lse + ((size_t)layer * p.sum_text + sq.text_off) * p.n_q_heads + u * p.group;
-    for (int t = 0; t < n_qt; ++t, ++qi) {
-      const int s = qi % STAGES;
-      if (!mbar_wait(bar_qfull + 8 * s, (qi / STAGES) & 1, abort_flag)) {
-        alive = false;
-        break;
-      }
-      const uint32_t q_base = q_sm + s * TILE_BYTES;
-      const int rows_valid = min(p.qt, sq.n_text - t * p.qt) * p.group;
-      if (wm * 64 < rows_valid) {
-        float acc[4][4][4];
-#pragma unroll
-        for (int mt = 0; mt < 4; ++mt)
-#pragma unroll
-          for (int nt = 0; nt < 4; ++nt) acc[mt][nt][0] = acc[mt][nt][1] = acc[mt][nt][2] = acc[mt][nt][3] = 0.f;
-#pragma unroll
-        for (int ks = 0; ks < KSTEPS; ++ks) {
-#pragma unroll
-          for (int mt = 0; mt < 4; ++mt) {
-            uint32_t a[4];
-            // A fragment: (rows 0-7, chunk 2ks), (rows 8-15, chunk 2ks), (rows 0-7, 2ks+1), (rows 8-15, 2ks+1)
-            const int qr = wm * 64 + mt * 16 + (mi & 1) * 8 + r8;
-            ldmatrix_x4(q_base + tile128_offset<D>(qr, 2 * ks + (mi >> 1)), a[0], a[1], a[2], a[3]);
-#pragma unroll
-            for (int nt = 0; nt < 4; ++nt) mma_bf16_16816(acc[mt][nt], a, kf[ks][nt][0], kf[ks][nt][1]);
-          }
-        }
-#pragma unroll
-        for (int mt = 0; mt < 4; ++mt) {
-#pragma unroll
-          for (int hf = 0; hf < 2; ++hf) {
-            const int r = wm * 64 + mt * 16 + (lane >> 2) + hf * 8;
-            if (r < rows_valid) {
-              const int il = r / p.group, hg = r - il * p.group;
-              const float lse = __ldg(lse_u + (size_t)(t * p.qt + il) * p.n_q_heads + hg) * kLog2e;
-#pragma unroll
-              for (int nt = 0; nt < 4; ++nt) {
-                colsum[nt][0] += fast_exp2(acc[mt][nt][hf * 2] * p.scale_log2 - lse);
-                colsum[nt][1] += fast_exp2(acc[mt][nt][hf * 2 + 1] * p.scale_log2 - lse);
-              }
-            }
-          }
-        }
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_qempty + 8 * s);
-    }
-  }
-  // rows: reduce over the 8 lanes that share (lane & 3), then over the two row halves
-#pragma unroll
-  for (int nt = 0; nt < 4; ++nt)
-#pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      float v = colsum[nt][e];
-      v += __shfl_xor_sync(0xffffffffu, v, 4);
-      v += __shfl_xor_sync(0xffffffffu, v, 8);
-      v += __shfl_xor_sync(0xffffffffu, v, 16);
-      colsum[nt][e] = v;
-    }
-  if (wm == 1 && lane < 4) {
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
-      red[wn * 32 + nt * 8 + col] = colsum[nt][0];
-      red[wn * 32 + nt * 8 + col + 1] = colsum[nt][1];
-    }
-  }
-  asm volatile("bar.sync 1, 256;" ::: "memory");
-  if (!alive || *abort_flag) {
-    if (tid == 0 && p.d_status) *p.d_status = SPECVLM_ERR_TIMEOUT;
-    return;
-  }
-  if (wm == 0 && lane < 4) {
-    float* out = p.partial + (size_t)layer * p.sum_video + sq.score_off;
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int c = wn * 32 + nt * 8 + col + e;
-        const int j = key0 + c - sq.video_start;        // video token index of column c
-        if (j >= 0 && j < sq.n_video) out[j] = colsum[nt][e] + red[c];
-      }
-    }
-  }
-}
-
-#ifndef SPECVLM_POLY_LSE
-#define SPECVLM_POLY_LSE 2
-#endif
-#ifndef SPECVLM_POLY_COLSUM
-#define SPECVLM_POLY_COLSUM 0
-#endif
-// Of every 8 pairs of logits, this many take their exponential on the FMA pipe (f2_exp2_poly)
-// instead of the special-function unit, which both rating passes nearly saturate.  Measured: the
-// polynomial costs about as many FMA-pipe cycles per value as the unit it relieves (8), so it only
-// pays where issue slots are left over: 2 of 8 in pass 1 (-3 %); none in pass 2, whose four
-// epilogue groups already keep the unit busy (every share made it slower).
-constexpr int kPolyOf8Lse = SPECVLM_POLY_LSE;
-constexpr int kPolyOf8Colsum = SPECVLM_POLY_COLSUM;
+// Of every 8 pairs of logits in pass 1, this many take their exponential on the FMA pipe
+// (f2_exp2_poly) instead of the special-function unit, which both rating passes nearly saturate.
+// Measured: the polynomial costs about as many FMA-pipe cycles per value as the unit it relieves
+// (8), so it only pays where issue slots are left over: 2 of 8 in pass 1 (-3 %); none in pass 2,
+// whose four epilogue groups already keep the unit busy (every share made it slower there).
+constexpr int kPolyOf8Lse = 2;
 
 // ---------------------------------------------------------------------------------------------
 // Pass 2 on the 5th-generation tensor cores.  CTA = (block of 128 video keys, layer), looping over
-// the layer's KV heads and the sequence's row tiles as above, but
+// the layer's KV heads and, for each, over all row tiles of the sequence:
 //   D[key][row] = K_block (A: 128 keys x d, K-major) * Q_tile^T (B: 128 rows x d, K-major)
 // is one chain of tcgen05.mma instructions (M = N = 128, K = 16 each) issued by a single thread,
 // with both operands read straight from the 128-byte-swizzled tiles the TMA wrote and the fp32
@@ -704,11 +300,8 @@ scores_colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
                                      f2_pack(l4.x, l4.y));
           const uint64_t tb = f2_fma(f2_pack(__uint_as_float(v[2 * q + 2]), __uint_as_float(v[2 * q + 3])), sc2,
                                      f2_pack(l4.z, l4.w));
-          // kPolyOf8Colsum of every 8 pairs take the polynomial, spread so both kinds interleave
-          const bool pa = ((q & 7) * kPolyOf8Colsum) / 8 != (((q & 7) + 1) * kPolyOf8Colsum) / 8;
-          const bool pb = (((q + 1) & 7) * kPolyOf8Colsum) / 8 != ((((q + 1) & 7) + 1) * kPolyOf8Colsum) / 8;
-          acc2[q & 3] = f2_add(acc2[q & 3], pa ? f2_exp2_poly(ta) : f2_exp2_sfu(ta));
-          acc2[(q + 1) & 3] = f2_add(acc2[(q + 1) & 3], pb ? f2_exp2_poly(tb) : f2_exp2_sfu(tb));
+          acc2[q & 3] = f2_add(acc2[q & 3], f2_exp2_sfu(ta));
+          acc2[(q + 1) & 3] = f2_add(acc2[(q + 1) & 3], f2_exp2_sfu(tb));
         }
       }
     }
@@ -1089,56 +682,28 @@ static int32_t setup_scores(const specvlm_kv_t* target_kv, const void* q_text, c
   return SPECVLM_OK;
 }
 
-static bool scores_legacy_mma() {
-  const char* impl = getenv("SPECVLM_SCORES_IMPL");
-  return impl && impl[0] == 'm';      // "mma": the mma.sync kernels
-}
-
 template <int D>
 static int32_t launch_lse(ScoreSetup& su, cudaStream_t st) {
   const dim3 grid((unsigned)su.n_row_tiles, (unsigned)su.kv.n_kv_heads, (unsigned)su.layer_count);
-  if (scores_legacy_mma()) {
-    constexpr int STAGES = 4;
-    constexpr int SMEM = STAGES * kKeyTile * D * 2 + 1024 + 16 * STAGES + 16 + 2 * 128 * 2 * 4;
-    auto k = scores_lse_kernel<D, STAGES>;
-    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
-      return SPECVLM_ERR_CUDA;
-    k<<<grid, 288, SMEM, st>>>(su.tk, su.p1);
-    return launch_status();
-  }
   constexpr int STAGES = 2;                              // two CTAs per SM: 3 x 32 KB each at d = 128
   constexpr int SMEM = (1 + STAGES) * kKeyTile * D * 2 + 1024 + 16 * STAGES + 40 + 16 + 128 * 8;
   auto k = scores_lse_tc_kernel<D, STAGES>;
-  if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
-    return SPECVLM_ERR_CUDA;
+  static std::atomic<uint64_t> attr_done{0};
+  if (!smem_attr_once(attr_done, reinterpret_cast<const void*>(k), SMEM)) return SPECVLM_ERR_CUDA;
   k<<<grid, 320, SMEM, st>>>(su.tk, su.tq, su.p1);
   return launch_status();
 }
 
 template <int D>
-static int32_t launch_colsum(ScoreSetup& su, float* scores, cudaStream_t st) {
-  const bool legacy = scores_legacy_mma();
-  int32_t rc;
-  if (legacy) {
-    constexpr int STAGES = 3;
-    constexpr int SMEM = (STAGES + 1) * kKeyTile * D * 2 + 1024 + 16 * STAGES + 16 + 16 + 128 * 4;
-    auto k = scores_colsum_kernel<D, STAGES>;
-    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
-      return SPECVLM_ERR_CUDA;
-    k<<<dim3((unsigned)su.n_key_blocks, (unsigned)su.layer_count), 288, SMEM, st>>>(su.tk, su.tq, su.p2);
-    rc = launch_status();
-  } else {
-    constexpr int STAGES = 4;
-    constexpr int SMEM = (2 + STAGES) * kKeyTile * D * 2 + 1024 + 16 * STAGES + 32 + 16 * kColsumGroups + 16 +
-                         kColsumGroups * 2 * 128 * 4;
-    auto k = scores_colsum_tc_kernel<D, STAGES>;
-    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
-      return SPECVLM_ERR_CUDA;
-    k<<<dim3((unsigned)su.n_key_blocks, (unsigned)su.layer_count), kColsumThreads, SMEM, st>>>(su.tk, su.tq, su.p2);
-    rc = launch_status();
-  }
-  (void)scores;
-  return rc;
+static int32_t launch_colsum(ScoreSetup& su, cudaStream_t st) {
+  constexpr int STAGES = 4;
+  constexpr int SMEM = (2 + STAGES) * kKeyTile * D * 2 + 1024 + 16 * STAGES + 32 + 16 * kColsumGroups + 16 +
+                       kColsumGroups * 2 * 128 * 4;
+  auto k = scores_colsum_tc_kernel<D, STAGES>;
+  static std::atomic<uint64_t> attr_done{0};
+  if (!smem_attr_once(attr_done, reinterpret_cast<const void*>(k), SMEM)) return SPECVLM_ERR_CUDA;
+  k<<<dim3((unsigned)su.n_key_blocks, (unsigned)su.layer_count), kColsumThreads, SMEM, st>>>(su.tk, su.tq, su.p2);
+  return launch_status();
 }
 
 }  // namespace specvlm
@@ -1154,6 +719,14 @@ extern "C" size_t specvlm_stage1_scores_workspace_bytes(const specvlm_kv_t* targ
   size_t a, c;
   ws_layout(target_kv->n_layers, n_q_heads, text_cu[batch], sum_video, a, c);
   return a + c;
+}
+
+extern "C" size_t specvlm_stage1_scores_layer_sums_offset(const specvlm_kv_t* target_kv, const int32_t* text_cu,
+                                                          int32_t batch, int32_t n_q_heads) {
+  if (!target_kv || !text_cu || batch < 1 || n_q_heads < 1) return 0;
+  size_t a, c;
+  ws_layout(target_kv->n_layers, n_q_heads, text_cu[batch], 0, a, c);
+  return a;
 }
 
 extern "C" int32_t specvlm_stage1_row_lse(const specvlm_kv_t* target_kv, const void* q_text,
@@ -1200,7 +773,7 @@ static int32_t stage1_scores_range(const specvlm_kv_t* target_kv, const void* q_
       if (rc != SPECVLM_OK) return rc;
     }
     su.p2.partial = partial_all + (size_t)layer_begin * su.p1.sum_video;
-    rc = d128 ? launch_colsum<128>(su, scores, st) : launch_colsum<64>(su, scores, st);
+    rc = d128 ? launch_colsum<128>(su, st) : launch_colsum<64>(su, st);
     if (rc != SPECVLM_OK) return rc;
   }
   if (!finish) return SPECVLM_OK;
