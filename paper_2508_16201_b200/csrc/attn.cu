@@ -388,18 +388,17 @@ attn_rows16_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 // ---------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------
-static int env_int(const char* name, int dflt) {
-  const char* s = getenv(name);
-  return s && *s ? atoi(s) : dflt;
-}
+// Test hook (specvlm_debug_set_attn_splits): > 0 forces the split count of the 16-row kernel so
+// that tests reach every path; 0 leaves the choice to the cost model below.
+static std::atomic<int> g_forced_splits{0};
 
 constexpr int kRows16Max = 16;     // windows up to this many rows run on attn_rows16_kernel
 
 // How many CTAs share one (layer, sequence, KV head): the split count with the lowest estimated
-// launch time.  SPECVLM_ATTN_SPLITS overrides the choice (tests use it to force every path).
+// launch time (a test hook can force it).
 static int choose_splits(int max_seq_len, int64_t items) {
   const int n_tiles = (max_seq_len + kTileTokens - 1) / kTileTokens;
-  const int forced = env_int("SPECVLM_ATTN_SPLITS", 0);
+  const int forced = g_forced_splits.load(std::memory_order_relaxed);
   int best = 1;
   if (forced > 0) {
     best = forced;
@@ -464,8 +463,8 @@ static int32_t launch_rows16_s(const CUtensorMap& tk, const CUtensorMap& tv, con
                                dim3 grid, cudaStream_t st) {
   constexpr int SMEM = STAGES * 2 * kTileTokens * D * 2 + 1024 + 16 * STAGES + 16;
   auto kern = attn_rows16_kernel<D, STAGES, NG>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
-    return SPECVLM_ERR_CUDA;
+  static std::atomic<uint64_t> attr_done{0};
+  if (!smem_attr_once(attr_done, reinterpret_cast<const void*>(kern), SMEM)) return SPECVLM_ERR_CUDA;
   // launched with programmatic stream serialization: see the kernel's griddepcontrol.wait
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
@@ -561,6 +560,10 @@ static int32_t attn_common(const specvlm_kv_t* kv, const void* q, int32_t batch,
 }  // namespace specvlm
 
 using namespace specvlm;
+
+extern "C" void specvlm_debug_set_attn_splits(int32_t n_splits) {
+  g_forced_splits.store(n_splits > 0 ? n_splits : 0, std::memory_order_relaxed);
+}
 
 extern "C" size_t specvlm_attn_workspace_bytes(const specvlm_kv_t* kv, int32_t batch,
                                                int32_t n_q_heads, int32_t gamma) {

@@ -927,11 +927,17 @@ static int32_t launch_tc_t(const CUtensorMap& tk, const CUtensorMap& tv, const C
                          int grid, cudaStream_t st) {
   using C = TcCfg<D, M>;
   auto kern = attn_tc_kernel<D, M, TREE>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::TOTAL) != cudaSuccess)
-    return SPECVLM_ERR_CUDA;
-  cudaFuncAttributes fa;
-  if (cudaFuncGetAttributes(&fa, kern) != cudaSuccess) return SPECVLM_ERR_CUDA;
-  if (fa.numRegs * kTcThreads < kRegsNeeded) return SPECVLM_ERR_CUDA;   // setmaxnreg could never be satisfied
+  // once per device and kernel variant: the opt-in shared-memory size, and the check that the
+  // compiled kernel's register pool can satisfy the setmaxnreg requests (it never changes)
+  static std::atomic<uint64_t> attr_done{0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SPECVLM_ERR_CUDA;
+  if (!(attr_done.load(std::memory_order_acquire) & (1ull << (dev & 63)))) {
+    cudaFuncAttributes fa;
+    if (cudaFuncGetAttributes(&fa, kern) != cudaSuccess) return SPECVLM_ERR_CUDA;
+    if (fa.numRegs * kTcThreads < kRegsNeeded) return SPECVLM_ERR_CUDA;   // setmaxnreg could never be satisfied
+    if (!smem_attr_once(attr_done, reinterpret_cast<const void*>(kern), C::TOTAL)) return SPECVLM_ERR_CUDA;
+  }
   kern<<<grid, kTcThreads, C::TOTAL, st>>>(tk, tv, tq, p);
   return launch_status();
 }

@@ -83,7 +83,8 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 // of fast polls the wall clock is consulted, and after kWaitLimitNs the wait gives up.  A CTA
 // shares one abort flag in shared memory so that one expired wait ends all the others at once.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                const uint64_t limit_ns) {
 #pragma unroll 1
   for (int i = 0; i < 2048; ++i)
     if (mbar_try_wait(bar, parity)) return true;
@@ -94,11 +95,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (global_timer_ns() - t0 > kWaitLimitNs) {
+    if (global_timer_ns() - t0 > limit_ns) {
       *abort_flag = 1;
       return false;
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  return mbar_wait_limit(bar, parity, abort_flag, kWaitLimitNs);
 }
 
 __device__ __forceinline__ void fence_proxy_async() {

@@ -95,4 +95,17 @@ inline int sm_count() {
   return n;
 }
 
+// The opt-in shared-memory size of a kernel is a per-device function attribute: it is set on a
+// device's first launch of that kernel and remembered (one bit per device ordinal in `done`, a
+// static of the launching function), so that later calls spend no host time on it.
+inline bool smem_attr_once(std::atomic<uint64_t>& done, const void* kern, int bytes) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  const uint64_t bit = 1ull << (dev & 63);
+  if (done.load(std::memory_order_acquire) & bit) return true;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+  done.fetch_or(bit, std::memory_order_release);
+  return true;
+}
+
 }  // namespace specvlm

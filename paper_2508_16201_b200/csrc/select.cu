@@ -380,9 +380,9 @@ static int32_t select_common(const float* scores, const int32_t* video_cu, const
     if (sm > max_smem) max_smem = sm;
   }
   if (max_smem > 232448) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
-  if (cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem) !=
-      cudaSuccess)
-    return SPECVLM_ERR_CUDA;
+  // the kernel may use up to a whole SM's shared memory; how much a launch gets is the launch's own figure
+  static std::atomic<uint64_t> attr_done{0};
+  if (!smem_attr_once(attr_done, reinterpret_cast<const void*>(select_kernel), 232448)) return SPECVLM_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   SelParams p;
   p.scores = scores;

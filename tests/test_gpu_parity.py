@@ -50,9 +50,8 @@ def _run_attn(L, Hq, Hkv, D, seq_lens, gamma, *, paged, seed, decode_api=False, 
     scale = 1.0 / math.sqrt(D)
     lse = torch.empty((L, B, nq, Hq), dtype=torch.float32, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    old = os.environ.get("SPECVLM_ATTN_SPLITS")
     if splits is not None:
-        os.environ["SPECVLM_ATTN_SPLITS"] = str(splits)
+        specvlm.debug_set_attn_splits(splits)
     try:
         if decode_api:
             assert gamma == 0
@@ -61,11 +60,7 @@ def _run_attn(L, Hq, Hkv, D, seq_lens, gamma, *, paged, seed, decode_api=False, 
         else:
             out = specvlm.verify_attn(cache, q, gamma, scale, lse=lse, d_status=status)
     finally:
-        if splits is not None:
-            if old is None:
-                del os.environ["SPECVLM_ATTN_SPLITS"]
-            else:
-                os.environ["SPECVLM_ATTN_SPLITS"] = old
+        specvlm.debug_set_attn_splits(0)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     ref, ref_lse = _oracle_attn(bits(q), k_host, v_host, seq_lens, scale)
