@@ -1,6 +1,10 @@
 // Cache maintenance around a speculative step: the K/V of the tokens a step feeds to a model are
 // appended to that model's cache before its attention runs, and the rows of rejected drafts are
 // dropped afterwards by shortening the sequence.  Pure byte movement and integer arithmetic.
+//
+// Sequence lengths, block tables and tree paths are device data: every value that becomes part
+// of an address is range-checked in the kernels.  What fails a check is skipped (no access is
+// made for it) and SPECVLM_ERR_INVALID_ARG is stored to d_status.
 #include "common.cuh"
 #include "host_util.h"
 
@@ -15,7 +19,7 @@ struct AppendParams {
   const int32_t* seq_lens; // lengths before the append
   int32_t* d_status;
   int64_t s_layer, s_block, s_head, s_token;   // cache strides in 16-byte units
-  int32_t block_tokens, max_blocks, max_seq_len;
+  int32_t block_tokens, max_blocks, max_seq_len, n_blocks;
   int32_t n_layers, batch, n_new, n_kv_heads, chunks_per_row;
 };
 
@@ -31,8 +35,8 @@ __global__ void __launch_bounds__(256) append_kv_kernel(const __grid_constant__ 
     const int layer = (int)(r / p.batch);
     const int len = p.seq_lens[b];
     const int pos = len + t;
-    if (len < 0 || pos >= p.max_seq_len) {
-      // no room (or a corrupt length): leave the cache alone and report
+    if (len < 0 || len + p.n_new > p.max_seq_len) {
+      // no room for all n_new rows (or a corrupt length): the sequence is left alone, every row of it
       if (p.d_status) *p.d_status = SPECVLM_ERR_INVALID_ARG;
       continue;
     }
@@ -40,6 +44,10 @@ __global__ void __launch_bounds__(256) append_kv_kernel(const __grid_constant__ 
     if (p.table) {
       blk = __ldg(p.table + (size_t)b * p.max_blocks + pos / p.block_tokens);
       off = pos % p.block_tokens;
+      if (blk < 0 || blk >= p.n_blocks) {
+        if (p.d_status) *p.d_status = SPECVLM_ERR_INVALID_ARG;
+        continue;
+      }
     }
     const int64_t dst = layer * p.s_layer + blk * p.s_block + head * p.s_head + off * p.s_token + chunk;
     p.k[dst] = __ldcs(p.new_k + i);
@@ -74,8 +82,9 @@ struct CompactParams {
   const int32_t* seq_lens;   // lengths including the n_nodes window
   const int32_t* path;       // [B][n_nodes]: accepted nodes in order, then -1
   const int32_t* accept_len; // [B]
+  int32_t* d_status;
   int64_t s_layer, s_block, s_head, s_token;
-  int32_t block_tokens, max_blocks, n_nodes, n_kv_heads, chunks_per_row;
+  int32_t block_tokens, max_blocks, n_blocks, max_seq_len, n_nodes, n_kv_heads, chunks_per_row;
 };
 
 // One CTA per (layer, KV head, sequence): the accepted nodes' rows move up behind the root.  A
@@ -84,37 +93,53 @@ __global__ void __launch_bounds__(256) compact_tree_kernel(const __grid_constant
   const int b = blockIdx.y;
   const int layer = blockIdx.x / p.n_kv_heads, head = blockIdx.x - layer * p.n_kv_heads;
   const int n = min(max(p.accept_len[b], 0), p.n_nodes - 1);
-  const int old = p.seq_lens[b] - p.n_nodes;
+  const int len = p.seq_lens[b];
+  const int old = len - p.n_nodes;
   const int cpr = p.chunks_per_row;
+  // address of (position, chunk), or -1 when the position's block-table entry is out of range
   auto addr = [&](int pos, int chunk) -> int64_t {
     int blk = b, off = pos;
     if (p.table) {
       blk = __ldg(p.table + (size_t)b * p.max_blocks + pos / p.block_tokens);
       off = pos % p.block_tokens;
+      if (blk < 0 || blk >= p.n_blocks) return -1;
     }
     return layer * p.s_layer + blk * p.s_block + head * p.s_head + off * p.s_token + chunk;
   };
   constexpr int kMaxPerThread = 2;          // 31 rows x 16 chunks = 496 chunks <= 2 x 256
   uint4 kk[kMaxPerThread], vv[kMaxPerThread];
-  if (old < 0) return;
+  bool have[kMaxPerThread] = {false, false};
+  if (old < 0 || len > p.max_seq_len) {     // tree_len_kernel reports the short sequence; a long one here
+    if (len > p.max_seq_len && p.d_status && threadIdx.x == 0) *p.d_status = SPECVLM_ERR_INVALID_ARG;
+    return;
+  }
 #pragma unroll
   for (int u = 0; u < kMaxPerThread; ++u) {
     const int idx = u * 256 + threadIdx.x;
     if (idx < n * cpr) {
       const int node = p.path[(size_t)b * p.n_nodes + idx / cpr];
-      const int64_t a = addr(old + node, idx % cpr);
-      kk[u] = p.k[a];
-      vv[u] = p.v[a];
+      const int64_t a = node >= 1 && node < p.n_nodes ? addr(old + node, idx % cpr) : -1;
+      if (a >= 0) {
+        kk[u] = p.k[a];
+        vv[u] = p.v[a];
+        have[u] = true;
+      } else if (p.d_status) {
+        *p.d_status = SPECVLM_ERR_INVALID_ARG;
+      }
     }
   }
   __syncthreads();
 #pragma unroll
   for (int u = 0; u < kMaxPerThread; ++u) {
     const int idx = u * 256 + threadIdx.x;
-    if (idx < n * cpr) {
+    if (have[u]) {
       const int64_t a = addr(old + 1 + idx / cpr, idx % cpr);
-      p.k[a] = kk[u];
-      p.v[a] = vv[u];
+      if (a >= 0) {
+        p.k[a] = kk[u];
+        p.v[a] = vv[u];
+      } else if (p.d_status) {
+        *p.d_status = SPECVLM_ERR_INVALID_ARG;
+      }
     }
   }
 }
@@ -155,6 +180,7 @@ extern "C" int32_t specvlm_append_kv(const specvlm_kv_t* kv, const void* new_k, 
   p.s_layer = c.stride_layer / 8; p.s_block = c.stride_block / 8; p.s_head = c.stride_head / 8;
   p.s_token = c.stride_token / 8;
   p.block_tokens = c.block_tokens; p.max_blocks = c.max_blocks; p.max_seq_len = c.max_seq_len;
+  p.n_blocks = c.n_blocks;
   p.n_layers = c.n_layers; p.batch = batch; p.n_new = n_new; p.n_kv_heads = c.n_kv_heads;
   p.chunks_per_row = c.head_dim / 8;
   const int64_t total = (int64_t)p.n_layers * batch * n_new * p.n_kv_heads * p.chunks_per_row;
@@ -199,6 +225,7 @@ extern "C" int32_t specvlm_compact_tree_kv(const specvlm_kv_t* kv, const int32_t
   p.s_layer = c.stride_layer / 8; p.s_block = c.stride_block / 8; p.s_head = c.stride_head / 8;
   p.s_token = c.stride_token / 8;
   p.block_tokens = c.block_tokens; p.max_blocks = c.max_blocks; p.n_nodes = n_nodes;
+  p.n_blocks = c.n_blocks; p.max_seq_len = c.max_seq_len; p.d_status = d_status;
   p.n_kv_heads = c.n_kv_heads; p.chunks_per_row = c.head_dim / 8;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   compact_tree_kernel<<<dim3((unsigned)(c.n_layers * c.n_kv_heads), (unsigned)batch), 256, 0, st>>>(p);

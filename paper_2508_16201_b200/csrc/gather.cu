@@ -1,6 +1,11 @@
 // Step 3: compaction of the surviving video tokens' K/V rows (plus all text rows) into the
 // draft cache.  Pure byte movement: 16-byte vector loads/stores, one (layer, KV head) slab per
 // blockIdx.y, consecutive lanes on consecutive 16-byte chunks of a token row.
+//
+// The kept indices and the block tables are device data that the host cannot validate: every
+// value that becomes part of an address is range-checked here.  A row whose index or block is out
+// of range is skipped (nothing is read or written for it) and SPECVLM_ERR_INVALID_ARG is stored
+// to d_status.
 #include "common.cuh"
 #include "host_util.h"
 
@@ -20,10 +25,11 @@ struct GatherParams {
   const int32_t* kept_idx;
   const int32_t* src_table;
   const int32_t* dst_table;
+  int32_t* d_status;
   // strides in 16-byte units
   int64_t s_layer, s_block, s_head, s_token;
   int64_t d_layer, d_block, d_head, d_token;
-  int32_t src_block_tokens, dst_block_tokens, src_max_blocks, dst_max_blocks;
+  int32_t src_block_tokens, dst_block_tokens, src_max_blocks, dst_max_blocks, src_n_blocks, dst_n_blocks;
   int32_t n_kv_heads, chunks_per_row, batch0;
   GatherSeq seq[kGatherMaxBatch];
 };
@@ -39,22 +45,31 @@ __global__ void __launch_bounds__(256) gather_kv_kernel(const __grid_constant__ 
   for (int j = blockIdx.x * rows_per_cta + threadIdx.x / cpr; j < sq.dst_len;
        j += gridDim.x * rows_per_cta) {
     int sp;                                  // source token position
+    bool ok = true;
     if (j < sq.video_start) {
       sp = j;
     } else if (j < sq.video_start + sq.kept_n) {
-      sp = sq.video_start + __ldg(p.kept_idx + sq.kept_off + (j - sq.video_start));
+      const int kj = __ldg(p.kept_idx + sq.kept_off + (j - sq.video_start));
+      ok = kj >= 0 && kj < sq.video_len;
+      sp = sq.video_start + kj;
     } else {
       sp = j - sq.kept_n + sq.video_len;
     }
     int sblk = b, soff = sp;
-    if (p.src_table) {
+    if (ok && p.src_table) {
       sblk = __ldg(p.src_table + (size_t)b * p.src_max_blocks + sp / p.src_block_tokens);
       soff = sp % p.src_block_tokens;
+      ok = sblk >= 0 && sblk < p.src_n_blocks;
     }
     int dblk = b, doff = j;
-    if (p.dst_table) {
+    if (ok && p.dst_table) {
       dblk = __ldg(p.dst_table + (size_t)b * p.dst_max_blocks + j / p.dst_block_tokens);
       doff = j % p.dst_block_tokens;
+      ok = dblk >= 0 && dblk < p.dst_n_blocks;
+    }
+    if (!ok) {
+      if (p.d_status && chunk == 0) *p.d_status = SPECVLM_ERR_INVALID_ARG;
+      continue;
     }
     const int64_t so = layer * p.s_layer + sblk * p.s_block + head * p.s_head + soff * p.s_token + chunk;
     const int64_t dof = layer * p.d_layer + dblk * p.d_block + head * p.d_head + doff * p.d_token + chunk;
@@ -73,7 +88,6 @@ extern "C" int32_t specvlm_gather_kv(const specvlm_kv_t* src, const int32_t* kep
                                      const int32_t* kept_cu, const int32_t* video_start,
                                      const int32_t* video_len, const int32_t* src_len, int32_t batch,
                                      const specvlm_kv_t* dst, int32_t* d_status, void* stream) {
-  (void)d_status;
   if (!src || !dst || !kept_idx || !kept_cu || !video_start || !video_len || !src_len || batch < 1)
     return SPECVLM_ERR_INVALID_ARG;
   // seq_lens are not read by this call; max_seq_len bounds the positions touched
@@ -114,6 +128,8 @@ extern "C" int32_t specvlm_gather_kv(const specvlm_kv_t* src, const int32_t* kep
   p.d_token = d.stride_token / 8;
   p.src_block_tokens = s.block_tokens; p.dst_block_tokens = d.block_tokens;
   p.src_max_blocks = s.max_blocks; p.dst_max_blocks = d.max_blocks;
+  p.src_n_blocks = s.n_blocks; p.dst_n_blocks = d.n_blocks;
+  p.d_status = d_status;
   p.n_kv_heads = s.n_kv_heads;
   p.chunks_per_row = s.head_dim / 8;
   const int rows_per_cta = 256 / p.chunks_per_row;
