@@ -19,7 +19,10 @@
  *   - Work is enqueued on the CUDA stream passed as `stream` (a cudaStream_t cast to void*;
  *     NULL = the legacy default stream).  No call synchronises the host with the device.
  *   - `d_status` (device int32_t*, optional): a kernel that gives up a bounded wait stores
- *     SPECVLM_ERR_TIMEOUT there and returns; it is never written otherwise.
+ *     SPECVLM_ERR_TIMEOUT there and returns.  A kernel that finds device-side data it would have
+ *     to turn into an address out of range (a kept index, a block-table entry, a tree-path node,
+ *     a sequence length) skips that access and stores SPECVLM_ERR_INVALID_ARG.  It is never
+ *     written otherwise; the caller zeroes it and reads it when convenient.
  *   - Scratch memory comes from the caller: `ws` (device, 256-byte aligned) of at least the
  *     size the matching *_workspace_bytes query returns.  Its contents need not be initialised
  *     and are unspecified afterwards.  Calls that share a workspace must not overlap on the GPU.
@@ -133,6 +136,18 @@ int32_t specvlm_stage1_scores_layers(const specvlm_kv_t* target_kv, const void* 
                                      size_t ws_bytes, int32_t layer_begin, int32_t layer_end, int32_t finish,
                                      int32_t* d_status, void* stream);
 
+/*
+ * Where a rating call leaves its per-layer sums (Eq. 5 before the average over layers): after
+ * specvlm_stage1_scores, or after the specvlm_stage1_scores_layers calls that rated a layer, the
+ * workspace holds, at the byte offset this query returns, fp32 [n_layers][video_cu[batch]]:
+ * entry (l, j) is the softmax probability that layer l puts on video token j, summed over all
+ * query heads and over the language queries of j's sequence (a fixed summation order).
+ * scores[j] = sum_l entry(l, j) / (n_layers * n_q_heads * n_text of the sequence).  Lets a caller
+ * inspect or re-weight single layers.  Returns 0 for invalid arguments.
+ */
+size_t specvlm_stage1_scores_layer_sums_offset(const specvlm_kv_t* target_kv, const int32_t* text_cu,
+                                               int32_t batch, int32_t n_q_heads);
+
 /* ---------------------------------------------------------------------------------------------
  * Steps 1b + 2 -- two-stage selection (Section 4.2).
  * Stage I keeps the k_stage1[b] highest-scored video tokens V_R (ranking "sort A, add in order"
@@ -148,7 +163,8 @@ int32_t specvlm_stage1_scores_layers(const specvlm_kv_t* target_kv, const void* 
  *   kept_idx    device int32 out: sequence b's kept video indices (sequence-local, ascending) at
  *               kept_cu[b] .. kept_cu[b]+k_total[b]-1
  * Requires 0 <= k_stage1 <= k_total <= n_video <= 57344 per sequence, n_frames <= 1024.
- * Uses no scratch memory.
+ * Uses no scratch memory.  d_status is accepted for uniformity and never written: the kernel has
+ * no bounded wait, and everything that becomes an address is host data checked before the launch.
  */
 int32_t specvlm_select(const float* scores, const int32_t* video_cu, const int32_t* n_frames,
                        int32_t tokens_per_frame, const int32_t* k_stage1, const int32_t* k_total,
@@ -209,6 +225,9 @@ int32_t specvlm_select_baseline(int32_t mode, uint64_t seed, const int32_t* n_fr
  *   src, dst    host structs with the same n_layers, n_kv_heads, head_dim; either may be paged
  *   kept_idx    device int32 (as written by specvlm_select); kept_cu, video_start, video_len,
  *               src_len host int32 ([batch+1] / [batch]); src_len[b] = tokens of sequence b in src
+ * Device-side range checks: a kept index outside [0, video_len[b]) or a block-table entry outside
+ * [0, n_blocks) of its cache makes the kernel skip that row (nothing is read or written for it)
+ * and store SPECVLM_ERR_INVALID_ARG to d_status.
  */
 int32_t specvlm_gather_kv(const specvlm_kv_t* src, const int32_t* kept_idx, const int32_t* kept_cu,
                           const int32_t* video_start, const int32_t* video_len,
@@ -273,8 +292,9 @@ int32_t specvlm_accept(const float* target_logits, const int32_t* draft_tokens, 
  *   new_k, new_v device bf16 [n_layers][batch][n_new][n_kv_heads][head_dim]
  *   seq_lens_inout  device int32 [batch], read then updated on the stream
  * A sequence without room (seq_lens[b] + n_new > kv->max_seq_len) is left unchanged and
- * SPECVLM_ERR_INVALID_ARG is stored to d_status.  With a block table the pages of the new
- * positions must already be mapped.
+ * SPECVLM_ERR_INVALID_ARG is stored to d_status: none of its n_new rows is written and its length
+ * stays.  With a block table the pages of the new positions must already be mapped; a row whose
+ * table entry is outside [0, n_blocks) is skipped and reported the same way.
  *
  * specvlm_rollback_kv drops the rejected drafts after verification: a cache that held the
  * gamma + 1 tokens of the window keeps accept_len[b] + 1 of them,
@@ -316,7 +336,9 @@ int32_t specvlm_rollback_kv(int32_t* seq_lens_inout, const int32_t* accept_len, 
  *
  * specvlm_compact_tree_kv: after acceptance the rows of the accepted nodes move up behind the
  * root (window position path[i] -> position 1 + i) and the sequence keeps 1 + accept_len of the
- * window's n_nodes rows, so that the cache is a plain sequence again.
+ * window's n_nodes rows, so that the cache is a plain sequence again.  A path node outside
+ * [1, n_nodes), a block-table entry outside [0, n_blocks) or a sequence longer than max_seq_len
+ * makes the kernel skip that row's move and store SPECVLM_ERR_INVALID_ARG to d_status.
  */
 size_t specvlm_verify_tree_workspace_bytes(const specvlm_kv_t* kv, int32_t batch, int32_t n_q_heads,
                                            int32_t n_nodes);
@@ -367,6 +389,23 @@ int32_t specvlm_accept_noalloc(const float* target_logits, const int32_t* draft_
  * nothing, allocates nothing, touches no global memory.
  */
 int32_t specvlm_debug_poison_shared_memory(void* stream);
+
+/*
+ * Diagnostic for tests; the paper has no counterpart.  Runs the library's bounded barrier wait on
+ * a barrier that nothing ever arrives at, with a limit of limit_ms (1..1000) milliseconds instead
+ * of the product kernels' 2 s: the wait gives up, the kernel stores SPECVLM_ERR_TIMEOUT to
+ * d_status (device, required) and the CTA's abort flag to d_abort_flag_or_null (device int32),
+ * and returns normally -- the way every kernel of the library reports an expired wait.
+ */
+int32_t specvlm_debug_wait_timeout(int32_t limit_ms, int32_t* d_status, int32_t* d_abort_flag_or_null,
+                                   void* stream);
+
+/*
+ * Test hook; the paper has no counterpart.  n_splits > 0 makes every later attention call of up
+ * to 16 rows per KV head cut each sequence into that many CTAs (capped by its tile count), so
+ * that tests reach the split-merge path at any size; 0 restores the built-in choice.  Process-wide.
+ */
+void specvlm_debug_set_attn_splits(int32_t n_splits);
 
 #ifdef __cplusplus
 }

@@ -48,13 +48,14 @@ _lib = None
 EXPORTS = [
     "specvlm_version", "specvlm_status_string",
     "specvlm_stage1_scores_workspace_bytes", "specvlm_stage1_row_lse", "specvlm_stage1_scores",
-    "specvlm_stage1_scores_layers",
+    "specvlm_stage1_scores_layers", "specvlm_stage1_scores_layer_sums_offset",
     "specvlm_select", "specvlm_select_top_p", "specvlm_select_baseline", "specvlm_gather_kv",
     "specvlm_attn_workspace_bytes", "specvlm_draft_decode_attn", "specvlm_verify_attn",
     "specvlm_accept_workspace_bytes", "specvlm_accept", "specvlm_accept_noalloc",
     "specvlm_append_kv", "specvlm_rollback_kv",
     "specvlm_verify_tree_workspace_bytes", "specvlm_verify_tree_attn", "specvlm_accept_tree",
-    "specvlm_compact_tree_kv", "specvlm_debug_poison_shared_memory",
+    "specvlm_compact_tree_kv", "specvlm_debug_poison_shared_memory", "specvlm_debug_wait_timeout",
+    "specvlm_debug_set_attn_splits",
 ]
 
 
@@ -73,6 +74,8 @@ def lib():
         L.specvlm_status_string.argtypes = [c_int32]
         L.specvlm_stage1_scores_workspace_bytes.restype = c_size_t
         L.specvlm_stage1_scores_workspace_bytes.argtypes = [kvp, i32p, i32p, c_int32, c_int32]
+        L.specvlm_stage1_scores_layer_sums_offset.restype = c_size_t
+        L.specvlm_stage1_scores_layer_sums_offset.argtypes = [kvp, i32p, c_int32, c_int32]
         L.specvlm_stage1_scores.restype = c_int32
         L.specvlm_stage1_scores.argtypes = [kvp, c_void_p, i32p, i32p, i32p, i32p, i32p, c_int32, c_int32,
                                             c_float, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p,
@@ -95,6 +98,10 @@ def lib():
                                            c_void_p, c_void_p, c_void_p]
         L.specvlm_debug_poison_shared_memory.restype = c_int32
         L.specvlm_debug_poison_shared_memory.argtypes = [c_void_p]
+        L.specvlm_debug_wait_timeout.restype = c_int32
+        L.specvlm_debug_wait_timeout.argtypes = [c_int32, c_void_p, c_void_p, c_void_p]
+        L.specvlm_debug_set_attn_splits.restype = None
+        L.specvlm_debug_set_attn_splits.argtypes = [c_int32]
         L.specvlm_verify_tree_workspace_bytes.restype = c_size_t
         L.specvlm_verify_tree_workspace_bytes.argtypes = [kvp, c_int32, c_int32, c_int32]
         L.specvlm_verify_tree_attn.restype = c_int32
@@ -257,6 +264,12 @@ def stage1_scores_workspace_bytes(kv: KvCache, text_cu, video_len, n_q_heads: in
     batch = len(video_len)
     return int(lib().specvlm_stage1_scores_workspace_bytes(byref(kv.struct), _i32(text_cu), _i32(video_len),
                                                            batch, n_q_heads))
+
+
+def stage1_scores_layer_sums_offset(kv: KvCache, text_cu, n_q_heads: int) -> int:
+    """Byte offset, inside a rating call's workspace, of the per-layer sums fp32 [n_layers][sum_video]."""
+    return int(lib().specvlm_stage1_scores_layer_sums_offset(byref(kv.struct), _i32(text_cu), len(text_cu) - 1,
+                                                             n_q_heads))
 
 
 def stage1_row_lse(kv: KvCache, q_text: torch.Tensor, text_cu, text_start, sm_scale: float,
@@ -426,6 +439,17 @@ def accept_tree(target_logits: torch.Tensor, node_tokens: torch.Tensor, parents:
 def debug_poison_shared_memory() -> None:
     """Fills the SMs' shared memory with NaN bit patterns (test diagnostic)."""
     _check(lib().specvlm_debug_poison_shared_memory(_stream()), "specvlm_debug_poison_shared_memory")
+
+
+def debug_wait_timeout(limit_ms: int, d_status: torch.Tensor, d_abort_flag: torch.Tensor | None = None) -> None:
+    """Runs the bounded barrier wait on a barrier nobody arrives at (test diagnostic)."""
+    _check(lib().specvlm_debug_wait_timeout(int(limit_ms), _ptr(d_status), _ptr(d_abort_flag), _stream()),
+           "specvlm_debug_wait_timeout")
+
+
+def debug_set_attn_splits(n_splits: int) -> None:
+    """Forces the split count of the 16-row attention kernel (0 = built-in choice; test hook)."""
+    lib().specvlm_debug_set_attn_splits(int(n_splits))
 
 
 def compact_tree_kv(kv: KvCache, path: torch.Tensor, accept_len: torch.Tensor,

@@ -271,6 +271,11 @@ def test_attention_against_library_sdpa(n_q):
     mask = torch.arange(n)[None, :] <= (torch.arange(n_q)[:, None] + n - n_q)
     ref = torch.nn.functional.scaled_dot_product_attention(qd, kd, vd, attn_mask=mask, scale=scale)
     np.testing.assert_allclose(o, ref[0].permute(1, 0, 2).numpy(), rtol=1e-10, atol=1e-13)
+    # the second output, the natural-log sum-exp of each row's scaled visible logits, against a
+    # library log-sum-exp of the masked logit matrix
+    logits = torch.einsum("hqd,hkd->qhk", qd[0], kd[0]).numpy() * scale              # [n_q][Hq][n]
+    logits = np.where(mask.numpy()[:, None, :], logits, -np.inf)
+    np.testing.assert_allclose(lse, scipy.special.logsumexp(logits, axis=-1), rtol=1e-12)
 
 
 def test_verify_rows_equal_truncated_decode_and_split_invariance():

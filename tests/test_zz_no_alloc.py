@@ -1,12 +1,14 @@
 """specvlm_accept_noalloc: the acceptance step for callers that cannot allocate device memory
 (a plug-in inside someone else's memory plan, a serving loop that must not call cudaMalloc) and
-have no workspace to pass.  Its scratch is a fixed array inside the library, so the only thing to
-check is that it gives exactly what specvlm_accept gives -- also on a second call, when the
-array still holds the first call's candidates -- and that it refuses problems larger than the
-array.  Collected last on purpose: a failure here cannot hide any other test."""
+have no workspace to pass.  Its scratch is a fixed array inside the library, so the thing to
+check is that it gives exactly what specvlm_accept gives (and what the CPU oracle gives) -- also
+on a second call, when the array still holds the first call's candidates -- and that it refuses
+problems larger than the array.  Collected last on purpose: a failure here cannot hide any other test."""
+import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2508_16201_b200 import specvlm, synth
 
 pytestmark = pytest.mark.gpu
@@ -22,6 +24,12 @@ def _both(batch, gamma, vocab, seed):
     torch.cuda.synchronize()
     # integer results: the tolerance of the other acceptance tests is bit-exactness
     assert torch.equal(n, ref_n) and torch.equal(nxt, ref_next) and torch.equal(g, ref_g)
+    # and against the CPU oracle on the same logits and drafts, so that a defect shared by the two
+    # CUDA entry points cannot pass
+    lg, dr = logits.cpu().numpy(), drafts.cpu().numpy()
+    for b in range(batch):
+        on, onext, og = oracle.accept_fast(lg[b], dr[b])
+        assert (int(n[b]), int(nxt[b])) == (on, onext) and np.array_equal(g[b].cpu().numpy(), og)
 
 
 def test_noalloc_matches_accept_on_two_calls_in_a_row():
