@@ -33,7 +33,12 @@ sys.path.insert(0, ROOT)
 METRIC = "draft-decode + verify attention KV GB/s"
 UNIT = "GB/s"
 HBM_NOMINAL_GBS = 8000.0
-EX2_PEAK_GOPS = 16 * 148 * 1.965          # special-function units: exponentials per ns, whole GPU
+EX2_PER_CLK_PER_SM = 16                   # special-function units: base-2 exponentials per clock per SM
+
+
+def ex2_peak_gops(n_sms, sm_max_mhz):
+    """Exponentials per ns of the whole GPU at its maximum SM clock."""
+    return EX2_PER_CLK_PER_SM * n_sms * sm_max_mhz * 1e-3
 
 
 def measured_peaks():
@@ -42,14 +47,16 @@ def measured_peaks():
         with open(path) as f:
             d = json.load(f)
         return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
-                "bf16_tflops_sustained": float(d["bf16_tflops_sustained"]), "source": "measured"}
-    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+                "bf16_tflops_sustained": float(d["bf16_tflops_sustained"]),
+                "sm_max_mhz": float(d.get("sm_max_mhz", 0) or 0), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "sm_max_mhz": 0.0,
+            "source": "fallback"}
 
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
 # summarised under profiles/; None where no capture of that launch exists.  Each capture ran a
-# subset of the layers (the capture-size rule) and is scaled to the layers one launch processes:
-# traffic is proportional to the layers streamed.  verify: 216.0 MB for 8 of 80 layers; rating
+# subset of the layers (a many-pass capture has to stay small) and is scaled to the layers one
+# launch processes: traffic is proportional to the layers streamed.  verify: 216.0 MB for 8 of 80 layers; rating
 # passes: 156.5 MB and 153.2 MB for 10 of 80 layers; decode: 43.5 MB, captured whole.
 NCU_TRAFFIC_BYTES = {"verify": 216.0e6 * 10, "decode": 43.5e6, "scores_colsum": 153.2e6 * 8, "scores_lse": 156.5e6 * 8}
 
@@ -122,6 +129,58 @@ def max_over_ranks(times_ms, world, device):
 def replicas_value(bytes_per_replica, ms, world):
     """Whole-job K/V GB/s: every replica moved `bytes_per_replica` in the slowest rank's time."""
     return world * bytes_per_replica / (ms * 1e-3) / 1e9
+
+
+class GraphTimer:
+    """Times a call the way the headline is timed: the call (its C-ABI entry point with every
+    launch and memset it makes) is captured once into a CUDA graph and the graph is replayed;
+    CUDA events bracket each replay on the replaying stream.  With `flush`, a buffer larger than
+    the L2 cache is overwritten before every replay (outside the event pair), so that a call whose
+    inputs would fit in L2 still reads them from HBM."""
+
+    def __init__(self, device, eager=False, flush_mb=512):
+        import torch
+        self.torch, self.eager = torch, eager
+        self.side = torch.cuda.Stream()
+        self.flush_buf = torch.empty(flush_mb << 20, dtype=torch.uint8, device=device)
+
+    def prepare(self, fn, warm=3):
+        torch = self.torch
+        for _ in range(warm):
+            fn()
+        torch.cuda.synchronize()
+        if self.eager:
+            return fn
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(self.side):
+            with torch.cuda.graph(g, stream=self.side):
+                fn()
+        torch.cuda.synchronize()
+        g.replay()
+        torch.cuda.synchronize()
+        return g.replay
+
+    def time(self, fn, reps=20, warm=3, flush=True, prepared=False):
+        """Median and minimum device time of `fn` in microseconds."""
+        torch = self.torch
+        run = fn if prepared else self.prepare(fn, warm)
+        ts = []
+        for _ in range(reps):
+            if flush:
+                self.flush_buf.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            run()
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b) * 1e3)
+        return statistics.median(ts), min(ts)
+
+
+def sd_projection(tau, gamma, t_draft, t_target, t_verify):
+    """Speed-up of speculative decoding over plain target decoding by the paper's latency model
+    (Section 3.1, Eq. 1-3): tau / (gamma * T_d / T_t + T_t^gamma / T_t)."""
+    return tau / (gamma * t_draft / t_target + t_verify / t_target)
 
 
 def build_inputs(w, device, n_copies):
@@ -328,57 +387,57 @@ def run_ours(args, rank, world):
     # ---------------- end-to-end leg: inputs from pinned host memory, results read back
     e2e = run_e2e(args, path, inp, w, device, attn_bytes)
 
-    # ---------------- extras outside the timed region: unpruned draft cache (the SD baseline draft)
+    # ---------------- extras outside the timed region, each timed like the headline calls: captured
+    # once into its own CUDA graph, replayed 20 times behind an L2 flush, median of the event times
     extra = {}
+    gt = GraphTimer(device, eager=args.eager)
     dsrc = inp["dsrc"]
     ws_u = torch.empty(max(256, specvlm.attn_workspace_bytes(dsrc, 1, w.d_q_heads, 0)), dtype=torch.uint8,
                        device=device)
-    ts = []
-    for i in range(3 + 10):
-        a, b = E(), E()
-        a.record()
-        specvlm.draft_decode_attn(dsrc, inp["q_dec"][0], path.scale, out=path.o_dec[0], ws=ws_u)
-        b.record()
-        torch.cuda.synchronize()
-        if i >= 3:
-            ts.append(a.elapsed_time(b))
+    # the unpruned draft cache: the draft of plain speculative decoding (the paper's SD baseline)
+    us_unpruned, _ = gt.time(lambda: specvlm.draft_decode_attn(dsrc, inp["q_dec"][0], path.scale, out=path.o_dec[0],
+                                                               ws=ws_u, d_status=path.status))
     bytes_unpruned = 2 * (nv + nt) * w.d_kv_heads * D * 2 * w.d_layers
-    # the same pruned copy at every draft step, launched back to back: what a draft loop does.  The
-    # 43 MB stay in the L2 cache, so the step is no longer an HBM stream (the headline never reuses a
-    # copy and counts HBM bytes only)
+    extra["decode_unpruned_us"] = us_unpruned
+    extra["decode_unpruned_kv_gbs"] = bytes_unpruned / (us_unpruned * 1e-6) / 1e9
+    # the same pruned copy at every draft step, replayed back to back without a flush: what a draft
+    # loop does.  The 43 MB stay in the L2 cache, so the step is no longer an HBM stream (the
+    # headline never reuses a copy and counts HBM bytes only)
+    run_l2 = gt.prepare(lambda: path.decode_call(0, inp["dpruned"][1]))
     a, b = E(), E()
-    for i in range(3):
-        path.decode_call(0, inp["dpruned"][1])
-    torch.cuda.synchronize()
     a.record()
     for i in range(20):
-        path.decode_call(0, inp["dpruned"][1])
+        run_l2()
     b.record()
     torch.cuda.synchronize()
     extra["decode_pruned_l2_resident_us"] = a.elapsed_time(b) * 1e3 / 20
-    extra["decode_unpruned_us"] = statistics.median(ts) * 1e3
-    extra["decode_unpruned_kv_gbs"] = bytes_unpruned / (statistics.median(ts) * 1e-3) / 1e9
+    # T_t: the target's own single-token decode attention over the full cache (verification with
+    # gamma = 0), against T_t^gamma (the verification call of the step) and T_d (a draft step): the
+    # terms of the paper's latency model (Section 3.1, Eq. 1-3), attention only
+    q_t = inp["q_ver"][:, :, :1].contiguous()
+    o_t = torch.empty_like(q_t)
+    ws_t0 = torch.empty(max(256, specvlm.attn_workspace_bytes(inp["tcache"], 1, w.t_q_heads, 0)), dtype=torch.uint8,
+                        device=device)
+    us_tt, _ = gt.time(lambda: specvlm.verify_attn(inp["tcache"], q_t, 0, path.scale, out=o_t, ws=ws_t0,
+                                                   d_status=path.status))
+    extra["target_decode_T_t_us"] = us_tt
+    extra["target_decode_T_t_kv_gbs"] = bytes_ver / (us_tt * 1e-6) / 1e9
+    extra["verify_over_target_decode_ratio"] = mean["verify"] * 1e3 / us_tt
+    # illustrative only: attention times stand in for whole-model times, tau is the paper's printed
+    # average accept length for chain drafting on the 72B/7B pair (2.79 pruned draft, 3.12 unpruned)
+    extra["eq3_projection_pruned_draft_tau_2.79"] = sd_projection(2.79, gamma, mean["decode"] * 1e3, us_tt,
+                                                                  mean["verify"] * 1e3)
+    extra["eq3_projection_unpruned_draft_tau_3.12"] = sd_projection(3.12, gamma, us_unpruned, us_tt,
+                                                                    mean["verify"] * 1e3)
 
-    # the calls outside the step's fixed path (Top-P selection, tree drafting, cache maintenance),
-    # one after the other, median of 10 after 3 warm-ups; launches back to back without a host sync
-    # inside the timed pair would hide nothing here, each is a single short call
-    def timed(fn, reps=10):
-        out = []
-        for i in range(3 + reps):
-            a, b = E(), E()
-            a.record()
-            fn()
-            b.record()
-            torch.cuda.synchronize()
-            if i >= 3:
-                out.append(a.elapsed_time(b))
-        return statistics.median(out) * 1e3
-
-    extra["select_top_p_us"] = timed(lambda: specvlm.select_top_p(path.scores, [0, nv], [w.n_frames[0]],
-                                                                  w.tokens_per_frame, [400], [path.kt], [0, path.kt]))
-    extra["select_random_us"] = timed(lambda: specvlm.select_baseline(specvlm.SEL_RANDOM, [w.n_frames[0]],
-                                                                      w.tokens_per_frame, [path.kt], [0, path.kt],
-                                                                      seed=1, device=device))
+    kept_tp = torch.empty(path.kt, dtype=torch.int32, device=device)
+    k1_tp = torch.empty(1, dtype=torch.int32, device=device)
+    extra["select_top_p_us"], _ = gt.time(lambda: specvlm.select_top_p(
+        path.scores, [0, nv], [w.n_frames[0]], w.tokens_per_frame, [400], [path.kt], [0, path.kt], kept_idx=kept_tp,
+        k_stage1_out=k1_tp))
+    extra["select_random_us"], _ = gt.time(lambda: specvlm.select_baseline(
+        specvlm.SEL_RANDOM, [w.n_frames[0]], w.tokens_per_frame, [path.kt], [0, path.kt], seed=1, device=device,
+        kept_idx=kept_tp, want_counts=False))
     # tree drafting: the widest tree one 128-row launch holds (16 nodes at 8 query heads per KV head),
     # and a 26-node static tree (root + 25 candidates, the size of the static draft tree the paper
     # adopts; its shape here is a binary heap, the paper's figure being unavailable): 208 rows, two launches
@@ -392,23 +451,27 @@ def run_ours(args, rank, world):
         o_tree = torch.empty_like(q_tree)
         ws_t = torch.empty(specvlm.lib().specvlm_verify_tree_workspace_bytes(ctypes_byref(tcache), 1, w.t_q_heads, n_nodes),
                            dtype=torch.uint8, device=device)
-        us = timed(lambda: specvlm.verify_tree_attn(tcache, q_tree, parents, path.scale, out=o_tree, ws=ws_t), reps=5)
+        us, _ = gt.time(lambda: specvlm.verify_tree_attn(tcache, q_tree, parents, path.scale, out=o_tree, ws=ws_t,
+                                                         d_status=path.status), reps=10)
         extra["verify_tree_%d_nodes_us" % n_nodes] = us
         extra["verify_tree_%d_nodes_kv_gbs_per_pass" % n_nodes] = (
             2 * n_tree * w.t_kv_heads * D * 2 * w.t_layers * ((n_nodes * (w.t_q_heads // w.t_kv_heads) + 127) // 128)
             / (us * 1e-6) / 1e9)
         lg = torch.randn((1, n_nodes, w.vocab), device=device)
         toks = torch.zeros((1, n_nodes), dtype=torch.int32, device=device)
-        extra["accept_tree_%d_nodes_us" % n_nodes] = timed(lambda: specvlm.accept_tree(lg, toks, parents))
+        t_out = specvlm.accept_tree_buffers(1, n_nodes, w.vocab, device)
+        extra["accept_tree_%d_nodes_us" % n_nodes], _ = gt.time(lambda: specvlm.accept_tree(lg, toks, parents, out=t_out))
         del tk, tv, tcache, q_tree, o_tree, lg, ws_t
     new_kv = synth.randn_bf16((w.t_layers, 1, gamma + 1, w.t_kv_heads, D), device, 2, "newKV")
     lens_keep = inp["tcache"].seq_lens.clone()
+    lens_base = torch.tensor([nv + nt], dtype=torch.int32, device=device)
 
     def append_once():
-        inp["tcache"].seq_lens.fill_(nv + nt)                    # room for the gamma+1 new rows again
-        specvlm.append_kv(inp["tcache"], new_kv, new_kv)
-    extra["append_kv_us_incl_len_reset"] = timed(append_once)
+        inp["tcache"].seq_lens.copy_(lens_base)                  # room for the gamma+1 new rows again
+        specvlm.append_kv(inp["tcache"], new_kv, new_kv, d_status=path.status)
+    extra["append_kv_us_incl_len_reset"], _ = gt.time(append_once)
     inp["tcache"].seq_lens.copy_(lens_keep)
+    assert int(path.status.item()) == 0
 
     # max over ranks
     total_ms, attn_ms = max_over_ranks([total_ms, attn_ms], world, device)
@@ -423,16 +486,22 @@ def run_ours(args, rank, world):
                 "frac": round(ach / peaks["hbm_gbs"], 4), "frac_of_nominal_8000": round(ach / HBM_NOMINAL_GBS, 4),
                 "traffic": traffic, "peak_source": peaks["source"], "launch_ms": round(ms, 5)}
 
+    n_sms = torch.cuda.get_device_properties(device).multi_processor_count
+    sm_max_mhz = peaks["sm_max_mhz"] or (clocks or {}).get("sm_max_mhz") or 1965.0
+    ex2_peak = ex2_peak_gops(n_sms, sm_max_mhz)
+
     def rating(name, n_exp, flops, ms, traffic):
         # The rating passes evaluate one base-2 exponential per (query row, key) logit on the
-        # special-function units: 16 per clock per SM x 148 SMs x 1.965 GHz = 4653 G/s.  That bound
-        # (0.89 ms per pass here) is tighter than the tensor-core one (1.05 TFLOP at the measured
-        # dense bf16 rate: 0.75 ms), so it is the roofline; the tensor view is reported beside it.
+        # special-function units: 16 per clock per SM x the device's SM count x its maximum SM clock
+        # (148 x 1.965 GHz: 4653 G/s).  That bound (0.89 ms per pass here) is tighter than the
+        # tensor-core one (1.05 TFLOP at the measured dense bf16 rate: 0.75 ms), so it is the
+        # roofline; the tensor view is reported beside it.
         ach = n_exp / (ms * 1e-3) / 1e9
         tf = flops / (ms * 1e-3) / 1e12
-        return {"kernel": name, "bound": "alu", "achieved": round(ach, 1), "peak": EX2_PEAK_GOPS, "unit": "Gex2/s",
-                "frac": round(ach / EX2_PEAK_GOPS, 4), "traffic": traffic,
-                "peak_source": "derived: 16 ex2/clk/SM x 148 SMs x 1965 MHz", "launch_ms": round(ms, 5),
+        return {"kernel": name, "bound": "alu", "achieved": round(ach, 1), "peak": round(ex2_peak, 1), "unit": "Gex2/s",
+                "frac": round(ach / ex2_peak, 4), "traffic": traffic,
+                "peak_source": "derived: %d ex2/clk/SM x %d SMs x %.0f MHz" % (EX2_PER_CLK_PER_SM, n_sms, sm_max_mhz),
+                "launch_ms": round(ms, 5),
                 "tensor_tflops": round(tf, 1), "tensor_frac_of_measured_sustained": round(tf / peaks["bf16_tflops_sustained"], 4)}
 
     rows = w.t_layers * w.t_q_heads * nt
@@ -763,9 +832,200 @@ def run_case_batched(args, w, device):
                       "gbs": round(nbytes / (med * 1e-3) / 1e9, 1)}))
 
 
+# ------------------------------------------------------------------------------------------------
+# --workloads: every call of the path on every synthetic workload, with the sweeps
+# ------------------------------------------------------------------------------------------------
+class WorkloadCase:
+    """Device-resident synthetic tensors of one workload shape (any batch; contiguous caches for a
+    single sequence, 64-token pages scattered over a pool for a batch) and its calls.  The verifier
+    side may hold fewer layers than the workload names when device memory is short: every layer is
+    an independent, equally sized problem for every call, so a call's time is the sum over layer
+    chunks; the chunks being alike, one is timed and multiplied by their number."""
+
+    def __init__(self, w, device, gamma_max, retention_max_permille, t_layers=None):
+        import torch
+        from paper_2508_16201_b200 import specvlm, synth
+        self.w, self.device, self.sv, self.torch, self.synth = w, device, specvlm, torch, synth
+        self.B, self.D = w.batch, w.head_dim
+        B, D = self.B, self.D
+        self.scale = 1.0 / math.sqrt(D)
+        self.t_layers = t_layers or w.t_layers
+        self.t_chunks = -(-w.t_layers // self.t_layers)
+        self.nv = [w.n_video(b) for b in range(B)]
+        self.nt = [w.n_text[b] for b in range(B)]
+        self.text_cu = [0] + [sum(self.nt[:b + 1]) for b in range(B)]
+        self.video_cu = [0] + [sum(self.nv[:b + 1]) for b in range(B)]
+        self.gamma_max = gamma_max
+        cap_t = [self.nv[b] + self.nt[b] + gamma_max + 1 for b in range(B)]
+        self.tk, self.tv, self.t_table = self._alloc(self.t_layers, w.t_kv_heads, cap_t, "t")
+        self.q_text = synth.randn_bf16((self.t_layers, self.text_cu[-1], w.t_q_heads, D), device, 0, "Qtext")
+        for b in range(B):
+            sal = synth.salient_set(self.nv[b], w.planted_permille, 0, b)
+            qb = self.q_text[:, self.text_cu[b]:self.text_cu[b + 1]]
+            if self.t_table is None:
+                synth.plant_salient_(self.tk[:, 0, :, :self.nv[b], :], qb, sal)
+            else:
+                synth.plant_salient_paged_(self.tk, self.t_table[b], 0, self.nv[b], qb, sal)
+        self.prompt = self.cache(self.tk, self.tv, [self.nv[b] + self.nt[b] for b in range(B)], self.t_table)
+        cap_d = [self.nv[b] + self.nt[b] for b in range(B)]
+        self.sk, self.svv, self.s_table = self._alloc(w.d_layers, w.d_kv_heads, cap_d, "d")
+        self.dsrc = self.cache(self.sk, self.svv, cap_d, self.s_table)
+        cap_p = [self.nv[b] * retention_max_permille // 1000 + self.nt[b] for b in range(B)]
+        self.pk, self.pv, self.p_table = self._alloc(w.d_layers, w.d_kv_heads, cap_p, "p")
+        self.q_dec = synth.randn_bf16((w.d_layers, B, w.d_q_heads, D), device, 0, "Qd")
+        self.o_dec = torch.empty_like(self.q_dec)
+        self.logits, self.drafts = synth.logits_and_drafts(B, gamma_max, w.vocab, device, 0)
+        self.row_lse = torch.empty((self.t_layers, self.text_cu[-1], w.t_q_heads), dtype=torch.float32, device=device)
+        self.scores = torch.empty(self.video_cu[-1], dtype=torch.float32, device=device)
+        self.ws_scores = torch.empty(specvlm.stage1_scores_workspace_bytes(self.prompt, self.text_cu, self.nv,
+                                                                           w.t_q_heads), dtype=torch.uint8, device=device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+
+    def _alloc(self, n_layers, n_kv_heads, caps, tag):
+        torch, synth, B, D = self.torch, self.synth, self.B, self.D
+        if B == 1 and not self.w.paged:
+            shape, table = (n_layers, 1, n_kv_heads, caps[0], D), None
+        else:
+            need = [(n + 63) // 64 for n in caps]
+            pool = sum(need) + 3
+            table = synth.page_table(B, max(need) + 1, pool, need, 0, self.device)
+            shape = (n_layers, pool, n_kv_heads, 64, D)
+        return (synth.randn_bf16(shape, self.device, 0, tag + "K"), synth.randn_bf16(shape, self.device, 0, tag + "V"),
+                table)
+
+    def cache(self, k, v, lens, table):
+        lens_t = self.torch.tensor(lens, dtype=self.torch.int32, device=self.device)
+        return self.sv.KvCache(k, v, lens_t, max(lens), table)
+
+    def kv_bytes(self, lens, n_kv_heads, n_layers):
+        return 2 * sum(lens) * n_kv_heads * self.D * 2 * n_layers
+
+    def ws(self, cache, n_q_heads, gamma):
+        return self.torch.empty(max(256, self.sv.attn_workspace_bytes(cache, self.B, n_q_heads, gamma)),
+                                dtype=self.torch.uint8, device=self.device)
+
+
+def run_workloads(args):
+    """Every call of the path on workloads 2-5 (and the tiny workload 1), one JSON line per
+    workload: median device time of 20 graph replays behind an L2 flush, K/V GB/s and the fraction
+    of the measured HBM peak where the call is a stream.  Workload 4 sweeps the retention (5, 10,
+    20, 50 %), workload 5 the draft length gamma (3..8); workload 5 runs batched and paged."""
+    import torch
+    from paper_2508_16201_b200 import specvlm, synth
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    peaks = measured_peaks()
+    gt = GraphTimer(device, eager=args.eager)
+    reps = args.iters if args.iters > 10 else 20
+    which = [int(x) for x in args.workloads.split(",")]
+
+    def rec(us, mn, nbytes=None, chunks=1):
+        """us, mn, nbytes: of one layer chunk; the call's time is the chunk's time x chunks."""
+        r = {"us": round(us * chunks, 2), "min_us": round(mn * chunks, 2)}
+        if chunks > 1:
+            r["layer_chunks"] = chunks
+        if nbytes:
+            r["gbs"] = round(nbytes / (us * 1e-6) / 1e9, 1)
+            r["frac_of_measured_%d" % int(peaks["hbm_gbs"])] = round(r["gbs"] / peaks["hbm_gbs"], 4)
+            r["frac_of_nominal_8000"] = round(r["gbs"] / HBM_NOMINAL_GBS, 4)
+        return r
+
+    for i in which:
+        w = synth.workload(i)
+        sweep_ret = [50, 100, 200, 500] if i == 4 else [w.retention_permille]
+        sweep_gamma = list(range(3, 9)) if i == 5 else [w.gamma]
+        B, D = w.batch, w.head_dim
+        # verifier layers held at once: all of them when its K/V fits in 60 % of the free memory
+        free, _ = torch.cuda.mem_get_info(device)
+        per_layer = 2 * sum(w.seq_len(b) + 9 + 64 for b in range(B)) * w.t_kv_heads * D * 2
+        t_layers = w.t_layers
+        while t_layers > 1 and t_layers * per_layer > 0.6 * free:
+            t_layers = (t_layers + 1) // 2
+        c = WorkloadCase(w, device, max(sweep_gamma), max(sweep_ret), t_layers)
+        ch = c.t_chunks
+        L_t = c.t_layers * ch                                  # layers the chunked time stands for (>= w.t_layers)
+        out = {"workload": w.name, "batch": B, "paged": c.t_table is not None,
+               "verifier_layers_held": c.t_layers, "verifier_layer_chunks": ch,
+               "launch": "eager" if args.eager else "one CUDA graph per call, replayed behind a 512 MB L2 flush",
+               "reps": reps, "calls": {}, "sweeps": {}}
+        calls = out["calls"]
+        # ---- prune side
+        calls["row_lse"] = rec(*gt.time(lambda: specvlm.stage1_row_lse(c.prompt, c.q_text, c.text_cu, c.nv, c.scale,
+                                                                       row_lse=c.row_lse, d_status=c.status), reps), chunks=ch)
+        calls["scores_given_lse"] = rec(*gt.time(lambda: specvlm.stage1_scores(
+            c.prompt, c.q_text, c.text_cu, c.nv, [0] * B, c.nv, c.video_cu, c.scale, scores=c.scores, ws=c.ws_scores,
+            d_status=c.status, row_lse=c.row_lse), reps), chunks=ch)
+        n_exp = sum(w.t_q_heads * c.nt[b] * c.nv[b] for b in range(B)) * float(L_t)
+        calls["scores_given_lse"]["gex2_per_s"] = round(n_exp / (calls["scores_given_lse"]["us"] * 1e-6) / 1e9, 1)
+        sel, gat, dec = {}, {}, {}
+        for ret in sweep_ret:
+            wr = synth.workload(i, retention_permille=ret)
+            kt = [wr.k_total(b) for b in range(B)]
+            k1 = [wr.k_stage1(b) for b in range(B)]
+            kept_cu = [0] + [sum(kt[:b + 1]) for b in range(B)]
+            kept = torch.empty(max(kept_cu[-1], 1), dtype=torch.int32, device=device)
+            sel[ret] = rec(*gt.time(lambda: specvlm.select(c.scores, c.video_cu, list(w.n_frames), w.tokens_per_frame,
+                                                           k1, kt, kept_cu, kept_idx=kept, d_status=c.status), reps))
+            plens = [kt[b] + c.nt[b] for b in range(B)]
+            pruned = c.cache(c.pk, c.pv, plens, c.p_table)
+            src_len = [c.nv[b] + c.nt[b] for b in range(B)]
+            gat[ret] = rec(*gt.time(lambda: specvlm.gather_kv(c.dsrc, kept, kept_cu, [0] * B, c.nv, src_len, pruned,
+                                                              d_status=c.status), reps),
+                           nbytes=2 * c.kv_bytes(plens, w.d_kv_heads, w.d_layers))
+            ws_d = c.ws(pruned, w.d_q_heads, 0)
+            dec[ret] = rec(*gt.time(lambda: specvlm.draft_decode_attn(pruned, c.q_dec, c.scale, out=c.o_dec, ws=ws_d,
+                                                                      d_status=c.status), reps),
+                           nbytes=c.kv_bytes(plens, w.d_kv_heads, w.d_layers))
+            dec[ret]["tokens"] = plens if B > 1 else plens[0]
+        base = w.retention_permille
+        calls["select"], calls["gather"], calls["decode_pruned"] = sel[base], gat[base], dec[base]
+        if len(sweep_ret) > 1:
+            out["sweeps"]["retention_permille"] = {str(r): {"select": sel[r], "gather": gat[r], "decode_pruned": dec[r]}
+                                                   for r in sweep_ret}
+        ws_u = c.ws(c.dsrc, w.d_q_heads, 0)
+        calls["decode_unpruned"] = rec(*gt.time(lambda: specvlm.draft_decode_attn(
+            c.dsrc, c.q_dec, c.scale, out=c.o_dec, ws=ws_u, d_status=c.status), reps),
+            nbytes=c.kv_bytes([c.nv[b] + c.nt[b] for b in range(B)], w.d_kv_heads, w.d_layers))
+        # ---- verification and acceptance
+        ver, acc = {}, {}
+        for g in sorted(set(sweep_gamma + [0])):
+            lens = [c.nv[b] + c.nt[b] + g + 1 for b in range(B)]
+            tc = c.cache(c.tk, c.tv, lens, c.t_table)
+            q = synth.randn_bf16((c.t_layers, B, g + 1, w.t_q_heads, D), device, 0, "Qv", g)
+            o = torch.empty_like(q)
+            ws_v = c.ws(tc, w.t_q_heads, g)
+            ver[g] = rec(*gt.time(lambda: specvlm.verify_attn(tc, q, g, c.scale, out=o, ws=ws_v, d_status=c.status),
+                                  reps), nbytes=c.kv_bytes(lens, w.t_kv_heads, c.t_layers), chunks=ch)
+            ver[g]["rows_per_kv_head"] = (g + 1) * (w.t_q_heads // w.t_kv_heads)
+            if g == 0:
+                continue
+            lg = c.logits[:, :g + 1].contiguous()
+            dr = c.drafts[:, :g].contiguous()
+            a_out = (torch.empty(B, dtype=torch.int32, device=device), torch.empty(B, dtype=torch.int32, device=device), None)
+            ws_a = torch.empty(specvlm.accept_workspace_bytes(B, g, w.vocab), dtype=torch.uint8, device=device)
+            acc[g] = rec(*gt.time(lambda: specvlm.accept(lg, dr, ws=ws_a, out=a_out), reps), nbytes=B * (g + 1) * w.vocab * 4)
+            del q, o, ws_v
+        calls["verify"], calls["accept"], calls["target_decode_T_t"] = ver[w.gamma], acc[w.gamma], ver[0]
+        if len(sweep_gamma) > 1:
+            out["sweeps"]["gamma"] = {str(g): {"verify": ver[g], "accept": acc[g]} for g in sweep_gamma}
+        assert int(c.status.item()) == 0, "a device-side check or wait reported an error"
+        calls["prune_us"] = round(calls["row_lse"]["us"] + calls["scores_given_lse"]["us"] + calls["select"]["us"], 2)
+        calls["prune_us_with_caller_lse"] = round(calls["scores_given_lse"]["us"] + calls["select"]["us"], 2)
+        t_d, t_t, t_v = calls["decode_pruned"]["us"], calls["target_decode_T_t"]["us"], calls["verify"]["us"]
+        out["latency_model_eq1_3"] = {
+            "T_d_us": t_d, "T_t_us": t_t, "T_t_gamma_us": t_v, "verify_over_target_decode": round(t_v / t_t, 4),
+            "illustrative_speedup_tau_2.79": round(sd_projection(2.79, w.gamma, t_d, t_t, t_v), 3),
+            "note": "attention-only times in the paper's latency model; tau is the paper's printed chain figure"}
+        print(json.dumps(out), flush=True)
+        del c
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--case", default=None, help="run one call only (small case for profiling / sweeps)")
+    ap.add_argument("--workloads", default=None, help="comma-separated workload numbers (e.g. 2,3,4,5): time every "
+                                                      "call of the path on each, with the sweeps; one JSON line each")
     ap.add_argument("--layers", type=int, default=0)
     ap.add_argument("--frames", type=int, default=0)
     ap.add_argument("--workload", type=int, default=2)
@@ -783,6 +1043,9 @@ def main():
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
+    if args.workloads:
+        run_workloads(args)
+        return
     if args.case:
         run_case(args)
         return

@@ -360,11 +360,13 @@ SEL_WINDOW_FRONT, SEL_WINDOW_MIDDLE, SEL_WINDOW_END, SEL_FRAMES, SEL_RANDOM = 0,
 
 
 def select_baseline(mode: int, n_frames, tokens_per_frame: int, k_total, kept_cu, seed: int = 0,
-                    device="cuda"):
-    """Returns (kept_idx, kept_n): the index lists of an attention-agnostic selector."""
+                    device="cuda", kept_idx: torch.Tensor | None = None, want_counts: bool = True):
+    """Returns (kept_idx, kept_n): the index lists of an attention-agnostic selector (kept_n None
+    when the counts are not asked for)."""
     batch = len(n_frames)
-    kept_idx = torch.empty(max(int(kept_cu[-1]), 1), dtype=torch.int32, device=device)
-    kept_n = torch.empty(batch, dtype=torch.int32, device=device)
+    if kept_idx is None:
+        kept_idx = torch.empty(max(int(kept_cu[-1]), 1), dtype=torch.int32, device=device)
+    kept_n = torch.empty(batch, dtype=torch.int32, device=device) if want_counts else None
     rc = lib().specvlm_select_baseline(int(mode), int(seed), _i32(n_frames), int(tokens_per_frame), _i32(k_total),
                                        _i32(kept_cu), batch, _ptr(kept_idx), _ptr(kept_n), _stream())
     _check(rc, "specvlm_select_baseline")
@@ -418,18 +420,24 @@ def verify_tree_attn(kv: KvCache, q: torch.Tensor, parents: torch.Tensor, sm_sca
     return out
 
 
+def accept_tree_buffers(batch: int, n_nodes: int, vocab: int, device, want_argmax: bool = False):
+    """Output tensors and scratch of accept_tree, for callers that reuse them across calls:
+    (accept_len, next_token, path, argmax or None, ws)."""
+    n = torch.empty(batch, dtype=torch.int32, device=device)
+    nxt = torch.empty(batch, dtype=torch.int32, device=device)
+    path = torch.empty((batch, n_nodes), dtype=torch.int32, device=device)
+    g = torch.empty((batch, n_nodes), dtype=torch.int32, device=device) if want_argmax else None
+    return n, nxt, path, g, _ws(accept_workspace_bytes(batch, n_nodes - 1, vocab), device)
+
+
 def accept_tree(target_logits: torch.Tensor, node_tokens: torch.Tensor, parents: torch.Tensor,
-                want_argmax: bool = False):
+                want_argmax: bool = False, out=None):
     """Returns (accept_len [B], next_token [B], path [B][n_nodes], argmax [B][n_nodes] or None)."""
     B, N, V = target_logits.shape
     assert target_logits.dtype == torch.float32 and target_logits.is_contiguous()
     assert node_tokens.dtype == torch.int32 and parents.dtype == torch.int32
     dev = target_logits.device
-    n = torch.empty(B, dtype=torch.int32, device=dev)
-    nxt = torch.empty(B, dtype=torch.int32, device=dev)
-    path = torch.empty((B, N), dtype=torch.int32, device=dev)
-    g = torch.empty((B, N), dtype=torch.int32, device=dev) if want_argmax else None
-    ws = _ws(accept_workspace_bytes(B, N - 1, V), dev)
+    n, nxt, path, g, ws = out if out is not None else accept_tree_buffers(B, N, V, dev, want_argmax)
     rc = lib().specvlm_accept_tree(_ptr(target_logits), _ptr(node_tokens), _ptr(parents), B, N, V, _ptr(n), _ptr(nxt),
                                    _ptr(path), _ptr(g), _ptr(ws), ws.numel(), _stream())
     _check(rc, "specvlm_accept_tree")

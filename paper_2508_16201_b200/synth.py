@@ -124,6 +124,20 @@ def plant_salient_(k_video: torch.Tensor, q_text: torch.Tensor, salient: torch.T
     k_video[:, :, idx, :] = rows.to(torch.bfloat16)
 
 
+def plant_salient_paged_(k_pool: torch.Tensor, block_table_row: torch.Tensor, video_start: int, n_video: int,
+                         q_text: torch.Tensor, salient: torch.Tensor, strength: float = 2.0) -> None:
+    """plant_salient_ for one sequence of a paged cache: k_pool bf16 [L][n_blocks][Hkv][page][d],
+    block_table_row int32 [max_blocks] of that sequence; the video occupies positions
+    video_start .. video_start + n_video - 1."""
+    page = k_pool.shape[3]
+    pos = torch.arange(video_start, video_start + n_video, device=k_pool.device)
+    blk = block_table_row.to(k_pool.device)[pos // page].long()
+    off = pos % page
+    rows = k_pool[:, blk, :, off, :].permute(1, 2, 0, 3).contiguous()          # [L][Hkv][n_video][d]
+    plant_salient_(rows, q_text, salient, strength)
+    k_pool[:, blk, :, off, :] = rows.permute(2, 0, 1, 3)
+
+
 def page_table(batch: int, max_blocks: int, n_pool_blocks: int, blocks_needed, seed: int,
                device) -> torch.Tensor:
     """Scattered block table [batch][max_blocks] (int32): a seeded permutation of the pool;

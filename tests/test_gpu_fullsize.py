@@ -228,16 +228,6 @@ def test_scores_cfg4_shape_2_layers_one_by_the_oracle():
     assert float(both.sum()) <= 1.0 and float(both.min()) >= 0.0
 
 
-def _plant_paged(cache, b, nv, q_b, salient):
-    """plant_salient_ on the video rows (positions 0 .. nv-1) of sequence b of a paged cache."""
-    pos = torch.arange(nv, device=cache.k.device)
-    blk = cache.block_table[b, pos // 64].long()
-    off = pos % 64
-    rows = cache.k[:, blk, :, off, :].permute(1, 2, 0, 3).contiguous()      # [L][H][nv][D]
-    synth.plant_salient_(rows, q_b, salient)
-    cache.k[:, blk, :, off, :] = rows.permute(2, 0, 1, 3)
-
-
 def test_scores_cfg5_ragged_paged_batch_of_16():
     """Token rating on workload 5: 16 sequences of 32-128 frames and 64-227 language queries in
     64-token pages scattered over the pool, one call for the batch; 2 of 80 layers run, the oracle
@@ -255,7 +245,8 @@ def test_scores_cfg5_ragged_paged_batch_of_16():
         video_cu.append(video_cu[-1] + nv[b])
     q = synth.randn_bf16((L, text_cu[-1], w.t_q_heads, D), "cuda", 133, "Qtext")
     for b in range(B):
-        _plant_paged(cache, b, nv[b], q[:, text_cu[b]:text_cu[b + 1]], synth.salient_set(nv[b], w.planted_permille, 133, b))
+        synth.plant_salient_paged_(cache.k, cache.block_table[b], 0, nv[b], q[:, text_cu[b]:text_cu[b + 1]],
+                                   synth.salient_set(nv[b], w.planted_permille, 133, b))
     from gpu_util import host_view
     k_host = host_view(cache.k[1:2], cache.block_table, lens)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
