@@ -366,8 +366,8 @@ int32_t specvlm_compact_tree_kv(const specvlm_kv_t* kv, const int32_t* path, con
  * held until the process exits) instead of `ws`.
  *
  * Arguments and results are those of specvlm_accept, minus ws / ws_bytes.
- * Limit: batch * (gamma+1) * ceil(vocab / 4096) <= 16384 candidates (e.g. batch 16, gamma 8,
- * vocab 152064 needs 5472); larger problems return SPECVLM_ERR_TOO_LARGE and launch nothing.
+ * Limit: batch * (gamma+1) * ceil(vocab / 8192) <= 16384 candidates (e.g. batch 16, gamma 8,
+ * vocab 152064 needs 2736); larger problems return SPECVLM_ERR_TOO_LARGE and launch nothing.
  * The call allocates and frees nothing, on the host side or the device side.
  * The first call on each device looks up the device address of that device's copy of the array
  * (a cheap runtime query, cached afterwards); make that first call with the device current and

@@ -1,6 +1,9 @@
-// Step 4c: greedy acceptance.  Kernel 1 streams the fp32 logits once (16-byte loads) and leaves
-// one (max, lowest index) candidate per (row, vocab chunk); kernel 2 finishes the argmax of the
-// gamma+1 rows of a sequence and counts the leading draft tokens that equal it.
+// Step 4c: greedy acceptance.  Kernel 1 streams the fp32 logits once (16-byte loads, all of a
+// thread's loads in flight together) and leaves one (max, lowest index) candidate per (row, vocab
+// chunk); kernel 2 finishes the argmax of the gamma+1 rows of a sequence and counts the leading
+// draft tokens that equal it.  Kernel 2 is launched with programmatic stream serialization: its
+// CTAs are scheduled while kernel 1 still runs and wait (griddepcontrol.wait) for kernel 1's
+// results, so the second launch costs no gap on the stream.
 #include <mutex>
 
 #include "common.cuh"
@@ -8,8 +11,9 @@
 
 namespace specvlm {
 
-constexpr int kAcceptChunk = 4096;     // logits per CTA in kernel 1
 constexpr int kAcceptThreads = 256;
+constexpr int kAcceptVec = 8;                                      // float4 loads per thread, all issued up front
+constexpr int kAcceptChunk = kAcceptThreads * kAcceptVec * 4;      // 8192 logits per CTA in kernel 1
 
 struct Cand {
   float v;
@@ -26,6 +30,8 @@ __device__ __forceinline__ void take_better(float& av, int& ai, float bv, int bi
 
 __global__ void __launch_bounds__(kAcceptThreads)
 accept_partial_kernel(const float* __restrict__ logits, int vocab, int n_chunks, Cand* __restrict__ part) {
+  // the dependent kernel may be scheduled from now on; it waits for this grid's completion itself
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int row = blockIdx.y, chunk = blockIdx.x;
   const float* base = logits + (size_t)row * vocab;
   const int lo = chunk * kAcceptChunk;
@@ -35,14 +41,20 @@ accept_partial_kernel(const float* __restrict__ logits, int vocab, int n_chunks,
   if (((reinterpret_cast<uintptr_t>(base + lo)) & 15u) == 0) {
     const int n4 = (hi - lo) >> 2;
     const float4* b4 = reinterpret_cast<const float4*>(base + lo);
-    for (int k = threadIdx.x; k < n4; k += kAcceptThreads) {
-      const float4 x = __ldcs(b4 + k);
-      const int i0 = lo + 4 * k;
+    float4 x[kAcceptVec];
+#pragma unroll
+    for (int u = 0; u < kAcceptVec; ++u) {
+      const int k = threadIdx.x + u * kAcceptThreads;
+      x[u] = k < n4 ? __ldcs(b4 + k) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    }
+#pragma unroll
+    for (int u = 0; u < kAcceptVec; ++u) {
+      const int i0 = lo + 4 * (threadIdx.x + u * kAcceptThreads);
       // ascending index with strict '>' keeps the lowest index among equals
-      if (x.x > bv) { bv = x.x; bi = i0; }
-      if (x.y > bv) { bv = x.y; bi = i0 + 1; }
-      if (x.z > bv) { bv = x.z; bi = i0 + 2; }
-      if (x.w > bv) { bv = x.w; bi = i0 + 3; }
+      if (x[u].x > bv) { bv = x[u].x; bi = i0; }
+      if (x[u].y > bv) { bv = x[u].y; bi = i0 + 1; }
+      if (x[u].z > bv) { bv = x[u].z; bi = i0 + 2; }
+      if (x[u].w > bv) { bv = x[u].w; bi = i0 + 3; }
     }
     for (int i = lo + 4 * n4 + threadIdx.x; i < hi; i += kAcceptThreads) take_better(bv, bi, base[i], i);
   } else {
@@ -68,16 +80,20 @@ accept_partial_kernel(const float* __restrict__ logits, int vocab, int n_chunks,
 }
 
 // one warp per (sequence, t); one CTA of (gamma+1) warps per sequence
-__global__ void accept_finish_kernel(const Cand* __restrict__ part, int n_chunks,
+__global__ void accept_finish_kernel(const Cand* part, int n_chunks,
                                      const int32_t* __restrict__ draft, int gamma,
                                      int32_t* __restrict__ accept_len, int32_t* __restrict__ next_token,
                                      int32_t* __restrict__ g_out) {
   __shared__ int g_sm[16];
   const int b = blockIdx.x, t = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const Cand* row = part + ((size_t)b * (gamma + 1) + t) * n_chunks;
+  asm volatile("griddepcontrol.wait;" ::: "memory");         // kernel 1 has completed, its candidates are visible
   float bv = -INFINITY;
   int bi = 0x7fffffff;
-  for (int c = lane; c < n_chunks; c += 32) take_better(bv, bi, row[c].v, row[c].i);
+  for (int c = lane; c < n_chunks; c += 32) {
+    const int2 raw = __ldcg(reinterpret_cast<const int2*>(row + c));     // from L2: written by the grid before
+    take_better(bv, bi, __int_as_float(raw.x), raw.y);
+  }
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) {
     const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
@@ -99,7 +115,7 @@ __global__ void accept_finish_kernel(const Cand* __restrict__ part, int n_chunks
 
 // Tree drafting: one warp per node finishes its arg-max, then one thread walks from the root to
 // the child whose token is the target's choice at the current node, as long as there is one.
-__global__ void accept_tree_finish_kernel(const Cand* __restrict__ part, int n_chunks,
+__global__ void accept_tree_finish_kernel(const Cand* part, int n_chunks,
                                           const int32_t* __restrict__ node_tokens,
                                           const int32_t* __restrict__ parents, int n_nodes,
                                           int32_t* __restrict__ accept_len, int32_t* __restrict__ next_token,
@@ -107,9 +123,13 @@ __global__ void accept_tree_finish_kernel(const Cand* __restrict__ part, int n_c
   __shared__ int g_sm[32];
   const int b = blockIdx.x, t = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const Cand* row = part + ((size_t)b * n_nodes + t) * n_chunks;
+  asm volatile("griddepcontrol.wait;" ::: "memory");         // kernel 1 has completed, its candidates are visible
   float bv = -INFINITY;
   int bi = 0x7fffffff;
-  for (int c = lane; c < n_chunks; c += 32) take_better(bv, bi, row[c].v, row[c].i);
+  for (int c = lane; c < n_chunks; c += 32) {
+    const int2 raw = __ldcg(reinterpret_cast<const int2*>(row + c));
+    take_better(bv, bi, __int_as_float(raw.x), raw.y);
+  }
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) {
     const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
@@ -141,6 +161,24 @@ __global__ void accept_tree_finish_kernel(const Cand* __restrict__ part, int n_c
     accept_len[b] = n;
     next_token[b] = g_sm[cur];
   }
+}
+
+// Launches `kern` so that it may be scheduled while the kernel before it in the stream still runs
+// (programmatic stream serialization); the kernel itself waits for that kernel's results.
+template <typename... KArgs, typename... Args>
+static int32_t launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...) != cudaSuccess) return SPECVLM_ERR_CUDA;
+  return launch_status();
 }
 
 // Built-in scratch of specvlm_accept_noalloc: room for kStaticCands (row, vocab chunk) candidates.
@@ -177,10 +215,9 @@ extern "C" int32_t specvlm_accept(const float* target_logits, const int32_t* dra
       target_logits, vocab, n_chunks, part);
   int32_t rc = launch_status();
   if (rc != SPECVLM_OK) return rc;
-  accept_finish_kernel<<<(unsigned)batch, 32 * (gamma + 1), 0, st>>>(part, n_chunks, draft_tokens, gamma,
-                                                                     accept_len, next_token,
-                                                                     target_argmax_or_null);
-  return launch_status();
+  return launch_dependent(accept_finish_kernel, dim3((unsigned)batch), dim3(32u * (gamma + 1)), st,
+                          static_cast<const Cand*>(part), n_chunks, draft_tokens, gamma, accept_len, next_token,
+                          target_argmax_or_null);
 }
 
 extern "C" int32_t specvlm_accept_noalloc(const float* target_logits, const int32_t* draft_tokens,
@@ -219,10 +256,9 @@ extern "C" int32_t specvlm_accept_noalloc(const float* target_logits, const int3
       target_logits, vocab, n_chunks, part);
   int32_t rc = launch_status();
   if (rc != SPECVLM_OK) return rc;
-  accept_finish_kernel<<<(unsigned)batch, 32 * (gamma + 1), 0, st>>>(part, n_chunks, draft_tokens, gamma,
-                                                                     accept_len, next_token,
-                                                                     target_argmax_or_null);
-  return launch_status();
+  return launch_dependent(accept_finish_kernel, dim3((unsigned)batch), dim3(32u * (gamma + 1)), st,
+                          static_cast<const Cand*>(part), n_chunks, draft_tokens, gamma, accept_len, next_token,
+                          target_argmax_or_null);
 }
 
 extern "C" int32_t specvlm_accept_tree(const float* target_logits, const int32_t* node_tokens,
@@ -243,8 +279,7 @@ extern "C" int32_t specvlm_accept_tree(const float* target_logits, const int32_t
       target_logits, vocab, n_chunks, part);
   int32_t rc = launch_status();
   if (rc != SPECVLM_OK) return rc;
-  accept_tree_finish_kernel<<<(unsigned)batch, 32 * n_nodes, 0, st>>>(part, n_chunks, node_tokens, parents, n_nodes,
-                                                                      accept_len, next_token, path,
-                                                                      target_argmax_or_null);
-  return launch_status();
+  return launch_dependent(accept_tree_finish_kernel, dim3((unsigned)batch), dim3(32u * n_nodes), st,
+                          static_cast<const Cand*>(part), n_chunks, node_tokens, parents, n_nodes, accept_len,
+                          next_token, path, target_argmax_or_null);
 }

@@ -30,6 +30,11 @@ attn_rows16_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
   constexpr int KSTEPS = D / 16;
   constexpr int NT_O = D / 8;
   constexpr int OPITCH = D + 8;            // fp32 pitch of the end-of-kernel merge buffer
+  // A consumer group must see every phase of the ring slots it waits on: with the groups on
+  // alternate tiles that holds only when a slot always belongs to the same group.  (A wait on a
+  // phase two behind the barrier returns at once, the group then releases a slot it never read,
+  // and the surplus arrival on the barrier is undefined behaviour: it faulted the kernel.)
+  static_assert(STAGES % NG == 0, "ring depth must be a multiple of the number of consumer groups");
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -278,10 +283,16 @@ attn_rows16_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
   l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
   {
     float* ow = o_sm + warp * 16 * OPITCH;
+    // only the rows in use (7 of the 16 for the 7-head group of a decode step)
+    if (row0 < p.rows) {
 #pragma unroll
-    for (int nt = 0; nt < NT_O; ++nt) {
-      *reinterpret_cast<float2*>(ow + row0 * OPITCH + nt * 8 + col) = make_float2(o[nt][0], o[nt][1]);
-      *reinterpret_cast<float2*>(ow + row1 * OPITCH + nt * 8 + col) = make_float2(o[nt][2], o[nt][3]);
+      for (int nt = 0; nt < NT_O; ++nt)
+        *reinterpret_cast<float2*>(ow + row0 * OPITCH + nt * 8 + col) = make_float2(o[nt][0], o[nt][1]);
+    }
+    if (row1 < p.rows) {
+#pragma unroll
+      for (int nt = 0; nt < NT_O; ++nt)
+        *reinterpret_cast<float2*>(ow + row1 * OPITCH + nt * 8 + col) = make_float2(o[nt][2], o[nt][3]);
     }
     if ((lane & 3) == 0) {
       m_sm[warp * 16 + row0] = m0;
@@ -291,39 +302,33 @@ attn_rows16_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     }
   }
   asm volatile("bar.sync 1, %0;" ::"n"(128 * NG) : "memory");
-  // The weights of the NW partials are the same for every channel of a row: one thread per
-  // (warp, row) turns its (max, sum) into the weight 2^(m - M) / den in place, thread (0, row)
-  // also leaves the row's log2-sum-exp in l_sm.
-  if (tid < NW * 16) {
-    const int w_me = tid >> 4, r = tid & 15;
+  // Every thread of the final pass derives its row's weights 2^(m_w - M) / den itself (16 shared
+  // loads and NW exponentials): cheaper than a separate weight phase behind two more barriers.
+  const int item = lb * p.n_kv_heads + g;
+  for (int idx = tid; idx < p.rows * (D / 4); idx += 128 * NG) {
+    const int r = idx / (D / 4), c = (idx - r * (D / 4)) * 4;
     float M = -INFINITY;
 #pragma unroll
     for (int w = 0; w < NW; ++w) M = fmaxf(M, m_sm[w * 16 + r]);
     float den = 0.f;
-    if (M != -INFINITY) {
+    float wt[NW];
 #pragma unroll
-      for (int w = 0; w < NW; ++w) den += l_sm[w * 16 + r] * fast_exp2(m_sm[w * 16 + r] - M);
+    for (int w = 0; w < NW; ++w) {
+      wt[w] = M != -INFINITY ? fast_exp2(m_sm[w * 16 + r] - M) : 0.f;
+      den += l_sm[w * 16 + r] * wt[w];
     }
-    const float wt = den > 0.f ? fast_exp2(m_sm[tid] - M) / den : 0.f;
-    asm volatile("bar.sync 2, %0;" ::"n"(NW * 16) : "memory");        // every (max, sum) has been read
-    m_sm[tid] = wt;
-    if (w_me == 0) l_sm[r] = den > 0.f ? M + log2f(den) : -INFINITY;
-  }
-  asm volatile("bar.sync 1, %0;" ::"n"(128 * NG) : "memory");
-  const int item = lb * p.n_kv_heads + g;
-  for (int idx = tid; idx < p.rows * (D / 4); idx += 128 * NG) {
-    const int r = idx / (D / 4), c = (idx - r * (D / 4)) * 4;
+    const float inv = den > 0.f ? 1.f / den : 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
     for (int w = 0; w < NW; ++w) {
-      const float f = m_sm[w * 16 + r];
+      const float f = wt[w] * inv;
       const float4 x = *reinterpret_cast<const float4*>(o_sm + (w * 16 + r) * OPITCH + c);
       acc.x += x.x * f;
       acc.y += x.y * f;
       acc.z += x.z * f;
       acc.w += x.w * f;
     }
-    const float lse2 = l_sm[r];
+    const float lse2 = den > 0.f ? M + log2f(den) : -INFINITY;
     if (p.n_splits == 1) {
       const int t = r / p.group, h = g * p.group + (r - t * p.group);
       const size_t orow = ((size_t)lb * p.n_q + t) * p.n_q_heads + h;

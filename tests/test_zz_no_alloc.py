@@ -43,8 +43,8 @@ def test_noalloc_matches_accept_on_two_calls_in_a_row():
 def test_noalloc_rejects_oversized_problem_and_bad_arguments():
     logits = torch.zeros((1, 2, 8), dtype=torch.float32, device="cuda")
     L = specvlm.lib()
-    # 64 * 9 * ceil(152064 / 4096) = 21888 candidates > 16384: refused before any launch
-    rc = L.specvlm_accept_noalloc(logits.data_ptr(), logits.data_ptr(), 64, 8, 152064, logits.data_ptr(),
+    # 128 * 9 * ceil(152064 / 8192) = 21888 candidates > 16384: refused before any launch
+    rc = L.specvlm_accept_noalloc(logits.data_ptr(), logits.data_ptr(), 128, 8, 152064, logits.data_ptr(),
                                   logits.data_ptr(), None, None)
     assert rc == specvlm.ERR_TOO_LARGE
     assert "built-in scratch" in specvlm.status_string(rc)
