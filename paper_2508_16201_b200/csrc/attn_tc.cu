@@ -541,6 +541,139 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       // (A used row always has its own bit set, so a zero mask also marks an unused row.)
       // The chain keeps the equivalent limit form: key tok is visible to token t when tok < lim.
       const int win0 = kv_len - p.n_win;
+      float2* const seg_stats = stats;
+      if constexpr (M == 128) {
+        // ------------------------------------------------------------ 128-row windows: a thread owns a row
+        // With M = 128 row r sits in TMEM lane r, so thread `lane` of the warp of quadrant q reads row
+        // 32 q + lane whole (tcgen05.ld 32x32b): its maximum and sum need no shuffles, its 128
+        // probabilities leave as sixteen 16-byte stores into the swizzled P tile, and the TMEM load of
+        // the next 32 columns is in flight while the current 32 are worked on.
+        const int my_row = 32 * quarter + lane;
+        const bool warp_on = p.rows > 32 * quarter;         // warp-uniform: some row of this quadrant is in use
+        uint32_t my_a;                                       // the row's window mask (tree) or key limit (chain)
+        if constexpr (TREE) {
+          my_a = my_row < p.rows ? __ldg(p.anc + (size_t)sg.b * p.n_win + p.q0 + my_row / p.group) : 0u;
+        } else {
+          my_a = my_row < p.rows ? (uint32_t)(win0 + p.q0 + my_row / p.group + 1) : 0u;
+        }
+        float m_row = -INFINITY, l_row = 0.f;
+        const uint32_t prow = p_sm + grp * P_BYTES + my_row * 128;
+        const uint32_t psw = (uint32_t)(my_row & 7);
+
+        for (int j = (i0 + grp) & 1; j < sg.n_tiles; j += 2) {
+          const int i = i0 + j;
+          const int tile_tok0 = (sg.tile0 + j) * kBigTokens;
+          const bool need_mask = tile_tok0 + kBigTokens > win0 + (TREE ? 0 : 1);
+          SM_WAIT(bar_s_full + 8 * grp, (i >> 1) & 1);
+          tc_fence_after_sync();
+          if (!warp_on) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_s_empty + 8 * grp);
+            if (i >= 2) SM_WAIT(bar_p_empty + 8 * grp, ((i >> 1) - 1) & 1);
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_p_full + 8 * grp);
+            continue;
+          }
+          const uint32_t saddr = tmem_base + ((uint32_t)(32 * quarter) << 16) + C::COL_S + grp * kBigTokens;
+          if (__builtin_expect(need_mask, 0)) {
+            // the out-of-line mask routine works on 16-lane halves with two rows per thread
+#pragma unroll 1
+            for (int h = 0; h < nh; ++h) {
+              const uint32_t a0 = __shfl_sync(0xffffffffu, my_a, 16 * h + lr);
+              const uint32_t a1 = __shfl_sync(0xffffffffu, my_a, 16 * h + lr + 8);
+              mask_s_half<TREE>(saddr + ((uint32_t)(16 * h) << 16), tile_tok0, win0, lc, a0, a1);
+            }
+          }
+          uint32_t va[32], vb[32];
+          // pass 1: the row's maximum over the tile's 128 logits (raw products: the scale is positive)
+          float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+          tmem_ld_x32(saddr, va);
+#pragma unroll 1
+          for (int cc = 0; cc < 2; ++cc) {
+            tmem_ld_wait();
+            tmem_ld_x32(saddr + (2 * cc + 1) * 32, vb);
+#pragma unroll
+            for (int k = 0; k < 32; ++k) mx4[k & 3] = fmaxf(mx4[k & 3], __uint_as_float(va[k]));
+            tmem_ld_wait();
+            if (cc == 0) tmem_ld_x32(saddr + 64, va);
+#pragma unroll
+            for (int k = 0; k < 32; ++k) mx4[k & 3] = fmaxf(mx4[k & 3], __uint_as_float(vb[k]));
+          }
+          const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
+          // the group's previous product has completed: P may be overwritten, O may be rescaled
+          if (i >= 2) SM_WAIT(bar_p_empty + 8 * grp, ((i >> 1) - 1) & 1);
+          if (j < 2) {
+            m_row = mx;                          // the group's first tile of the item: O is overwritten
+          } else {
+            const bool up = mx > m_row + kRescaleThreshold;
+            if (__builtin_expect(__any_sync(0xffffffffu, up) != 0, 0)) {
+              const float a = up ? fast_exp2(m_row - mx) : 1.f;
+              if (up) m_row = mx;
+              l_row *= a;
+              tc_fence_after_sync();
+#pragma unroll 1
+              for (int h = 0; h < nh; ++h) {
+                const float f0 = __shfl_sync(0xffffffffu, a, 16 * h + lr);
+                const float f1 = __shfl_sync(0xffffffffu, a, 16 * h + lr + 8);
+                rescale_o_half<D>(tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + C::COL_O + grp * D, f0, f1);
+              }
+              tc_fence_before_sync();
+            }
+          }
+          // pass 2: p = 2^(s * scale - m), with a row that sees nothing yet kept at zero
+          const float nmu = m_row == -INFINITY ? 0.f : -m_row;
+          float ps[2] = {0.f, 0.f};
+          tmem_ld_x32(saddr, va);
+#pragma unroll 1
+          for (int cc = 0; cc < 2; ++cc) {       // the tile's two 64-token blocks
+            const uint32_t pblk = prow + cc * (M * 128);
+            tmem_ld_wait();
+            tmem_ld_x32(saddr + (2 * cc + 1) * 32, vb);
+#pragma unroll
+            for (int k4 = 0; k4 < 4; ++k4) {     // 8 logits -> one 16-byte chunk of the row
+              uint32_t w[4];
+#pragma unroll
+              for (int u = 0; u < 4; ++u) {
+                const float p0 = fast_exp2(fmaf(__uint_as_float(va[8 * k4 + 2 * u]), p.scale_log2, nmu));
+                const float p1 = fast_exp2(fmaf(__uint_as_float(va[8 * k4 + 2 * u + 1]), p.scale_log2, nmu));
+                ps[u & 1] += p0 + p1;
+                w[u] = pack_bf16x2(p0, p1);
+              }
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(pblk + (((uint32_t)k4 ^ psw) << 4)),
+                           "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+            }
+            tmem_ld_wait();
+            if (cc == 0) {
+              tmem_ld_x32(saddr + 64, va);
+            } else {
+              tc_fence_before_sync();            // every logit of the tile has been read: S is free
+              __syncwarp();
+              if (lane == 0) mbar_arrive(bar_s_empty + 8 * grp);
+            }
+#pragma unroll
+            for (int k4 = 0; k4 < 4; ++k4) {
+              uint32_t w[4];
+#pragma unroll
+              for (int u = 0; u < 4; ++u) {
+                const float p0 = fast_exp2(fmaf(__uint_as_float(vb[8 * k4 + 2 * u]), p.scale_log2, nmu));
+                const float p1 = fast_exp2(fmaf(__uint_as_float(vb[8 * k4 + 2 * u + 1]), p.scale_log2, nmu));
+                ps[u & 1] += p0 + p1;
+                w[u] = pack_bf16x2(p0, p1);
+              }
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(pblk + (((uint32_t)(4 + k4) ^ psw) << 4)),
+                           "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+            }
+          }
+          l_row += ps[0] + ps[1];
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_p_full + 8 * grp);
+        }
+        // publish this group's row statistics for the merge below
+        if (seg_idx >= 1) SM_WAIT(bar_o_empty, (seg_idx - 1) & 1);
+        if (warp_on) seg_stats[grp * M + my_row] = make_float2(m_row, l_row);
+      } else {
       uint32_t vis[NH][2];
       int lim[NH][2];
       float m_used[NH][2], l_sum[NH][2];
@@ -681,27 +814,29 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         if (lane == 0) mbar_arrive(bar_p_full + 8 * grp);
       }
 
+        // publish this group's row statistics for the merge below.  A group may get here while the
+        // other one still reads the previous segment's statistics: wait until both have left that
+        // epilogue (the barrier the PV issuer waits on as well)
+        if (seg_idx >= 1) SM_WAIT(bar_o_empty, (seg_idx - 1) & 1);
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+          if (h >= nh) break;
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            float lt = l_sum[h][e];
+            lt += __shfl_xor_sync(0xffffffffu, lt, 1);
+            lt += __shfl_xor_sync(0xffffffffu, lt, 2);
+            if ((lane & 3) == 0) seg_stats[grp * M + row0(h) + lr + 8 * e] = make_float2(m_used[h][e], lt);
+          }
+        }
+      }
+
       // ---------------------------------------------------------------- end of the item's segment
-      // publish this group's row statistics, then merge the two groups' accumulators:
+      // merge the two groups' accumulators:
       //   O = (w0 O0 + w1 O1) / (w0 l0 + w1 l1),  w_g = 2^(m_g - max(m0, m1))
       const bool complete = sg.tile0 == 0 && sg.n_tiles == sg.item_tiles;
       const int lb = sg.layer * p.batch + sg.b;
       const int slot = partial_slot(cta, T0, sg.item_begin);
-      // a group may get here while the other one still reads the previous segment's statistics:
-      // wait until both have left that epilogue (the barrier the PV issuer waits on as well)
-      float2* const seg_stats = stats;
-      if (seg_idx >= 1) SM_WAIT(bar_o_empty, (seg_idx - 1) & 1);
-#pragma unroll
-      for (int h = 0; h < NH; ++h) {
-        if (h >= nh) break;
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          float lt = l_sum[h][e];
-          lt += __shfl_xor_sync(0xffffffffu, lt, 1);
-          lt += __shfl_xor_sync(0xffffffffu, lt, 2);
-          if ((lane & 3) == 0) seg_stats[grp * M + row0(h) + lr + 8 * e] = make_float2(m_used[h][e], lt);
-        }
-      }
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_ep_stats);
       SM_WAIT(bar_ep_stats, seg_idx & 1);
