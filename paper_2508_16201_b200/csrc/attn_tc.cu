@@ -586,85 +586,97 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             }
           }
           uint32_t va[32], vb[32];
-          // pass 1: the row's maximum over the tile's 128 logits (raw products: the scale is positive)
-          float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-          tmem_ld_x32(saddr, va);
-#pragma unroll 1
-          for (int cc = 0; cc < 2; ++cc) {
-            tmem_ld_wait();
-            tmem_ld_x32(saddr + (2 * cc + 1) * 32, vb);
-#pragma unroll
-            for (int k = 0; k < 32; ++k) mx4[k & 3] = fmaxf(mx4[k & 3], __uint_as_float(va[k]));
-            tmem_ld_wait();
-            if (cc == 0) tmem_ld_x32(saddr + 64, va);
-#pragma unroll
-            for (int k = 0; k < 32; ++k) mx4[k & 3] = fmaxf(mx4[k & 3], __uint_as_float(vb[k]));
-          }
-          const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
           // the group's previous product has completed: P may be overwritten, O may be rescaled
           if (i >= 2) SM_WAIT(bar_p_empty + 8 * grp, ((i >> 1) - 1) & 1);
           if (j < 2) {
-            m_row = mx;                          // the group's first tile of the item: O is overwritten
-          } else {
+            // The group's first tile of the item (O is overwritten by its product): the row's reference
+            // maximum is the tile's own, found by a pass of its own over the 128 logits (raw products:
+            // the scale is positive).
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            tmem_ld_x32(saddr, va);
+#pragma unroll 1
+            for (int cc = 0; cc < 2; ++cc) {
+              tmem_ld_wait();
+              tmem_ld_x32(saddr + (2 * cc + 1) * 32, vb);
+#pragma unroll
+              for (int k = 0; k < 32; ++k) mx4[k & 3] = fmaxf(mx4[k & 3], __uint_as_float(va[k]));
+              tmem_ld_wait();
+              if (cc == 0) tmem_ld_x32(saddr + 64, va);
+#pragma unroll
+              for (int k = 0; k < 32; ++k) mx4[k & 3] = fmaxf(mx4[k & 3], __uint_as_float(vb[k]));
+            }
+            m_row = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
+          }
+          // Every later tile takes ONE pass: p = 2^(s * scale - m) against the reference maximum the row
+          // already has, the tile's own maximum being gathered on the way.  Only if that maximum turns
+          // out more than the lazy-rescale threshold above the reference (a warp vote; rare after the
+          // first tiles) is the reference raised, O rescaled in tensor memory and the pass repeated: S
+          // stays in place until the decision is taken, and the probabilities of the abandoned pass are
+          // simply overwritten (whatever they were, up to infinity, they never reach a product).
+          float ps[2];
+#pragma unroll 1
+          for (int attempt = 0; attempt < 2; ++attempt) {
+            const float nmu = m_row == -INFINITY ? 0.f : -m_row;   // a row that sees nothing yet stays at zero
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            ps[0] = ps[1] = 0.f;
+            tmem_ld_x32(saddr, va);
+#pragma unroll 1
+            for (int cc = 0; cc < 2; ++cc) {     // the tile's two 64-token blocks
+              const uint32_t pblk = prow + cc * (M * 128);
+              tmem_ld_wait();
+              tmem_ld_x32(saddr + (2 * cc + 1) * 32, vb);
+#pragma unroll
+              for (int k4 = 0; k4 < 4; ++k4) {   // 8 logits -> one 16-byte chunk of the row
+                uint32_t w[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                  const float s0 = __uint_as_float(va[8 * k4 + 2 * u]), s1 = __uint_as_float(va[8 * k4 + 2 * u + 1]);
+                  mx4[u] = fmaxf(mx4[u], fmaxf(s0, s1));
+                  const float p0 = fast_exp2(fmaf(s0, p.scale_log2, nmu));
+                  const float p1 = fast_exp2(fmaf(s1, p.scale_log2, nmu));
+                  ps[u & 1] += p0 + p1;
+                  w[u] = pack_bf16x2(p0, p1);
+                }
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(pblk + (((uint32_t)k4 ^ psw) << 4)),
+                             "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+              }
+              tmem_ld_wait();
+              if (cc == 0) tmem_ld_x32(saddr + 64, va);
+#pragma unroll
+              for (int k4 = 0; k4 < 4; ++k4) {
+                uint32_t w[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                  const float s0 = __uint_as_float(vb[8 * k4 + 2 * u]), s1 = __uint_as_float(vb[8 * k4 + 2 * u + 1]);
+                  mx4[u] = fmaxf(mx4[u], fmaxf(s0, s1));
+                  const float p0 = fast_exp2(fmaf(s0, p.scale_log2, nmu));
+                  const float p1 = fast_exp2(fmaf(s1, p.scale_log2, nmu));
+                  ps[u & 1] += p0 + p1;
+                  w[u] = pack_bf16x2(p0, p1);
+                }
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(pblk + (((uint32_t)(4 + k4) ^ psw) << 4)),
+                             "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+              }
+            }
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
             const bool up = mx > m_row + kRescaleThreshold;
-            if (__builtin_expect(__any_sync(0xffffffffu, up) != 0, 0)) {
-              const float a = up ? fast_exp2(m_row - mx) : 1.f;
-              if (up) m_row = mx;
-              l_row *= a;
-              tc_fence_after_sync();
+            if (__builtin_expect(__any_sync(0xffffffffu, up) == 0, 1)) break;
+            // raise the reference maximum of those rows, rescale their sums and their O rows, go again
+            const float a = up ? fast_exp2(m_row - mx) : 1.f;
+            if (up) m_row = mx;
+            l_row *= a;
+            tc_fence_after_sync();
 #pragma unroll 1
-              for (int h = 0; h < nh; ++h) {
-                const float f0 = __shfl_sync(0xffffffffu, a, 16 * h + lr);
-                const float f1 = __shfl_sync(0xffffffffu, a, 16 * h + lr + 8);
-                rescale_o_half<D>(tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + C::COL_O + grp * D, f0, f1);
-              }
-              tc_fence_before_sync();
+            for (int h = 0; h < nh; ++h) {
+              const float f0 = __shfl_sync(0xffffffffu, a, 16 * h + lr);
+              const float f1 = __shfl_sync(0xffffffffu, a, 16 * h + lr + 8);
+              rescale_o_half<D>(tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + C::COL_O + grp * D, f0, f1);
             }
+            tc_fence_before_sync();
           }
-          // pass 2: p = 2^(s * scale - m), with a row that sees nothing yet kept at zero
-          const float nmu = m_row == -INFINITY ? 0.f : -m_row;
-          float ps[2] = {0.f, 0.f};
-          tmem_ld_x32(saddr, va);
-#pragma unroll 1
-          for (int cc = 0; cc < 2; ++cc) {       // the tile's two 64-token blocks
-            const uint32_t pblk = prow + cc * (M * 128);
-            tmem_ld_wait();
-            tmem_ld_x32(saddr + (2 * cc + 1) * 32, vb);
-#pragma unroll
-            for (int k4 = 0; k4 < 4; ++k4) {     // 8 logits -> one 16-byte chunk of the row
-              uint32_t w[4];
-#pragma unroll
-              for (int u = 0; u < 4; ++u) {
-                const float p0 = fast_exp2(fmaf(__uint_as_float(va[8 * k4 + 2 * u]), p.scale_log2, nmu));
-                const float p1 = fast_exp2(fmaf(__uint_as_float(va[8 * k4 + 2 * u + 1]), p.scale_log2, nmu));
-                ps[u & 1] += p0 + p1;
-                w[u] = pack_bf16x2(p0, p1);
-              }
-              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(pblk + (((uint32_t)k4 ^ psw) << 4)),
-                           "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
-            }
-            tmem_ld_wait();
-            if (cc == 0) {
-              tmem_ld_x32(saddr + 64, va);
-            } else {
-              tc_fence_before_sync();            // every logit of the tile has been read: S is free
-              __syncwarp();
-              if (lane == 0) mbar_arrive(bar_s_empty + 8 * grp);
-            }
-#pragma unroll
-            for (int k4 = 0; k4 < 4; ++k4) {
-              uint32_t w[4];
-#pragma unroll
-              for (int u = 0; u < 4; ++u) {
-                const float p0 = fast_exp2(fmaf(__uint_as_float(vb[8 * k4 + 2 * u]), p.scale_log2, nmu));
-                const float p1 = fast_exp2(fmaf(__uint_as_float(vb[8 * k4 + 2 * u + 1]), p.scale_log2, nmu));
-                ps[u & 1] += p0 + p1;
-                w[u] = pack_bf16x2(p0, p1);
-              }
-              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(pblk + (((uint32_t)(4 + k4) ^ psw) << 4)),
-                           "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
-            }
-          }
+          tc_fence_before_sync();                // every read of the tile's logits is complete: S is free
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_s_empty + 8 * grp);
           l_row += ps[0] + ps[1];
           fence_proxy_async();
           __syncwarp();

@@ -467,3 +467,50 @@ def test_scores_row_lse_entry():
     a = specvlm.stage1_scores(cache, q, [0, nt], [nv], [0], [nv], [0, nv], scale)
     b = specvlm.stage1_scores(cache, q, [0, nt], [nv], [0], [nv], [0, nv], scale, row_lse=lse)
     assert torch.equal(a, b)
+
+
+# ------------------------------------------------------------------------------- rising maxima
+@pytest.mark.parametrize("Hq,Hkv,gamma,D", [(64, 8, 8, 128),    # 72 rows: the 128-row tiles
+                                            (64, 8, 5, 128),    # 48 rows: the 64-row tiles
+                                            (28, 4, 0, 128),    # 7 rows: the decode kernel
+                                            (16, 2, 8, 64)])    # 72 rows, d = 64
+def test_attention_with_maxima_rising_along_the_sequence(Hq, Hkv, gamma, D):
+    """Random N(0,1) logits never move a row's running maximum by much after the first tile, so the
+    kernels' rescaling of the running sums and of the O accumulator would go untested.  Here the
+    keys carry a ramp along a direction u and the query rows carry +a u, +a u / 2, 0 or -a u: the
+    logits of a row rise (or fall) by about 12 log2 units per 128 tokens, with a drop half way, so
+    that the reference maximum must be raised again and again for some rows of a warp and never
+    for others."""
+    from gpu_util import make_cache
+    L, n = 2, 1500 + gamma + 1
+    cache, _, _ = make_cache(L, Hkv, D, [n, 700], paged=False, seed=90)
+    g = torch.Generator(device="cuda").manual_seed(91)
+    u = torch.randn(D, generator=g, device="cuda")
+    u = u / u.norm()
+    scale = 1.0 / math.sqrt(D)
+    a = 10.0
+    b = 12.0 / (scale * a * math.log2(math.e))                    # ramp height per 128 tokens
+    pos = torch.arange(cache.k.shape[3], device="cuda", dtype=torch.float32)
+    ramp = torch.where(pos < 800, pos, pos - 640.0) / 128.0       # rises, drops by 5 tiles' worth, rises again
+    cache.k.copy_((cache.k.float() + (b * ramp)[None, None, None, :, None] * u).to(torch.bfloat16))
+    nq = gamma + 1
+    q = synth.randn_bf16((L, 2, nq, Hq, D), "cuda", 92, "Q").float()
+    slope = torch.tensor([1.0, 0.5, 0.0, -1.0], device="cuda")[torch.arange(Hq, device="cuda") % 4]
+    q = (q + a * slope[None, None, None, :, None] * u).to(torch.bfloat16)
+    from gpu_util import host_view
+    k_host = host_view(cache.k, None, [n, 700])
+    v_host = host_view(cache.v, None, [n, 700])
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    lse = torch.empty((L, 2, nq, Hq), dtype=torch.float32, device="cuda")
+    if gamma == 0:
+        out = specvlm.draft_decode_attn(cache, q[:, :, 0].contiguous(), scale, lse=lse, d_status=status)[:, :, None]
+    else:
+        out = specvlm.verify_attn(cache, q, gamma, scale, lse=lse, d_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ref, ref_lse = _oracle_attn(bits(q), k_host, v_host, [n, 700], scale)
+    got = f64(out)
+    assert np.isfinite(got).all()
+    err = row_rel_err(got, ref)
+    assert err <= ATTN_TOL, f"row rel err {err}"
+    np.testing.assert_allclose(lse.cpu().numpy(), ref_lse, rtol=0, atol=2e-3 + 1e-4 * np.abs(ref_lse).max())

@@ -130,3 +130,39 @@ def test_tree_step_chain_verify_accept_compact(paged):
         rv, _ = oracle.compact_tree_kv(v_host[b], lens[b], n_nodes, rpath)
         assert new_lens[b] == nl == lens[b] - n_nodes + 1 + rn
         assert np.array_equal(gk[b], rk[:, :, :nl]) and np.array_equal(gv[b], rv[:, :, :nl])
+
+
+def test_tree_attention_with_maxima_rising_along_the_sequence():
+    """The 128-row tree variant on logits that rise by about 12 log2 units per 128 tokens for some
+    rows and fall for others: the reference maximum of a row has to be raised tile after tile."""
+    L, Hq, Hkv, D, n_nodes = 2, 64, 8, 128, 16
+    lens = [1400 + n_nodes, 300]
+    rng = np.random.default_rng(95)
+    cache, _, _ = make_cache(L, Hkv, D, lens, paged=False, seed=95)
+    g = torch.Generator(device="cuda").manual_seed(96)
+    u = torch.randn(D, generator=g, device="cuda")
+    u = u / u.norm()
+    scale = 1.0 / math.sqrt(D)
+    a = 10.0
+    b = 12.0 / (scale * a * math.log2(math.e))
+    pos = torch.arange(cache.k.shape[3], device="cuda", dtype=torch.float32)
+    cache.k.copy_((cache.k.float() + (b * pos / 128.0)[None, None, None, :, None] * u).to(torch.bfloat16))
+    k_host = host_view(cache.k, None, lens)
+    v_host = host_view(cache.v, None, lens)
+    parents = [_random_tree(rng, n_nodes) for _ in lens]
+    par = torch.tensor(parents, dtype=torch.int32, device="cuda")
+    q = synth.randn_bf16((L, 2, n_nodes, Hq, D), "cuda", 97, "Qt").float()
+    slope = torch.tensor([1.0, -1.0, 0.5, 0.0], device="cuda")[torch.arange(Hq, device="cuda") % 4]
+    q = (q + a * slope[None, None, None, :, None] * u).to(torch.bfloat16)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = specvlm.verify_tree_attn(cache, q, par, scale, d_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    got, qh = f64(out), bits(q)
+    assert np.isfinite(got).all()
+    worst = 0.0
+    for l in range(L):
+        for bb in range(2):
+            ref, _ = oracle.attention_tree(qh[l, bb], k_host[bb][l], v_host[bb][l], lens[bb], parents[bb], scale)
+            worst = max(worst, row_rel_err(got[l, bb], ref))
+    assert worst <= 1e-2, f"row rel err {worst}"
