@@ -1019,6 +1019,16 @@ def run_workloads(args):
             a_out = (torch.empty(B, dtype=torch.int32, device=device), torch.empty(B, dtype=torch.int32, device=device), None)
             ws_a = torch.empty(specvlm.accept_workspace_bytes(B, g, w.vocab), dtype=torch.uint8, device=device)
             acc[g] = rec(*gt.time(lambda: specvlm.accept(lg, dr, ws=ws_a, out=a_out), reps), nbytes=B * (g + 1) * w.vocab * 4)
+            # the same call four times in one graph, each on its own logits: what the call costs inside
+            # a longer graph (a lone graph launch adds about 4 us between the event and the first kernel)
+            lgs = [lg] + [torch.randn_like(lg) for _ in range(3)]
+
+            def four_calls():
+                for x in lgs:
+                    specvlm.accept(x, dr, ws=ws_a, out=a_out)
+            us4, mn4 = gt.time(four_calls, reps)
+            acc[g]["in_graph_of_4"] = rec(us4 / 4, mn4 / 4, nbytes=B * (g + 1) * w.vocab * 4)
+            del lgs
             del q, o, ws_v
         calls["verify"], calls["accept"], calls["target_decode_T_t"] = ver[w.gamma], acc[w.gamma], ver[0]
         if len(sweep_gamma) > 1:

@@ -28,79 +28,54 @@ __device__ __forceinline__ void take_better(float& av, int& ai, float bv, int bi
   }
 }
 
-// Unit = one (row, vocab chunk).  A CTA walks the units blockIdx.x, blockIdx.x + gridDim.x, ... and
-// has the next unit's loads in flight while it reduces the current one, so that a grid of a few
-// CTAs per SM keeps the memory system busy without paying a CTA launch per 32 KB.
-__device__ __forceinline__ void accept_load_unit(const float* __restrict__ logits, int vocab, int n_chunks, int unit,
-                                                 float4 (&x)[kAcceptVec], bool& vec) {
-  const int row = unit / n_chunks, chunk = unit - row * n_chunks;
+__global__ void __launch_bounds__(kAcceptThreads)
+accept_partial_kernel(const float* __restrict__ logits, int vocab, int n_chunks, Cand* __restrict__ part) {
+  // the dependent kernel may be scheduled from now on; it waits for this grid's completion itself
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int row = blockIdx.y, chunk = blockIdx.x;
   const float* base = logits + (size_t)row * vocab;
   const int lo = chunk * kAcceptChunk;
   const int hi = lo + kAcceptChunk < vocab ? lo + kAcceptChunk : vocab;
-  vec = ((reinterpret_cast<uintptr_t>(base + lo)) & 15u) == 0;
-  if (vec) {
+  float bv = -INFINITY;
+  int bi = 0x7fffffff;
+  if (((reinterpret_cast<uintptr_t>(base + lo)) & 15u) == 0) {
     const int n4 = (hi - lo) >> 2;
     const float4* b4 = reinterpret_cast<const float4*>(base + lo);
+    float4 x[kAcceptVec];
 #pragma unroll
     for (int u = 0; u < kAcceptVec; ++u) {
       const int k = threadIdx.x + u * kAcceptThreads;
       x[u] = k < n4 ? __ldcs(b4 + k) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
     }
+#pragma unroll
+    for (int u = 0; u < kAcceptVec; ++u) {
+      const int i0 = lo + 4 * (threadIdx.x + u * kAcceptThreads);
+      // ascending index with strict '>' keeps the lowest index among equals
+      if (x[u].x > bv) { bv = x[u].x; bi = i0; }
+      if (x[u].y > bv) { bv = x[u].y; bi = i0 + 1; }
+      if (x[u].z > bv) { bv = x[u].z; bi = i0 + 2; }
+      if (x[u].w > bv) { bv = x[u].w; bi = i0 + 3; }
+    }
+    for (int i = lo + 4 * n4 + threadIdx.x; i < hi; i += kAcceptThreads) take_better(bv, bi, base[i], i);
+  } else {
+    for (int i = lo + threadIdx.x; i < hi; i += kAcceptThreads) take_better(bv, bi, base[i], i);
   }
-}
-
-__global__ void __launch_bounds__(kAcceptThreads)
-accept_partial_kernel(const float* __restrict__ logits, int vocab, int n_chunks, int n_units, Cand* __restrict__ part) {
-  // the dependent kernel may be scheduled from now on; it waits for this grid's completion itself
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+    const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+    take_better(bv, bi, ov, oi);
+  }
   __shared__ float sv[kAcceptThreads / 32];
   __shared__ int si[kAcceptThreads / 32];
-  float4 cur[kAcceptVec], nxt[kAcceptVec];
-  bool cur_vec = false, nxt_vec = false;
-  int unit = blockIdx.x;
-  if (unit < n_units) accept_load_unit(logits, vocab, n_chunks, unit, cur, cur_vec);
-  for (; unit < n_units; unit += gridDim.x) {
-    const int next = unit + gridDim.x;
-    if (next < n_units) accept_load_unit(logits, vocab, n_chunks, next, nxt, nxt_vec);
-    const int row = unit / n_chunks, chunk = unit - row * n_chunks;
-    const float* base = logits + (size_t)row * vocab;
-    const int lo = chunk * kAcceptChunk;
-    const int hi = lo + kAcceptChunk < vocab ? lo + kAcceptChunk : vocab;
-    float bv = -INFINITY;
-    int bi = 0x7fffffff;
-    if (cur_vec) {
-#pragma unroll
-      for (int u = 0; u < kAcceptVec; ++u) {
-        const int i0 = lo + 4 * (threadIdx.x + u * kAcceptThreads);
-        // ascending index with strict '>' keeps the lowest index among equals
-        if (cur[u].x > bv) { bv = cur[u].x; bi = i0; }
-        if (cur[u].y > bv) { bv = cur[u].y; bi = i0 + 1; }
-        if (cur[u].z > bv) { bv = cur[u].z; bi = i0 + 2; }
-        if (cur[u].w > bv) { bv = cur[u].w; bi = i0 + 3; }
-      }
-      for (int i = lo + 4 * ((hi - lo) >> 2) + threadIdx.x; i < hi; i += kAcceptThreads) take_better(bv, bi, base[i], i);
-    } else {
-      for (int i = lo + threadIdx.x; i < hi; i += kAcceptThreads) take_better(bv, bi, base[i], i);
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-      const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
-      const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
-      take_better(bv, bi, ov, oi);
-    }
-    if ((threadIdx.x & 31) == 0) {
-      sv[threadIdx.x >> 5] = bv;
-      si[threadIdx.x >> 5] = bi;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      for (int w = 1; w < kAcceptThreads / 32; ++w) take_better(bv, bi, sv[w], si[w]);
-      part[unit] = Cand{bv, bi};                 // unit = row * n_chunks + chunk
-    }
-    __syncthreads();                             // sv / si are reused by the next unit
-#pragma unroll
-    for (int u = 0; u < kAcceptVec; ++u) cur[u] = nxt[u];
-    cur_vec = nxt_vec;
+  if ((threadIdx.x & 31) == 0) {
+    sv[threadIdx.x >> 5] = bv;
+    si[threadIdx.x >> 5] = bi;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < kAcceptThreads / 32; ++w) take_better(bv, bi, sv[w], si[w]);
+    part[(size_t)row * n_chunks + chunk] = Cand{bv, bi};
   }
 }
 
@@ -206,16 +181,6 @@ static int32_t launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 block, c
   return launch_status();
 }
 
-// kernel 1 over all (row, chunk) units: at most three CTAs per SM, as many as its registers allow
-// to be resident (two units' loads, 64 KB, in flight each)
-static void launch_accept_partial(const float* logits, int vocab, int n_chunks, int n_rows, Cand* part,
-                                  cudaStream_t st) {
-  const int64_t n_units = (int64_t)n_rows * n_chunks;
-  const int64_t cap = (int64_t)sm_count() * 3;
-  accept_partial_kernel<<<(unsigned)(n_units < cap ? n_units : cap), kAcceptThreads, 0, st>>>(logits, vocab, n_chunks,
-                                                                                            (int)n_units, part);
-}
-
 // Built-in scratch of specvlm_accept_noalloc: room for kStaticCands (row, vocab chunk) candidates.
 // Every GPU that loads the library holds these 128 KB until the process exits.
 constexpr int kStaticCands = 16384;
@@ -239,15 +204,15 @@ extern "C" int32_t specvlm_accept(const float* target_logits, const int32_t* dra
     return SPECVLM_ERR_INVALID_ARG;
   if (gamma > 0 && !draft_tokens) return SPECVLM_ERR_INVALID_ARG;
   if (gamma > 15) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
-  if ((int64_t)batch * (gamma + 1) * (((int64_t)vocab + kAcceptChunk - 1) / kAcceptChunk) > 0x7fff0000)
-    return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  if ((int64_t)batch * (gamma + 1) > 65535) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   if ((reinterpret_cast<uintptr_t>(target_logits) & 3u) || (reinterpret_cast<uintptr_t>(ws) & 7u))
     return SPECVLM_ERR_INVALID_ARG;
   if (ws_bytes < specvlm_accept_workspace_bytes(batch, gamma, vocab)) return SPECVLM_ERR_WORKSPACE_TOO_SMALL;
   const int n_chunks = (vocab + kAcceptChunk - 1) / kAcceptChunk;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   Cand* part = static_cast<Cand*>(ws);
-  launch_accept_partial(target_logits, vocab, n_chunks, batch * (gamma + 1), part, st);
+  accept_partial_kernel<<<dim3((unsigned)n_chunks, (unsigned)(batch * (gamma + 1))), kAcceptThreads, 0, st>>>(
+      target_logits, vocab, n_chunks, part);
   int32_t rc = launch_status();
   if (rc != SPECVLM_OK) return rc;
   return launch_dependent(accept_finish_kernel, dim3((unsigned)batch), dim3(32u * (gamma + 1)), st,
@@ -262,8 +227,7 @@ extern "C" int32_t specvlm_accept_noalloc(const float* target_logits, const int3
     return SPECVLM_ERR_INVALID_ARG;
   if (gamma > 0 && !draft_tokens) return SPECVLM_ERR_INVALID_ARG;
   if (gamma > 15) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
-  if ((int64_t)batch * (gamma + 1) * (((int64_t)vocab + kAcceptChunk - 1) / kAcceptChunk) > 0x7fff0000)
-    return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  if ((int64_t)batch * (gamma + 1) > 65535) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   if (reinterpret_cast<uintptr_t>(target_logits) & 3u) return SPECVLM_ERR_INVALID_ARG;
   const int n_chunks = (vocab + kAcceptChunk - 1) / kAcceptChunk;
   if ((int64_t)batch * (gamma + 1) * n_chunks > kStaticCands) return SPECVLM_ERR_TOO_LARGE;
@@ -288,7 +252,8 @@ extern "C" int32_t specvlm_accept_noalloc(const float* target_logits, const int3
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // every candidate slot that kernel 2 reads is written by kernel 1 of the same call first, so
   // nothing left over from an earlier call has to be cleared
-  launch_accept_partial(target_logits, vocab, n_chunks, batch * (gamma + 1), part, st);
+  accept_partial_kernel<<<dim3((unsigned)n_chunks, (unsigned)(batch * (gamma + 1))), kAcceptThreads, 0, st>>>(
+      target_logits, vocab, n_chunks, part);
   int32_t rc = launch_status();
   if (rc != SPECVLM_OK) return rc;
   return launch_dependent(accept_finish_kernel, dim3((unsigned)batch), dim3(32u * (gamma + 1)), st,
@@ -303,15 +268,15 @@ extern "C" int32_t specvlm_accept_tree(const float* target_logits, const int32_t
   if (!target_logits || !node_tokens || !parents || !accept_len || !next_token || !path || !ws || batch < 1 ||
       n_nodes < 1 || vocab < 1)
     return SPECVLM_ERR_INVALID_ARG;
-  if (n_nodes > 32 || (int64_t)batch * n_nodes * (((int64_t)vocab + kAcceptChunk - 1) / kAcceptChunk) > 0x7fff0000)
-    return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  if (n_nodes > 32 || (int64_t)batch * n_nodes > 65535) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   if ((reinterpret_cast<uintptr_t>(target_logits) & 3u) || (reinterpret_cast<uintptr_t>(ws) & 7u))
     return SPECVLM_ERR_INVALID_ARG;
   if (ws_bytes < specvlm_accept_workspace_bytes(batch, n_nodes - 1, vocab)) return SPECVLM_ERR_WORKSPACE_TOO_SMALL;
   const int n_chunks = (vocab + kAcceptChunk - 1) / kAcceptChunk;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   Cand* part = static_cast<Cand*>(ws);
-  launch_accept_partial(target_logits, vocab, n_chunks, batch * n_nodes, part, st);
+  accept_partial_kernel<<<dim3((unsigned)n_chunks, (unsigned)(batch * n_nodes)), kAcceptThreads, 0, st>>>(
+      target_logits, vocab, n_chunks, part);
   int32_t rc = launch_status();
   if (rc != SPECVLM_OK) return rc;
   return launch_dependent(accept_tree_finish_kernel, dim3((unsigned)batch), dim3(32u * n_nodes), st,
