@@ -687,10 +687,44 @@ def cpu_baseline(w):
         b, t = oracle_sample(w, n_layers)
         nbytes += b
         dt += t
-    return {"value": round(nbytes / dt / 1e9, 4), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-            "seconds": round(dt, 2),
-            "sample": f"fp64 oracle attention, {reps} steps: each {w.gamma} draft decode steps over the pruned cache "
-                      f"(all {w.d_layers} draft layers) + verification over all {n_layers} verifier layers"}
+    out = {"value": round(nbytes / dt / 1e9, 4), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+           "seconds": round(dt, 2),
+           "sample": f"fp64 oracle attention, {reps} steps: each {w.gamma} draft decode steps over the pruned cache "
+                     f"(all {w.d_layers} draft layers) + verification over all {n_layers} verifier layers"}
+    out["prune"] = oracle_prune_sample(w, 2)
+    return out
+
+
+def oracle_prune_sample(w, n_layers):
+    """Times the oracle's prune stage once: token rating on n_layers verifier layers (every layer is
+    the same amount of work, so the whole rating is extrapolated by the layer count), selection,
+    and the K/V gather of all draft layers."""
+    import numpy as np
+    import oracle
+    rng = np.random.default_rng(1)
+    D, nv, nt = w.head_dim, w.n_video(), w.n_text[0]
+
+    def bf16(shape):
+        return (rng.standard_normal(shape).astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
+    q = bf16((n_layers, nt, w.t_q_heads, D))
+    k = bf16((n_layers, w.t_kv_heads, nv + nt, D))
+    t0 = time.perf_counter()
+    a = oracle.stage1_scores(q, k, 0, nv, nv, 1.0 / math.sqrt(D))
+    t_rate = time.perf_counter() - t0
+    a32 = a.astype(np.float32)
+    t0 = time.perf_counter()
+    kept = oracle.select(a32, w.n_frames[0], w.tokens_per_frame, w.k_stage1(), w.k_total())
+    t_sel = time.perf_counter() - t0
+    src = bf16((w.d_layers, w.d_kv_heads, nv + nt, D))
+    t0 = time.perf_counter()
+    for _ in range(2):                                       # K and V
+        oracle.gather_kv(src, np.asarray(kept), 0, nv, nv + nt)
+    t_gat = time.perf_counter() - t0
+    rate_all = t_rate * w.t_layers / n_layers
+    return {"rating_s_extrapolated": round(rate_all, 2), "rating_layers_timed": n_layers, "select_s": round(t_sel, 4),
+            "gather_s": round(t_gat, 4), "prune_s_extrapolated": round(rate_all + t_sel, 2),
+            "note": f"fp64 oracle: rating timed on {n_layers} of {w.t_layers} verifier layers and scaled by the layer "
+                    f"count (extrapolated), selection and the gather of all {w.d_layers} draft layers timed whole"}
 
 
 def run_reference(args, rank):
