@@ -200,6 +200,7 @@ extern "C" int32_t specvlm_accept(const float* target_logits, const int32_t* dra
                                   int32_t batch, int32_t gamma, int32_t vocab, int32_t* accept_len,
                                   int32_t* next_token, int32_t* target_argmax_or_null, void* ws,
                                   size_t ws_bytes, void* stream) {
+  NvtxRange nvtx_range(__func__);
   if (!target_logits || !accept_len || !next_token || batch < 1 || gamma < 0 || vocab < 1 || !ws)
     return SPECVLM_ERR_INVALID_ARG;
   if (gamma > 0 && !draft_tokens) return SPECVLM_ERR_INVALID_ARG;
@@ -223,6 +224,7 @@ extern "C" int32_t specvlm_accept(const float* target_logits, const int32_t* dra
 extern "C" int32_t specvlm_accept_noalloc(const float* target_logits, const int32_t* draft_tokens,
                                           int32_t batch, int32_t gamma, int32_t vocab, int32_t* accept_len,
                                           int32_t* next_token, int32_t* target_argmax_or_null, void* stream) {
+  NvtxRange nvtx_range(__func__);
   if (!target_logits || !accept_len || !next_token || batch < 1 || gamma < 0 || vocab < 1)
     return SPECVLM_ERR_INVALID_ARG;
   if (gamma > 0 && !draft_tokens) return SPECVLM_ERR_INVALID_ARG;
@@ -265,6 +267,7 @@ extern "C" int32_t specvlm_accept_tree(const float* target_logits, const int32_t
                                        const int32_t* parents, int32_t batch, int32_t n_nodes, int32_t vocab,
                                        int32_t* accept_len, int32_t* next_token, int32_t* path,
                                        int32_t* target_argmax_or_null, void* ws, size_t ws_bytes, void* stream) {
+  NvtxRange nvtx_range(__func__);
   if (!target_logits || !node_tokens || !parents || !accept_len || !next_token || !path || !ws || batch < 1 ||
       n_nodes < 1 || vocab < 1)
     return SPECVLM_ERR_INVALID_ARG;

@@ -585,6 +585,7 @@ extern "C" int32_t specvlm_draft_decode_attn(const specvlm_kv_t* kv, const void*
                                              int32_t n_q_heads, float sm_scale, void* out,
                                              float* lse_or_null, void* ws, size_t ws_bytes,
                                              int32_t* d_status, void* stream) {
+  NvtxRange nvtx_range(__func__);
   return attn_common(kv, q, batch, n_q_heads, 1, sm_scale, out, lse_or_null, ws, ws_bytes, d_status,
                      stream);
 }
@@ -593,6 +594,7 @@ extern "C" int32_t specvlm_verify_attn(const specvlm_kv_t* kv, const void* q, in
                                        int32_t n_q_heads, int32_t gamma, float sm_scale, void* out,
                                        float* lse_or_null, void* ws, size_t ws_bytes,
                                        int32_t* d_status, void* stream) {
+  NvtxRange nvtx_range(__func__);
   if (gamma < 0 || gamma > 8) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   return attn_common(kv, q, batch, n_q_heads, gamma + 1, sm_scale, out, lse_or_null, ws, ws_bytes,
                      d_status, stream);
@@ -612,6 +614,7 @@ extern "C" int32_t specvlm_verify_tree_attn(const specvlm_kv_t* kv, const void* 
                                             int32_t batch, int32_t n_q_heads, int32_t n_nodes, float sm_scale,
                                             void* out, float* lse_or_null, void* ws, size_t ws_bytes,
                                             int32_t* d_status, void* stream) {
+  NvtxRange nvtx_range(__func__);
   int32_t rc = validate_kv(kv, batch, true);
   if (rc != SPECVLM_OK) return rc;
   if (!q || !out || !parents || n_q_heads < 1 || n_nodes < 1 || !(sm_scale > 0.f)) return SPECVLM_ERR_INVALID_ARG;

@@ -163,6 +163,7 @@ using namespace specvlm;
 
 extern "C" int32_t specvlm_append_kv(const specvlm_kv_t* kv, const void* new_k, const void* new_v, int32_t batch,
                                      int32_t n_new, int32_t* seq_lens_inout, int32_t* d_status, void* stream) {
+  NvtxRange nvtx_range(__func__);
   if (!kv || !new_k || !new_v || !seq_lens_inout || n_new < 1) return SPECVLM_ERR_INVALID_ARG;
   specvlm_kv_t c = *kv;
   c.seq_lens = seq_lens_inout;
@@ -199,6 +200,7 @@ extern "C" int32_t specvlm_append_kv(const specvlm_kv_t* kv, const void* new_k, 
 
 extern "C" int32_t specvlm_rollback_kv(int32_t* seq_lens_inout, const int32_t* accept_len, int32_t batch,
                                        int32_t gamma, int32_t* d_status, void* stream) {
+  NvtxRange nvtx_range(__func__);
   if (!seq_lens_inout || !accept_len || batch < 1 || gamma < 0) return SPECVLM_ERR_INVALID_ARG;
   seq_len_update_kernel<<<(unsigned)((batch + 127) / 128), 128, 0, static_cast<cudaStream_t>(stream)>>>(
       seq_lens_inout, accept_len, batch, 0, gamma, 0, d_status);
@@ -208,6 +210,7 @@ extern "C" int32_t specvlm_rollback_kv(int32_t* seq_lens_inout, const int32_t* a
 extern "C" int32_t specvlm_compact_tree_kv(const specvlm_kv_t* kv, const int32_t* path, const int32_t* accept_len,
                                            int32_t batch, int32_t n_nodes, int32_t* seq_lens_inout,
                                            int32_t* d_status, void* stream) {
+  NvtxRange nvtx_range(__func__);
   if (!kv || !path || !accept_len || !seq_lens_inout || n_nodes < 1) return SPECVLM_ERR_INVALID_ARG;
   if (n_nodes > 32) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   specvlm_kv_t c = *kv;

@@ -88,6 +88,7 @@ extern "C" int32_t specvlm_gather_kv(const specvlm_kv_t* src, const int32_t* kep
                                      const int32_t* kept_cu, const int32_t* video_start,
                                      const int32_t* video_len, const int32_t* src_len, int32_t batch,
                                      const specvlm_kv_t* dst, int32_t* d_status, void* stream) {
+  NvtxRange nvtx_range(__func__);
   if (!src || !dst || !kept_idx || !kept_cu || !video_start || !video_len || !src_len || batch < 1)
     return SPECVLM_ERR_INVALID_ARG;
   // seq_lens are not read by this call; max_seq_len bounds the positions touched

@@ -733,6 +733,7 @@ extern "C" int32_t specvlm_stage1_row_lse(const specvlm_kv_t* target_kv, const v
                                           const int32_t* text_cu, const int32_t* text_start, int32_t batch,
                                           int32_t n_q_heads, float sm_scale, float* row_lse,
                                           int32_t* d_status, void* stream) {
+  NvtxRange nvtx_range(__func__);
   if (!row_lse) return SPECVLM_ERR_INVALID_ARG;
   ScoreSetup su;
   int32_t rc = setup_scores(target_kv, q_text, text_cu, text_start, nullptr, nullptr, nullptr, batch,
@@ -790,6 +791,7 @@ extern "C" int32_t specvlm_stage1_scores(const specvlm_kv_t* target_kv, const vo
                                          const int32_t* video_cu, int32_t batch, int32_t n_q_heads,
                                          float sm_scale, const float* row_lse_or_null, float* scores,
                                          void* ws, size_t ws_bytes, int32_t* d_status, void* stream) {
+  NvtxRange nvtx_range(__func__);
   if (!target_kv) return SPECVLM_ERR_INVALID_ARG;
   return stage1_scores_range(target_kv, q_text, text_cu, text_start, video_start, video_len, video_cu, batch,
                              n_q_heads, sm_scale, row_lse_or_null, scores, ws, ws_bytes, 0, target_kv->n_layers, true,
@@ -803,6 +805,7 @@ extern "C" int32_t specvlm_stage1_scores_layers(const specvlm_kv_t* target_kv, c
                                                 float sm_scale, const float* row_lse_or_null, float* scores,
                                                 void* ws, size_t ws_bytes, int32_t layer_begin, int32_t layer_end,
                                                 int32_t finish, int32_t* d_status, void* stream) {
+  NvtxRange nvtx_range(__func__);
   return stage1_scores_range(target_kv, q_text, text_cu, text_start, video_start, video_len, video_cu, batch,
                              n_q_heads, sm_scale, row_lse_or_null, scores, ws, ws_bytes, layer_begin, layer_end,
                              finish != 0, d_status, stream);

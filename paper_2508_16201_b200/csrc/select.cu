@@ -415,6 +415,7 @@ extern "C" int32_t specvlm_select(const float* scores, const int32_t* video_cu, 
                                   int32_t tokens_per_frame, const int32_t* k_stage1,
                                   const int32_t* k_total, const int32_t* kept_cu, int32_t batch,
                                   int32_t* kept_idx, int32_t* d_status, void* stream) {
+  NvtxRange nvtx_range(__func__);
   (void)d_status;
   if (!k_stage1) return SPECVLM_ERR_INVALID_ARG;
   return select_common(scores, video_cu, n_frames, tokens_per_frame, k_stage1, nullptr, k_total, kept_cu, batch,
@@ -426,6 +427,7 @@ extern "C" int32_t specvlm_select_top_p(const float* scores, const int32_t* vide
                                         const int32_t* k_total, const int32_t* kept_cu, int32_t batch,
                                         int32_t* kept_idx, int32_t* k_stage1_out_or_null, int32_t* d_status,
                                         void* stream) {
+  NvtxRange nvtx_range(__func__);
   (void)d_status;
   if (!lambda_permille) return SPECVLM_ERR_INVALID_ARG;
   return select_common(scores, video_cu, n_frames, tokens_per_frame, nullptr, lambda_permille, k_total, kept_cu,
@@ -436,6 +438,7 @@ extern "C" int32_t specvlm_select_baseline(int32_t mode, uint64_t seed, const in
                                            int32_t tokens_per_frame, const int32_t* k_total,
                                            const int32_t* kept_cu, int32_t batch, int32_t* kept_idx,
                                            int32_t* kept_n_out_or_null, void* stream) {
+  NvtxRange nvtx_range(__func__);
   if (!n_frames || !k_total || !kept_cu || !kept_idx || batch < 1 || tokens_per_frame < 1)
     return SPECVLM_ERR_INVALID_ARG;
   if (mode < SPECVLM_SEL_WINDOW_FRONT || mode > SPECVLM_SEL_RANDOM) return SPECVLM_ERR_INVALID_ARG;
