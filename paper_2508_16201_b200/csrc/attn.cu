@@ -457,7 +457,7 @@ static size_t rows16_ws_bytes(const specvlm_kv_t* kv, int32_t batch, int rows) {
 }
 
 // tcgen05 path (attn_tc.cu)
-size_t attn_tc_ws_bytes(const specvlm_kv_t* kv, int32_t batch, int rows);
+size_t attn_tc_ws_bytes(const specvlm_kv_t* kv, int32_t batch, int rows, int group);
 size_t attn_tc_tree_extra_bytes(int32_t batch, int32_t n_nodes);
 int32_t attn_tc_launch(const specvlm_kv_t* kv, const void* q, int32_t batch, int32_t n_q_heads, int32_t n_q,
                        float sm_scale, void* out, float* lse, void* ws, size_t ws_bytes, int32_t* d_status,
@@ -577,7 +577,7 @@ extern "C" size_t specvlm_attn_workspace_bytes(const specvlm_kv_t* kv, int32_t b
     return 0;
   const int rows = (n_q_heads / kv->n_kv_heads) * (gamma + 1);
   if (n_q_heads / kv->n_kv_heads > 16 || gamma > 8) return 0;
-  if (rows > kRows16Max) return batch <= kSchedMaxBatch ? attn_tc_ws_bytes(kv, batch, rows) : 0;
+  if (rows > kRows16Max) return batch <= kSchedMaxBatch ? attn_tc_ws_bytes(kv, batch, rows, n_q_heads / kv->n_kv_heads) : 0;
   return rows16_ws_bytes(kv, batch, rows);
 }
 
@@ -607,7 +607,7 @@ extern "C" size_t specvlm_verify_tree_workspace_bytes(const specvlm_kv_t* kv, in
     return 0;
   const int rows = (n_q_heads / kv->n_kv_heads) * n_nodes;
   if (n_q_heads / kv->n_kv_heads > 16) return 0;
-  return attn_tc_ws_bytes(kv, batch, rows) + attn_tc_tree_extra_bytes(batch, n_nodes);
+  return attn_tc_ws_bytes(kv, batch, rows, n_q_heads / kv->n_kv_heads) + attn_tc_tree_extra_bytes(batch, n_nodes);
 }
 
 extern "C" int32_t specvlm_verify_tree_attn(const specvlm_kv_t* kv, const void* q, const int32_t* parents,

@@ -44,8 +44,10 @@ struct AttnTcParams {
   const int32_t* seq_lens;    // [B]
   int32_t* d_status;
   const uint32_t* anc;        // [B][n_win] ancestor masks of a draft tree, or null: the window is a chain
-  int32_t batch, n_layers, n_q, n_q_heads, n_kv_heads, group, rows;
-  int32_t n_win, q0;          // tokens of the whole window; first window token of this launch (n_q of them)
+  int32_t batch, n_layers, n_q_heads, n_kv_heads, group;
+  int32_t n_win;              // tokens of the whole window
+  int32_t n_parts, q_per;     // the window is cut into n_parts parts of q_per tokens (the last may be shorter)
+  int32_t rows;               // rows of a full part = q_per * group (<= 128): the row pitch of the scratch slots
   int32_t max_blocks, block_tokens, max_seq_len;
   float scale_log2;           // sm_scale * log2(e)
 };
@@ -311,9 +313,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   const uint32_t tmem_base = *tmem_slot;
   const int hkv = p.n_kv_heads;
   const int64_t total = (int64_t)p.n_layers * hkv * prefix[p.batch];
-  const int n_active = sched_active_ctas(total, (int)gridDim.x);
-  const int cta = blockIdx.x;
-  const bool active = total > 0 && cta < n_active;
+  // A window of more than 128 rows is cut into parts of q_per query tokens, the accumulators of one
+  // part filling the tensor memory.  The parts run side by side in this one launch: the grid is
+  // n_parts sets of CTAs, every set slices the same flat tile list in the same way, so CTA c of each
+  // set streams the same K/V tiles at about the same time and all but the first to ask find them in
+  // the L2 cache -- HBM delivers every tile once, not once per part.
+  const int ctas_per_part = (int)gridDim.x / p.n_parts;
+  const int part = blockIdx.x / ctas_per_part;          // >= n_parts: a spare CTA without work
+  const int cta = blockIdx.x - part * ctas_per_part;    // index inside the part's set
+  const int gcta = blockIdx.x;                          // index of this CTA's scratch slots
+  const int q0 = part * p.q_per;                        // first window token of the part
+  const int n_q_part = part < p.n_parts ? (p.n_win - q0 < p.q_per ? p.n_win - q0 : p.q_per) : 0;
+  const int rows = n_q_part > 0 ? n_q_part * p.group : 0;   // rows in use (of the M rows of a tile)
+  const int n_active = sched_active_ctas(total, ctas_per_part);
+  const bool active = total > 0 && rows > 0 && cta < n_active;
   const int64_t T0 = active ? slice_begin(cta, n_active, total) : 0;
   const int64_t T1 = active ? slice_begin(cta + 1, n_active, total) : 0;
   const int n_items = p.n_layers * p.batch * hkv;
@@ -352,7 +365,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           mbar_arrive_expect_tx(bar_q_full + 8 * qb, (uint32_t)p.rows * 128u * (D / 64));
 #pragma unroll
           for (int h = 0; h < D / 64; ++h)
-            tma_load_5d(q_sm + qb * Q_BYTES + h * (M * 128), &tm_q, bar_q_full + 8 * qb, h * 64, 0, p.q0, sg.g,
+            tma_load_5d(q_sm + qb * Q_BYTES + h * (M * 128), &tm_q, bar_q_full + 8 * qb, h * 64, 0, q0, sg.g,
                         sg.layer * p.batch + sg.b, policy_q);
         }
         const int n_sub_seq = (clamp_len(p.seq_lens[sg.b], p.max_seq_len) + kTileTokens - 1) / kTileTokens;
@@ -503,17 +516,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     const int lr = lane >> 2, lc = (lane & 3) * 2;   // row inside a 16-lane half (and +8), first column of a pair
     // rows of this warp: half h covers item rows row0(h) + [0, 16), held in TMEM lanes 32 * quarter + 16 h + [0, 16)
     auto row0 = [&](int h) { return M == 64 ? 16 * quarter : 32 * quarter + 16 * h; };
-    const int nh = (p.rows > row0(0) ? 1 : 0) + (NH > 1 && p.rows > row0(1) ? 1 : 0);
+    const int nh = (rows > row0(0) ? 1 : 0) + (NH > 1 && rows > row0(1) ? 1 : 0);
 
     // sequences without any token: their outputs are zero, their LSE -inf
-    if (*any_empty) {
-      for (int item = cta; item < n_items; item += gridDim.x) {
+    if (*any_empty && rows > 0) {
+      for (int item = cta; item < n_items; item += ctas_per_part) {
         const int lb = item / hkv, g = item - lb * hkv, b = lb % p.batch;
         if (prefix[b + 1] != prefix[b]) continue;
-        for (int idx = st; idx < p.rows * (D / 8); idx += 256) {
+        for (int idx = st; idx < rows * (D / 8); idx += 256) {
           const int r = idx / (D / 8), c8 = idx - r * (D / 8);
           const int t = r / p.group, h = g * p.group + (r - t * p.group);
-          const size_t orow = ((size_t)lb * p.n_win + p.q0 + t) * p.n_q_heads + h;
+          const size_t orow = ((size_t)lb * p.n_win + q0 + t) * p.n_q_heads + h;
           *reinterpret_cast<uint4*>(p.out + orow * D + c8 * 8) = make_uint4(0, 0, 0, 0);
           if (p.lse && c8 == 0) p.lse[orow] = -INFINITY;
         }
@@ -549,12 +562,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         // probabilities leave as sixteen 16-byte stores into the swizzled P tile, and the TMEM load of
         // the next 16 columns is in flight while the current 16 are worked on.
         const int my_row = 32 * quarter + lane;
-        const bool warp_on = p.rows > 32 * quarter;         // warp-uniform: some row of this quadrant is in use
+        const bool warp_on = rows > 32 * quarter;         // warp-uniform: some row of this quadrant is in use
         uint32_t my_a;                                       // the row's window mask (tree) or key limit (chain)
         if constexpr (TREE) {
-          my_a = my_row < p.rows ? __ldg(p.anc + (size_t)sg.b * p.n_win + p.q0 + my_row / p.group) : 0u;
+          my_a = my_row < rows ? __ldg(p.anc + (size_t)sg.b * p.n_win + q0 + my_row / p.group) : 0u;
         } else {
-          my_a = my_row < p.rows ? (uint32_t)(win0 + p.q0 + my_row / p.group + 1) : 0u;
+          my_a = my_row < rows ? (uint32_t)(win0 + q0 + my_row / p.group + 1) : 0u;
         }
         float m_row = -INFINITY, l_row = 0.f;
         const uint32_t prow = p_sm + grp * P_BYTES + my_row * 128;
@@ -700,9 +713,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           const int r = row0(h) + lr + 8 * e;
           const int t = r / p.group;
           if constexpr (TREE) {
-            vis[h][e] = r < p.rows ? __ldg(p.anc + (size_t)sg.b * p.n_win + p.q0 + t) : 0u;
+            vis[h][e] = r < rows ? __ldg(p.anc + (size_t)sg.b * p.n_win + q0 + t) : 0u;
           } else {
-            lim[h][e] = r < p.rows ? win0 + p.q0 + t + 1 : 0;
+            lim[h][e] = r < rows ? win0 + q0 + t + 1 : 0;
           }
           m_used[h][e] = -INFINITY;
           l_sum[h][e] = 0.f;
@@ -852,7 +865,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       //   O = (w0 O0 + w1 O1) / (w0 l0 + w1 l1),  w_g = 2^(m_g - max(m0, m1))
       const bool complete = sg.tile0 == 0 && sg.n_tiles == sg.item_tiles;
       const int lb = sg.layer * p.batch + sg.b;
-      const int slot = partial_slot(cta, T0, sg.item_begin);
+      const int slot = partial_slot(gcta, T0, sg.item_begin);
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_ep_stats);
       SM_WAIT(bar_ep_stats, seg_idx & 1);
@@ -890,7 +903,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 #pragma unroll
           for (int e = 0; e < 2; ++e) {
             const int r = row0(h) + lr + 8 * e;
-            if (r >= p.rows) continue;
+            if (r >= rows) continue;
             float res[16];
 #pragma unroll
             for (int jj = 0; jj < 8; ++jj)
@@ -904,7 +917,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               }
             if (complete) {
               const int t = r / p.group, hq = sg.g * p.group + (r - t * p.group);
-              const size_t orow = ((size_t)lb * p.n_win + p.q0 + t) * p.n_q_heads + hq;
+              const size_t orow = ((size_t)lb * p.n_win + q0 + t) * p.n_q_heads + hq;
               __nv_bfloat16* dst = p.out + orow * D + cc * 64 + lc;
 #pragma unroll
               for (int jj = 0; jj < 8; ++jj)
@@ -934,7 +947,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         const int c_last = slice_owner(item_end - 1, n_active, total);
         if (st == 0) {
           if (mbar_wait(bar_ep_done, n_partial & 1, abort_flag)) {
-            const int old = atomicAdd(p.ws_cnt + sg.item, 1);
+            const int old = atomicAdd(p.ws_cnt + (size_t)part * n_items + sg.item, 1);
             __threadfence();
             *last_flag = (old == c_last - c_first) ? 1 : 0;
           } else {
@@ -951,7 +964,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           // instead of one per part and value.  Parts are folded in slice order (fixed).
           constexpr int kMergeChunk = 4;
           const int n_parts = c_last - c_first + 1;
-          const int n_idx = p.rows * (D / 4);
+          const int n_idx = rows * (D / 4);
           for (int idx0 = st; idx0 < n_idx; idx0 += 512) {
             int r[2], c4[2];
             bool on[2];
@@ -971,7 +984,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               for (int q = 0; q < kMergeChunk; ++q) {
                 const bool have = pc + q < n_parts;
                 const int cpart = c_first + pc + q;
-                const int sl = have ? partial_slot(cpart, slice_begin(cpart, n_active, total), sg.item_begin) : 0;
+                const int sl = have ? partial_slot(part * ctas_per_part + cpart, slice_begin(cpart, n_active, total), sg.item_begin) : 0;
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
                   if (have && on[u]) {
@@ -1012,7 +1025,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               if (!on[u]) continue;
               const float invd = den[u] > 0.f ? 1.f / den[u] : 0.f;
               const int t = r[u] / p.group, hq = sg.g * p.group + (r[u] - t * p.group);
-              const size_t orow = ((size_t)lb * p.n_win + p.q0 + t) * p.n_q_heads + hq;
+              const size_t orow = ((size_t)lb * p.n_win + q0 + t) * p.n_q_heads + hq;
               uint2 packed;
               packed.x = pack_bf16x2(acc[u].x * invd, acc[u].y * invd);
               packed.y = pack_bf16x2(acc[u].z * invd, acc[u].w * invd);
@@ -1042,17 +1055,40 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 // ---------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------
-static int tc_grid(const specvlm_kv_t* kv, int32_t batch) {
-  const int64_t tiles_max = (int64_t)kv->n_layers * batch * kv->n_kv_heads *
-                            ((kv->max_seq_len + kBigTokens - 1) / kBigTokens);
-  return sched_active_ctas(tiles_max, sm_count());
+// How a window of `rows` rows is cut: n_parts parts of q_per query tokens (at most 128 rows each).
+static void tc_parts(int rows, int group, int& n_parts, int& q_per) {
+  const int n_q = rows / group;
+  n_parts = (rows + 127) / 128;
+  q_per = (n_q + n_parts - 1) / n_parts;
 }
 
-size_t attn_tc_ws_bytes(const specvlm_kv_t* kv, int32_t batch, int rows) {
-  const int grid = tc_grid(kv, batch);
+// One set of CTAs per part, every set as large as the SMs allow (and the tile count is worth).
+static int tc_grid(const specvlm_kv_t* kv, int32_t batch, int n_parts) {
+  const int64_t tiles_max = (int64_t)kv->n_layers * batch * kv->n_kv_heads *
+                            ((kv->max_seq_len + kBigTokens - 1) / kBigTokens);
+  int per_part = sm_count() / n_parts;
+  if (per_part < 1) per_part = 1;
+  return n_parts * sched_active_ctas(tiles_max, per_part);
+}
+
+// scratch: two partial results per CTA (rows of a full part each), their LSEs, one arrival counter
+// per (part, item)
+static void tc_ws_layout(const specvlm_kv_t* kv, int32_t batch, int rows, int group, size_t& o_bytes, size_t& lse_bytes,
+                         size_t& cnt_bytes) {
+  int n_parts, q_per;
+  tc_parts(rows, group, n_parts, q_per);
+  const int grid = tc_grid(kv, batch, n_parts);
   const size_t items = (size_t)kv->n_layers * batch * kv->n_kv_heads;
-  return round_up((size_t)2 * grid * rows * kv->head_dim * sizeof(float), 256) +
-         round_up((size_t)2 * grid * rows * sizeof(float), 256) + round_up(items * sizeof(int32_t), 256);
+  const size_t rows_part = (size_t)q_per * group;
+  o_bytes = round_up((size_t)2 * grid * rows_part * kv->head_dim * sizeof(float), 256);
+  lse_bytes = round_up((size_t)2 * grid * rows_part * sizeof(float), 256);
+  cnt_bytes = round_up(items * n_parts * sizeof(int32_t), 256);
+}
+
+size_t attn_tc_ws_bytes(const specvlm_kv_t* kv, int32_t batch, int rows, int group) {
+  size_t a, b, c;
+  tc_ws_layout(kv, batch, rows, group, a, b, c);
+  return a + b + c;
 }
 
 // Queries as a 5-D tensor (channel, head in group, query token, KV head, layer * batch + sequence):
@@ -1136,16 +1172,18 @@ int32_t attn_tc_launch(const specvlm_kv_t* kv, const void* q, int32_t batch, int
   const int64_t items = (int64_t)kv->n_layers * batch * kv->n_kv_heads;
   if (items > 0x3fffffff) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) return SPECVLM_ERR_INVALID_ARG;
-  const size_t base_bytes = attn_tc_ws_bytes(kv, batch, rows);
+  size_t o_bytes, lse_bytes, cnt_bytes;
+  tc_ws_layout(kv, batch, rows, group, o_bytes, lse_bytes, cnt_bytes);
+  const size_t base_bytes = o_bytes + lse_bytes + cnt_bytes;
   if (ws_bytes < base_bytes + (tree_parents ? attn_tc_tree_extra_bytes(batch, n_q) : 0))
     return SPECVLM_ERR_WORKSPACE_TOO_SMALL;
   if (tree_parents && n_q > 32) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
-  const int grid = tc_grid(kv, batch);
-  // A window of more than 128 rows is cut into launches of equal numbers of query tokens, each of
-  // which streams the K/V once more: the accumulators of one launch fill the tensor memory.
-  const int n_launch = (rows + 127) / 128;
-  const int q_per = (n_q + n_launch - 1) / n_launch;
+  // A window of more than 128 rows is cut into parts of equal numbers of query tokens (the
+  // accumulators of one part fill the tensor memory); the parts share one launch (see the kernel).
+  int n_parts, q_per;
+  tc_parts(rows, group, n_parts, q_per);
   if (q_per * group > 128) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  const int grid = tc_grid(kv, batch, n_parts);
 
   CUtensorMap tk, tv;
   int32_t rc = encode_kv_map(&tk, kv, kv->k, kTileTokens);
@@ -1156,13 +1194,13 @@ int32_t attn_tc_launch(const specvlm_kv_t* kv, const void* q, int32_t batch, int
   AttnTcParams p;
   p.out = static_cast<__nv_bfloat16*>(out);
   p.lse = lse;
-  const int rows_max = q_per * group;
   uint8_t* w = static_cast<uint8_t*>(ws);
   p.ws_o = reinterpret_cast<float*>(w);
-  w += round_up((size_t)2 * grid * rows_max * kv->head_dim * sizeof(float), 256);
-  p.ws_lse = reinterpret_cast<float*>(w);
-  w += round_up((size_t)2 * grid * rows_max * sizeof(float), 256);
-  p.ws_cnt = reinterpret_cast<int32_t*>(w);
+  p.ws_lse = reinterpret_cast<float*>(w + o_bytes);
+  p.ws_cnt = reinterpret_cast<int32_t*>(w + o_bytes + lse_bytes);
+  p.n_parts = n_parts;
+  p.q_per = q_per;
+  p.rows = q_per * group;
   p.block_table = kv->block_table;
   p.seq_lens = kv->seq_lens;
   p.d_status = d_status;
@@ -1186,21 +1224,15 @@ int32_t attn_tc_launch(const specvlm_kv_t* kv, const void* q, int32_t batch, int
     p.anc = anc;
   }
 
-  for (int q0 = 0; q0 < n_q; q0 += q_per) {
-    p.q0 = q0;
-    p.n_q = n_q - q0 < q_per ? n_q - q0 : q_per;
-    p.rows = p.n_q * group;
-    CUtensorMap tq;
-    rc = encode_q_map(&tq, q, kv->head_dim, group, n_q, p.n_q, kv->n_kv_heads, (int64_t)kv->n_layers * batch);
-    if (rc != SPECVLM_OK) return rc;
-    // the launches share the scratch memory: stream order keeps them apart
-    if (cudaMemsetAsync(p.ws_cnt, 0, (size_t)items * sizeof(int32_t), st) != cudaSuccess) return SPECVLM_ERR_CUDA;
-    if (kv->head_dim == 128)
-      rc = p.rows <= 64 ? launch_tc<128, 64>(tk, tv, tq, p, grid, st) : launch_tc<128, 128>(tk, tv, tq, p, grid, st);
-    else
-      rc = p.rows <= 64 ? launch_tc<64, 64>(tk, tv, tq, p, grid, st) : launch_tc<64, 128>(tk, tv, tq, p, grid, st);
-    if (rc != SPECVLM_OK) return rc;
-  }
+  CUtensorMap tq;
+  rc = encode_q_map(&tq, q, kv->head_dim, group, n_q, q_per, kv->n_kv_heads, (int64_t)kv->n_layers * batch);
+  if (rc != SPECVLM_OK) return rc;
+  if (cudaMemsetAsync(p.ws_cnt, 0, (size_t)items * n_parts * sizeof(int32_t), st) != cudaSuccess) return SPECVLM_ERR_CUDA;
+  if (kv->head_dim == 128)
+    rc = p.rows <= 64 ? launch_tc<128, 64>(tk, tv, tq, p, grid, st) : launch_tc<128, 128>(tk, tv, tq, p, grid, st);
+  else
+    rc = p.rows <= 64 ? launch_tc<64, 64>(tk, tv, tq, p, grid, st) : launch_tc<64, 128>(tk, tv, tq, p, grid, st);
+  if (rc != SPECVLM_OK) return rc;
   return SPECVLM_OK;
 }
 
