@@ -446,7 +446,7 @@ def run_ours(args, rank, world):
         kept_idx=kept_tp, want_counts=False))
     # tree drafting: the widest tree one 128-row launch holds (16 nodes at 8 query heads per KV head),
     # and a 26-node static tree (root + 25 candidates, the size of the static draft tree the paper
-    # adopts; its shape here is a binary heap, the paper's figure being unavailable): 208 rows, two launches
+    # adopts; its shape here is a binary heap, the paper's figure being unavailable): 208 rows, two parts of 13 nodes in one launch
     for n_nodes in (128 // (w.t_q_heads // w.t_kv_heads), 26):
         n_tree = nv + nt + n_nodes
         tk = synth.randn_bf16((w.t_layers, 1, w.t_kv_heads, n_tree, D), device, 1, "treeK")

@@ -251,7 +251,8 @@ int32_t specvlm_gather_kv(const specvlm_kv_t* src, const int32_t* kept_idx, cons
  * touches no global memory until that kernel's writes are complete and visible.
  * Supported: head_dim 64/128; group = n_q_heads/n_kv_heads in 1..16; 0 <= gamma <= 8;
  * batch <= 127 when group * (gamma+1) > 16.  A window of more than 128 rows (group * (gamma+1))
- * runs as several launches of at most 128 rows, each reading the cache once.
+ * is cut into parts of at most 128 rows that run side by side in one launch, so that the cache
+ * still comes from HBM once (the later readers of a tile find it in the L2 cache).
  */
 size_t specvlm_attn_workspace_bytes(const specvlm_kv_t* kv, int32_t batch, int32_t n_q_heads,
                                     int32_t gamma);
@@ -320,8 +321,8 @@ int32_t specvlm_rollback_kv(int32_t* seq_lens_inout, const int32_t* accept_len, 
  *   q, out    device bf16 [n_layers][batch][n_nodes][n_q_heads][head_dim]
  *   ws        device scratch, specvlm_verify_tree_workspace_bytes(kv, batch, n_q_heads, n_nodes)
  * Supported: n_nodes <= 32, n_q_heads / n_kv_heads in 1..16, batch <= 127.  A tree of more than 128
- * rows ((n_q_heads / n_kv_heads) * n_nodes) runs as several launches of at most 128 rows, each
- * reading the cache once.  A parents array that is not in topological order stores
+ * rows ((n_q_heads / n_kv_heads) * n_nodes) is cut into parts of at most 128 rows that run side by
+ * side in one launch (see specvlm_verify_attn).  A parents array that is not in topological order stores
  * SPECVLM_ERR_INVALID_ARG to d_status.
  *
  * specvlm_accept_tree: greedy acceptance along the tree.  With g[t] = argmax of node t's target

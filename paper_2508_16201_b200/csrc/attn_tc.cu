@@ -1,6 +1,6 @@
 // Streaming softmax attention over a bf16 K/V cache on the 5th-generation tensor cores of sm_100a:
 // (gamma+1)-query verification attention and tree verification, i.e. windows of 17 to 128 rows per
-// KV head and launch (wider windows run as several launches; up to 16 rows run on the kernel of
+// KV head and set of CTAs (a wider window is cut into parts that share one launch; up to 16 rows run on the kernel of
 // attn.cu).
 //
 // One persistent CTA per SM streams a contiguous slice of the flat (layer, sequence, KV head, tile)

@@ -137,7 +137,7 @@ def test_verify_row_counts(Hq, Hkv, gamma, D, paged):
 
 @pytest.mark.parametrize("paged", [False, True])
 def test_verify_window_wider_than_one_launch(paged):
-    # group 16 with gamma 8: 144 rows, cut into two launches of 5 and 4 query tokens
+    # group 16 with gamma 8: 144 rows, cut into two parts of 5 and 4 query tokens
     _run_attn(2, 32, 2, 128, [300, 64 + 9, 9], 8, paged=paged, seed=11, poison=True)
     _run_attn(1, 16, 1, 64, [200], 8, paged=paged, seed=12)
 

@@ -51,8 +51,8 @@ def _tree_case(L, Hq, Hkv, D, lens, n_nodes, *, paged, seed, chain=False):
                                               (28, 4, 9, 128),    # 63 rows, group 7
                                               (8, 2, 32, 64),     # 32 nodes, d = 64
                                               (4, 4, 3, 64),      # 3 rows: below the decode kernel's limit
-                                              (64, 8, 26, 128),   # 208 rows: two launches of 13 nodes
-                                              (32, 2, 32, 128),   # 512 rows, group 16: four launches of 8 nodes
+                                              (64, 8, 26, 128),   # 208 rows: two parts of 13 nodes
+                                              (32, 2, 32, 128),   # 512 rows, group 16: four parts of 8 nodes
                                               (24, 4, 30, 64)])   # 180 rows, group 6, d = 64: 15 + 15 nodes
 def test_tree_attention(Hq, Hkv, n_nodes, D, paged):
     _tree_case(2, Hq, Hkv, D, [300 + n_nodes, 128 + 3, n_nodes, 64 + n_nodes // 2], n_nodes, paged=paged, seed=60)
