@@ -320,7 +320,7 @@ int32_t specvlm_rollback_kv(int32_t* seq_lens_inout, const int32_t* accept_len, 
  *   parents   device int32 [batch][n_nodes]
  *   q, out    device bf16 [n_layers][batch][n_nodes][n_q_heads][head_dim]
  *   ws        device scratch, specvlm_verify_tree_workspace_bytes(kv, batch, n_q_heads, n_nodes)
- * Supported: n_nodes <= 32, n_q_heads / n_kv_heads in 1..16, batch <= 127.  A tree of more than 128
+ * Supported: n_nodes <= 64, n_q_heads / n_kv_heads in 1..16, batch <= 127.  A tree of more than 128
  * rows ((n_q_heads / n_kv_heads) * n_nodes) is cut into parts of at most 128 rows that run side by
  * side in one launch (see specvlm_verify_attn).  A parents array that is not in topological order stores
  * SPECVLM_ERR_INVALID_ARG to d_status.

@@ -120,25 +120,28 @@ __global__ void accept_tree_finish_kernel(const Cand* part, int n_chunks,
                                           const int32_t* __restrict__ parents, int n_nodes,
                                           int32_t* __restrict__ accept_len, int32_t* __restrict__ next_token,
                                           int32_t* __restrict__ path, int32_t* __restrict__ g_out) {
-  __shared__ int g_sm[32];
-  const int b = blockIdx.x, t = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const Cand* row = part + ((size_t)b * n_nodes + t) * n_chunks;
+  __shared__ int g_sm[64];
+  const int b = blockIdx.x, lane = threadIdx.x & 31;
   asm volatile("griddepcontrol.wait;" ::: "memory");         // kernel 1 has completed, its candidates are visible
-  float bv = -INFINITY;
-  int bi = 0x7fffffff;
-  for (int c = lane; c < n_chunks; c += 32) {
-    const int2 raw = __ldcg(reinterpret_cast<const int2*>(row + c));
-    take_better(bv, bi, __int_as_float(raw.x), raw.y);
-  }
+  // a warp per node; with more than 32 nodes the warps take a second one each
+  for (int t = threadIdx.x >> 5; t < n_nodes; t += blockDim.x >> 5) {
+    const Cand* row = part + ((size_t)b * n_nodes + t) * n_chunks;
+    float bv = -INFINITY;
+    int bi = 0x7fffffff;
+    for (int c = lane; c < n_chunks; c += 32) {
+      const int2 raw = __ldcg(reinterpret_cast<const int2*>(row + c));
+      take_better(bv, bi, __int_as_float(raw.x), raw.y);
+    }
 #pragma unroll
-  for (int off = 16; off > 0; off >>= 1) {
-    const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
-    const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
-    take_better(bv, bi, ov, oi);
-  }
-  if (lane == 0) {
-    g_sm[t] = bi;
-    if (g_out) g_out[(size_t)b * n_nodes + t] = bi;
+    for (int off = 16; off > 0; off >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+      take_better(bv, bi, ov, oi);
+    }
+    if (lane == 0) {
+      g_sm[t] = bi;
+      if (g_out) g_out[(size_t)b * n_nodes + t] = bi;
+    }
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -271,7 +274,7 @@ extern "C" int32_t specvlm_accept_tree(const float* target_logits, const int32_t
   if (!target_logits || !node_tokens || !parents || !accept_len || !next_token || !path || !ws || batch < 1 ||
       n_nodes < 1 || vocab < 1)
     return SPECVLM_ERR_INVALID_ARG;
-  if (n_nodes > 32 || (int64_t)batch * n_nodes > 65535) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  if (n_nodes > 64 || (int64_t)batch * n_nodes > 65535) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   if ((reinterpret_cast<uintptr_t>(target_logits) & 3u) || (reinterpret_cast<uintptr_t>(ws) & 7u))
     return SPECVLM_ERR_INVALID_ARG;
   if (ws_bytes < specvlm_accept_workspace_bytes(batch, n_nodes - 1, vocab)) return SPECVLM_ERR_WORKSPACE_TOO_SMALL;
@@ -282,7 +285,7 @@ extern "C" int32_t specvlm_accept_tree(const float* target_logits, const int32_t
       target_logits, vocab, n_chunks, part);
   int32_t rc = launch_status();
   if (rc != SPECVLM_OK) return rc;
-  return launch_dependent(accept_tree_finish_kernel, dim3((unsigned)batch), dim3(32u * n_nodes), st,
+  return launch_dependent(accept_tree_finish_kernel, dim3((unsigned)batch), dim3(32u * (n_nodes < 32 ? n_nodes : 32)), st,
                           static_cast<const Cand*>(part), n_chunks, node_tokens, parents, n_nodes, accept_len,
                           next_token, path, target_argmax_or_null);
 }

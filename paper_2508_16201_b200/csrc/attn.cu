@@ -602,7 +602,7 @@ extern "C" int32_t specvlm_verify_attn(const specvlm_kv_t* kv, const void* q, in
 
 extern "C" size_t specvlm_verify_tree_workspace_bytes(const specvlm_kv_t* kv, int32_t batch, int32_t n_q_heads,
                                                       int32_t n_nodes) {
-  if (!kv || batch < 1 || batch > kSchedMaxBatch || n_q_heads < 1 || n_nodes < 1 || n_nodes > 32 ||
+  if (!kv || batch < 1 || batch > kSchedMaxBatch || n_q_heads < 1 || n_nodes < 1 || n_nodes > 64 ||
       kv->n_kv_heads < 1 || n_q_heads % kv->n_kv_heads != 0 || kv->n_layers < 1 || kv->max_seq_len < 1)
     return 0;
   const int rows = (n_q_heads / kv->n_kv_heads) * n_nodes;
@@ -620,7 +620,7 @@ extern "C" int32_t specvlm_verify_tree_attn(const specvlm_kv_t* kv, const void* 
   if (!q || !out || !parents || n_q_heads < 1 || n_nodes < 1 || !(sm_scale > 0.f)) return SPECVLM_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(out) || n_q_heads % kv->n_kv_heads != 0) return SPECVLM_ERR_INVALID_ARG;
   const int group = n_q_heads / kv->n_kv_heads;
-  if (group > 16 || n_nodes > 32) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  if (group > 16 || n_nodes > 64) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   return attn_tc_launch(kv, q, batch, n_q_heads, n_nodes, sm_scale, out, lse_or_null, ws, ws_bytes, d_status,
                         static_cast<cudaStream_t>(stream), parents);
 }

@@ -43,7 +43,7 @@ struct AttnTcParams {
   const int32_t* block_table; // [B][max_blocks] or null
   const int32_t* seq_lens;    // [B]
   int32_t* d_status;
-  const uint32_t* anc;        // [B][n_win] ancestor masks of a draft tree, or null: the window is a chain
+  const uint64_t* anc;        // [B][n_win] ancestor masks of a draft tree (<= 64 nodes), or null: the window is a chain
   int32_t batch, n_layers, n_q_heads, n_kv_heads, group;
   int32_t n_win;              // tokens of the whole window
   int32_t n_parts, q_per;     // the window is cut into n_parts parts of q_per tokens (the last may be shorter)
@@ -53,6 +53,7 @@ struct AttnTcParams {
 };
 
 constexpr float kRescaleThreshold = 8.f;   // log2 units
+constexpr int kMaxTreeNodes = 64;          // a window mask is one 64-bit word per node
 constexpr int kBigTokens = 2 * kTileTokens;          // tokens per MMA tile
 constexpr int kTcThreads = 384;
 // setmaxnreg moves registers between the warps of a CTA inside the pool the CTA got at launch
@@ -122,8 +123,8 @@ __device__ __forceinline__ int clamp_len(int n, int max_len) { return n < 0 ? 0 
 // (a0, a1 = the rows' masks), positions up to t for a chain (a0, a1 = the rows' limits `lim`:
 // key tok is visible when tok < lim).
 template <bool TREE>
-__device__ __noinline__ void mask_s_half(uint32_t saddr, int tile_tok0, int win0, int lc, uint32_t a0, uint32_t a1) {
-  const uint32_t a[2] = {a0, a1};
+__device__ __noinline__ void mask_s_half(uint32_t saddr, int tile_tok0, int win0, int lc, uint64_t a0, uint64_t a1) {
+  const uint64_t a[2] = {a0, a1};
 #pragma unroll 1
   for (int c = 0; c < 2; ++c) {
     uint64_t mk[2];
@@ -138,7 +139,7 @@ __device__ __noinline__ void mask_s_half(uint32_t saddr, int tile_tok0, int win0
           if (sh > 0) full = sh >= 128 ? ~(unsigned __int128)0 : (((unsigned __int128)1 << sh) - 1);
           const unsigned __int128 w = a[e];
           full |= sh >= 0 ? (sh < 128 ? w << sh : (unsigned __int128)0)
-                          : (sh > -32 ? w >> (-sh) : (unsigned __int128)0);
+                          : (sh > -64 ? w >> (-sh) : (unsigned __int128)0);
         }
         mk[e] = (uint64_t)(full >> (64 * c)) >> lc;
       } else {
@@ -563,11 +564,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         // the next 16 columns is in flight while the current 16 are worked on.
         const int my_row = 32 * quarter + lane;
         const bool warp_on = rows > 32 * quarter;         // warp-uniform: some row of this quadrant is in use
-        uint32_t my_a;                                       // the row's window mask (tree) or key limit (chain)
+        uint64_t my_a;                                       // the row's window mask (tree) or key limit (chain)
         if constexpr (TREE) {
-          my_a = my_row < rows ? __ldg(p.anc + (size_t)sg.b * p.n_win + q0 + my_row / p.group) : 0u;
+          my_a = my_row < rows ? __ldg(p.anc + (size_t)sg.b * p.n_win + q0 + my_row / p.group) : 0ull;
         } else {
-          my_a = my_row < rows ? (uint32_t)(win0 + q0 + my_row / p.group + 1) : 0u;
+          my_a = my_row < rows ? (uint64_t)(win0 + q0 + my_row / p.group + 1) : 0ull;
         }
         float m_row = -INFINITY, l_row = 0.f;
         const uint32_t prow = p_sm + grp * P_BYTES + my_row * 128;
@@ -593,8 +594,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             // the out-of-line mask routine works on 16-lane halves with two rows per thread
 #pragma unroll 1
             for (int h = 0; h < nh; ++h) {
-              const uint32_t a0 = __shfl_sync(0xffffffffu, my_a, 16 * h + lr);
-              const uint32_t a1 = __shfl_sync(0xffffffffu, my_a, 16 * h + lr + 8);
+              const uint64_t a0 = __shfl_sync(0xffffffffu, my_a, 16 * h + lr);
+              const uint64_t a1 = __shfl_sync(0xffffffffu, my_a, 16 * h + lr + 8);
               mask_s_half<TREE>(saddr + ((uint32_t)(16 * h) << 16), tile_tok0, win0, lc, a0, a1);
             }
           }
@@ -703,7 +704,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         if (seg_idx >= 1) SM_WAIT(bar_o_empty, (seg_idx - 1) & 1);
         if (warp_on) seg_stats[grp * M + my_row] = make_float2(m_row, l_row);
       } else {
-      uint32_t vis[NH][2];
+      uint64_t vis[NH][2];
       int lim[NH][2];
       float m_used[NH][2], l_sum[NH][2];
 #pragma unroll
@@ -713,7 +714,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           const int r = row0(h) + lr + 8 * e;
           const int t = r / p.group;
           if constexpr (TREE) {
-            vis[h][e] = r < rows ? __ldg(p.anc + (size_t)sg.b * p.n_win + q0 + t) : 0u;
+            vis[h][e] = r < rows ? __ldg(p.anc + (size_t)sg.b * p.n_win + q0 + t) : 0ull;
           } else {
             lim[h][e] = r < rows ? win0 + q0 + t + 1 : 0;
           }
@@ -742,7 +743,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           const uint32_t saddr = tmem_base + ((uint32_t)(32 * quarter + 16 * h) << 16) + C::COL_S + grp * kBigTokens;
           if (__builtin_expect(need_mask, 0)) {
             if constexpr (TREE) mask_s_half<true>(saddr, tile_tok0, win0, lc, vis[0][0], vis[0][1]);
-            else mask_s_half<false>(saddr, tile_tok0, win0, lc, (uint32_t)lim[0][0], (uint32_t)lim[0][1]);
+            else mask_s_half<false>(saddr, tile_tok0, win0, lc, (uint64_t)lim[0][0], (uint64_t)lim[0][1]);
           }
           float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll 1
@@ -826,7 +827,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
               l_sum[0][e] = l_sum[NH - 1][e];
               l_sum[NH - 1][e] = tl;
               if constexpr (TREE) {
-                const uint32_t tv = vis[0][e];
+                const uint64_t tv = vis[0][e];
                 vis[0][e] = vis[NH - 1][e];
                 vis[NH - 1][e] = tv;
               } else {
@@ -1132,29 +1133,29 @@ static int32_t launch_tc_t(const CUtensorMap& tk, const CUtensorMap& tv, const C
 // Ancestor masks of a draft tree: bit w of anc[b][t] says that node t attends window position w
 // (itself and the nodes on its path to a root).  parents[b][t] < t, -1 for a root.
 __global__ void tree_ancestors_kernel(const int32_t* __restrict__ parents, int n, int n_nodes,
-                                      uint32_t* __restrict__ anc, int32_t* d_status) {
+                                      uint64_t* __restrict__ anc, int32_t* d_status) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   const int t = i % n_nodes;
   const int32_t* par = parents + (i - t);
-  uint32_t a = 1u << t;
+  uint64_t a = 1ull << t;
   int cur = t;
   for (int step = 0; step < n_nodes; ++step) {
     const int pp = par[cur];
     if (pp < 0) break;
     if (pp >= cur) {                      // not a tree in topological order: the node sees itself only
       if (d_status) *d_status = SPECVLM_ERR_INVALID_ARG;
-      a = 1u << t;
+      a = 1ull << t;
       break;
     }
-    a |= 1u << pp;
+    a |= 1ull << pp;
     cur = pp;
   }
   anc[i] = a;
 }
 
 size_t attn_tc_tree_extra_bytes(int32_t batch, int32_t n_nodes) {
-  return round_up((size_t)batch * n_nodes * sizeof(uint32_t), 256);
+  return round_up((size_t)batch * n_nodes * sizeof(uint64_t), 256);
 }
 
 template <int D, int M>
@@ -1177,7 +1178,7 @@ int32_t attn_tc_launch(const specvlm_kv_t* kv, const void* q, int32_t batch, int
   const size_t base_bytes = o_bytes + lse_bytes + cnt_bytes;
   if (ws_bytes < base_bytes + (tree_parents ? attn_tc_tree_extra_bytes(batch, n_q) : 0))
     return SPECVLM_ERR_WORKSPACE_TOO_SMALL;
-  if (tree_parents && n_q > 32) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  if (tree_parents && n_q > kMaxTreeNodes) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   // A window of more than 128 rows is cut into parts of equal numbers of query tokens (the
   // accumulators of one part fill the tensor memory); the parts share one launch (see the kernel).
   int n_parts, q_per;
@@ -1216,7 +1217,7 @@ int32_t attn_tc_launch(const specvlm_kv_t* kv, const void* q, int32_t batch, int
   p.scale_log2 = sm_scale * kLog2e;
   p.anc = nullptr;
   if (tree_parents) {
-    uint32_t* anc = reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(ws) + base_bytes);
+    uint64_t* anc = reinterpret_cast<uint64_t*>(static_cast<uint8_t*>(ws) + base_bytes);
     const int n = batch * n_q;
     tree_ancestors_kernel<<<(unsigned)((n + 127) / 128), 128, 0, st>>>(tree_parents, n, n_q, anc, d_status);
     rc = launch_status();

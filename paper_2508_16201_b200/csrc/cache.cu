@@ -106,9 +106,9 @@ __global__ void __launch_bounds__(256) compact_tree_kernel(const __grid_constant
     }
     return layer * p.s_layer + blk * p.s_block + head * p.s_head + off * p.s_token + chunk;
   };
-  constexpr int kMaxPerThread = 2;          // 31 rows x 16 chunks = 496 chunks <= 2 x 256
+  constexpr int kMaxPerThread = 4;          // 63 rows x 16 chunks = 1008 chunks <= 4 x 256
   uint4 kk[kMaxPerThread], vv[kMaxPerThread];
-  bool have[kMaxPerThread] = {false, false};
+  bool have[kMaxPerThread] = {false, false, false, false};
   if (old < 0 || len > p.max_seq_len) {     // tree_len_kernel reports the short sequence; a long one here
     if (len > p.max_seq_len && p.d_status && threadIdx.x == 0) *p.d_status = SPECVLM_ERR_INVALID_ARG;
     return;
@@ -212,7 +212,7 @@ extern "C" int32_t specvlm_compact_tree_kv(const specvlm_kv_t* kv, const int32_t
                                            int32_t* d_status, void* stream) {
   NvtxRange nvtx_range(__func__);
   if (!kv || !path || !accept_len || !seq_lens_inout || n_nodes < 1) return SPECVLM_ERR_INVALID_ARG;
-  if (n_nodes > 32) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
+  if (n_nodes > 64) return SPECVLM_ERR_UNSUPPORTED_SHAPE;
   specvlm_kv_t c = *kv;
   c.seq_lens = seq_lens_inout;
   int32_t rc = validate_kv(&c, batch, true);

@@ -65,7 +65,7 @@ def test_fuzz_tree_attention(seed):
     rng = np.random.default_rng(3000 + seed)
     Hq, Hkv = GROUPS[int(rng.integers(0, len(GROUPS)))]
     D = 64 if rng.random() < 0.3 else 128
-    n_nodes = int(rng.integers(1, 33))
+    n_nodes = int(rng.integers(1, 65)) if rng.random() < 0.3 else int(rng.integers(1, 33))
     L = int(rng.integers(1, 3))
     batch = int(rng.integers(1, 5))
     lens = _lens(rng, batch, 1, 500, n_nodes)

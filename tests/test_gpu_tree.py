@@ -53,7 +53,10 @@ def _tree_case(L, Hq, Hkv, D, lens, n_nodes, *, paged, seed, chain=False):
                                               (4, 4, 3, 64),      # 3 rows: below the decode kernel's limit
                                               (64, 8, 26, 128),   # 208 rows: two parts of 13 nodes
                                               (32, 2, 32, 128),   # 512 rows, group 16: four parts of 8 nodes
-                                              (24, 4, 30, 64)])   # 180 rows, group 6, d = 64: 15 + 15 nodes
+                                              (24, 4, 30, 64),    # 180 rows, group 6, d = 64: 15 + 15 nodes
+                                              (64, 8, 60, 128),   # 60 nodes (a dynamic draft tree's size): 480 rows, four parts of 15
+                                              (28, 4, 64, 128),   # 64 nodes, the mask's width, group 7: 448 rows, four parts of 16
+                                              (8, 8, 41, 64)])    # 41 rows of one head each: bits above 32 in a single 64-row part
 def test_tree_attention(Hq, Hkv, n_nodes, D, paged):
     _tree_case(2, Hq, Hkv, D, [300 + n_nodes, 128 + 3, n_nodes, 64 + n_nodes // 2], n_nodes, paged=paged, seed=60)
 
@@ -75,7 +78,7 @@ def test_tree_bad_parents_are_reported():
     assert int(status.item()) == specvlm.ERR_INVALID_ARG
 
 
-@pytest.mark.parametrize("batch,n_nodes,vocab", [(1, 26, 152064), (5, 9, 4099), (16, 32, 1000)])
+@pytest.mark.parametrize("batch,n_nodes,vocab", [(1, 26, 152064), (5, 9, 4099), (16, 32, 1000), (3, 64, 4099), (2, 47, 152064)])
 def test_tree_accept_bit_exact(batch, n_nodes, vocab):
     rng = np.random.default_rng(63)
     logits = torch.randn((batch, n_nodes, vocab), generator=torch.Generator().manual_seed(63)).cuda()
@@ -103,9 +106,10 @@ def test_tree_accept_bit_exact(batch, n_nodes, vocab):
         assert len(lens) > 1          # the cases really differ
 
 
+@pytest.mark.parametrize("n_nodes", [12, 60])
 @pytest.mark.parametrize("paged", [False, True])
-def test_tree_step_chain_verify_accept_compact(paged):
-    L, Hq, Hkv, D, n_nodes, vocab = 2, 16, 2, 128, 12, 997
+def test_tree_step_chain_verify_accept_compact(paged, n_nodes):
+    L, Hq, Hkv, D, vocab = 2, 16, 2, 128, 997
     rng = np.random.default_rng(64)
     lens = [150 + n_nodes, 64 + n_nodes, n_nodes]
     cache, k_host, v_host = make_cache(L, Hkv, D, lens, paged=paged, seed=64)

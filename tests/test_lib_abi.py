@@ -78,7 +78,7 @@ def test_host_validation_without_gpu():
     assert L.specvlm_stage1_scores_layers(*common, 3, 5, 0, None, None) == specvlm.ERR_INVALID_ARG
     assert L.specvlm_stage1_scores_layers(*common, 2, 1, 0, None, None) == specvlm.ERR_INVALID_ARG
     # tree verification: more nodes than the ancestor masks hold
-    rc = L.specvlm_verify_tree_attn(ctypes.byref(kv), 0x1000, 0x1000, 1, 4, 33, 0.1, 0x1000, None, 0x1000, 1 << 30,
+    rc = L.specvlm_verify_tree_attn(ctypes.byref(kv), 0x1000, 0x1000, 1, 4, 65, 0.1, 0x1000, None, 0x1000, 1 << 30,
                                     None, None)
     assert rc == specvlm.ERR_UNSUPPORTED_SHAPE
 
