@@ -62,8 +62,11 @@ NCU_TRAFFIC_BYTES = {"verify": 216.0e6 * 10, "decode": 43.5e6, "scores_colsum": 
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs.  Every sample carries
+    nvidia-smi's own timestamp; `stop(t0, t1)` keeps the samples taken between the two host wall-clock
+    times that bracket the timed region (all samples if none fell inside: a region of a few tens of
+    milliseconds can slip between two samples)."""
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
@@ -73,7 +76,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -84,7 +87,15 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append([x.strip() for x in line.split(",")])
 
-    def stop(self):
+    @staticmethod
+    def _when(stamp):
+        import datetime
+        try:
+            return datetime.datetime.strptime(stamp, "%Y/%m/%d %H:%M:%S.%f").timestamp()
+        except ValueError:
+            return None
+
+    def stop(self, t0=None, t1=None):
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -92,21 +103,24 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        parsed = []
         for r in self.rows:
-            if len(r) < 7:
+            if len(r) < 8:
                 continue
             try:
-                sm.append(float(r[0]))
-                mx.append(float(r[1]))
+                parsed.append((self._when(r[0]), float(r[1]), float(r[2]), r[4:8]))
             except ValueError:
                 continue
-            for name, val in zip(names, r[3:7]):
+        inside = [x for x in parsed if t0 is not None and x[0] is not None and t0 <= x[0] <= t1]
+        use = inside or parsed
+        sm, mx, reasons = [x[1] for x in use], [x[2] for x in use], set()
+        for x in use:
+            for name, val in zip(names, x[3]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "samples_inside_timed_region": len(inside), "reasons": sorted(reasons)}
 
 
 # ------------------------------------------------------------------------------------------------
@@ -366,17 +380,19 @@ def run_ours(args, rank, world):
     ev = {k: [] for k in SEGMENTS}
     t0, t1 = E(), E()
     torch.cuda.synchronize()
+    wall0 = time.time()
     t0.record()
     for _ in range(args.steps):
         step(ev)
     t1.record()
     torch.cuda.synchronize()
+    wall1 = time.time()
     if world > 1:
         dist.barrier()
     total_ms = t0.elapsed_time(t1)
     if rank == 0:
         time.sleep(0.2)
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop(wall0, wall1) if rank == 0 else None
     assert int(path.status.item()) == 0, "a device-side wait timed out"
     seg_ms = {k: [a.elapsed_time(b) / (gamma if k == "decode" else 1) for a, b in v] for k, v in ev.items()}
     mean = {k: sum(v) / len(v) for k, v in seg_ms.items()}          # per call (decode: per draft step)
