@@ -1059,8 +1059,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 // How a window of `rows` rows is cut: n_parts parts of q_per query tokens (at most 128 rows each).
 static void tc_parts(int rows, int group, int& n_parts, int& q_per) {
   const int n_q = rows / group;
-  n_parts = (rows + 127) / 128;
-  q_per = (n_q + n_parts - 1) / n_parts;
+  const int q_max = 128 / group;                       // whole query tokens that fit the 128 rows of a part
+  n_parts = (n_q + q_max - 1) / q_max;
+  q_per = (n_q + n_parts - 1) / n_parts;               // the parts are made as equal as the tokens allow
 }
 
 // One set of CTAs per part, every set as large as the SMs allow (and the tile count is worth).

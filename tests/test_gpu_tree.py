@@ -54,6 +54,8 @@ def _tree_case(L, Hq, Hkv, D, lens, n_nodes, *, paged, seed, chain=False):
                                               (64, 8, 26, 128),   # 208 rows: two parts of 13 nodes
                                               (32, 2, 32, 128),   # 512 rows, group 16: four parts of 8 nodes
                                               (24, 4, 30, 64),    # 180 rows, group 6, d = 64: 15 + 15 nodes
+                                              (40, 8, 51, 128),   # group 5 x 51 nodes = 255 rows: 25 tokens fill a part, so three parts of 17
+                                              (30, 2, 17, 64),    # group 15 x 17 nodes = 255 rows: three parts of 6, 6 and 5 tokens
                                               (64, 8, 60, 128),   # 60 nodes (a dynamic draft tree's size): 480 rows, four parts of 15
                                               (28, 4, 64, 128),   # 64 nodes, the mask's width, group 7: 448 rows, four parts of 16
                                               (8, 8, 41, 64)])    # 41 rows of one head each: bits above 32 in a single 64-row part
