@@ -28,7 +28,8 @@ def _seeds(n):
     return range(FIRST, FIRST + n * SCALE)
 
 
-GROUPS = [(4, 4), (8, 2), (28, 4), (40, 8), (64, 8), (16, 1), (12, 2)]     # (query heads, KV heads)
+GROUPS = [(4, 4), (8, 2), (28, 4), (40, 8), (64, 8), (16, 1), (12, 2),     # (query heads, KV heads)
+          (6, 3), (6, 2), (18, 2), (11, 1), (26, 2), (30, 2)]              # groups of 2, 3, 9, 11, 13, 15 heads
 
 
 def _lens(rng, batch, lo, hi, n_q):
