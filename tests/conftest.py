@@ -26,6 +26,18 @@ def pytest_collection_modifyitems(config, items):
             item.add_marker(skip)
 
 
+@pytest.fixture(scope="session", autouse=True)
+def _library_is_built():
+    """The CUDA library is built in-tree and kept out of the history: a fresh checkout compiles it
+    (nvcc, sm_100a; works without a GPU) before the first test needs it.  There is no other path to
+    fall back to, so a failed build fails the session here."""
+    from paper_2508_16201_b200 import specvlm
+    if not os.path.exists(specvlm.LIB_PATH):
+        from paper_2508_16201_b200 import build
+        build.build()
+    yield
+
+
 @pytest.fixture(autouse=True)
 def _poisoned_shared_memory(request):
     """Before every GPU test the SMs' shared memory is filled with NaN bit patterns: a kernel that
