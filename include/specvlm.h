@@ -408,6 +408,14 @@ int32_t specvlm_debug_wait_timeout(int32_t limit_ms, int32_t* d_status, int32_t*
  */
 void specvlm_debug_set_attn_splits(int32_t n_splits);
 
+/*
+ * Test hook, host only; the paper has no counterpart.  Reports how a verification window of n_q
+ * query tokens at `group` = n_q_heads / n_kv_heads heads per KV head is cut into the parts that run
+ * side by side in one launch: n_parts parts of q_per tokens (the last may be shorter), each of at
+ * most 128 rows.  n_parts, q_per: host int32 out.  Launches nothing.
+ */
+int32_t specvlm_debug_window_parts(int32_t n_q, int32_t group, int32_t* n_parts, int32_t* q_per);
+
 #ifdef __cplusplus
 }
 #endif

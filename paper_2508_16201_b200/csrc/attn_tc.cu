@@ -1239,3 +1239,14 @@ int32_t attn_tc_launch(const specvlm_kv_t* kv, const void* q, int32_t batch, int
 }
 
 }  // namespace specvlm
+
+// Host-only: how a verification window of n_q query tokens at `group` heads per KV head is cut into
+// parts (see tc_parts); lets a CPU test sweep the rule.
+extern "C" int32_t specvlm_debug_window_parts(int32_t n_q, int32_t group, int32_t* n_parts, int32_t* q_per) {
+  if (n_q < 1 || group < 1 || group > 16 || !n_parts || !q_per) return SPECVLM_ERR_INVALID_ARG;
+  int a, b;
+  specvlm::tc_parts(n_q * group, group, a, b);
+  *n_parts = a;
+  *q_per = b;
+  return SPECVLM_OK;
+}

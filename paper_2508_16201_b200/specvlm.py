@@ -55,7 +55,7 @@ EXPORTS = [
     "specvlm_append_kv", "specvlm_rollback_kv",
     "specvlm_verify_tree_workspace_bytes", "specvlm_verify_tree_attn", "specvlm_accept_tree",
     "specvlm_compact_tree_kv", "specvlm_debug_poison_shared_memory", "specvlm_debug_wait_timeout",
-    "specvlm_debug_set_attn_splits",
+    "specvlm_debug_set_attn_splits", "specvlm_debug_window_parts",
 ]
 
 
@@ -100,6 +100,8 @@ def lib():
         L.specvlm_debug_poison_shared_memory.argtypes = [c_void_p]
         L.specvlm_debug_wait_timeout.restype = c_int32
         L.specvlm_debug_wait_timeout.argtypes = [c_int32, c_void_p, c_void_p, c_void_p]
+        L.specvlm_debug_window_parts.restype = c_int32
+        L.specvlm_debug_window_parts.argtypes = [c_int32, c_int32, i32p, i32p]
         L.specvlm_debug_set_attn_splits.restype = None
         L.specvlm_debug_set_attn_splits.argtypes = [c_int32]
         L.specvlm_verify_tree_workspace_bytes.restype = c_size_t

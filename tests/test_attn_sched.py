@@ -13,3 +13,23 @@ def test_attention_work_partition(tmp_path):
                    check=True)
     out = subprocess.run([str(exe)], capture_output=True, text=True)
     assert out.returncode == 0 and out.stdout.strip() == "ok", out.stdout + out.stderr
+
+
+def test_wide_window_parts_hold_whole_tokens_and_fit_a_tile():
+    """A verification window of more than 128 rows is cut into parts of whole query tokens: for every
+    supported (heads per KV head, window tokens) a part has at most 128 rows, no part is empty, the
+    parts cover the window, and no cut is made when the window fits one part."""
+    import ctypes
+
+    from paper_2508_16201_b200 import specvlm
+    L = specvlm.lib()
+    for group in range(1, 17):
+        for n_q in range(1, 65):
+            n_parts, q_per = ctypes.c_int32(), ctypes.c_int32()
+            assert L.specvlm_debug_window_parts(n_q, group, ctypes.byref(n_parts), ctypes.byref(q_per)) == 0
+            n, q = n_parts.value, q_per.value
+            assert q * group <= 128, (group, n_q, n, q)
+            assert (n - 1) * q < n_q <= n * q, (group, n_q, n, q)
+            assert (n == 1) == (n_q * group <= 128 or n_q <= 128 // group)
+            assert n == -(-n_q // (128 // group))
+    assert L.specvlm_debug_window_parts(0, 8, None, None) == specvlm.ERR_INVALID_ARG
