@@ -65,7 +65,7 @@ class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs.  Every sample carries
     nvidia-smi's own timestamp; `stop(t0, t1)` keeps the samples taken between the two host wall-clock
     times that bracket the timed region (all samples if none fell inside: a region of a few tens of
-    milliseconds can slip between two samples)."""
+    milliseconds can slip between two samples; the samples within 50 ms of it are tried first)."""
     Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
@@ -113,6 +113,8 @@ class ClockSampler:
             except ValueError:
                 continue
         inside = [x for x in parsed if t0 is not None and x[0] is not None and t0 <= x[0] <= t1]
+        if not inside and t0 is not None:       # nearest neighbours of a region shorter than the sampling interval
+            inside = [x for x in parsed if x[0] is not None and t0 - 0.05 <= x[0] <= t1 + 0.05]
         use = inside or parsed
         sm, mx, reasons = [x[1] for x in use], [x[2] for x in use], set()
         for x in use:
