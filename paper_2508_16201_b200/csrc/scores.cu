@@ -65,12 +65,14 @@ __device__ __forceinline__ void load_key_tile(const CUtensorMap* tm_k, const Sco
   }
 }
 
-// Of every 8 pairs of logits in pass 1, this many take their exponential on the FMA pipe
-// (f2_exp2_poly) instead of the special-function unit, which both rating passes nearly saturate.
-// Measured: the polynomial costs about as many FMA-pipe cycles per value as the unit it relieves
-// (8), so it only pays where issue slots are left over: 2 of 8 in pass 1 (-3 %); none in pass 2,
-// whose four epilogue groups already keep the unit busy (every share made it slower there).
+// Some of the exponentials are taken on the FMA pipe (f2_exp2_poly) instead of the special-function
+// unit, which both rating passes nearly saturate.  The polynomial costs about as many FMA-pipe cycles
+// per value as the unit it relieves (8) plus issue slots, so only a small share pays, and the best
+// share is a measured one.  Pass 1: 2 of every 8 pairs (1 / 2 / 3 / 4 of 8: 1144 / 1106 / 1175 /
+// 1224 us).  Pass 2: 2 of the 16 pairs of a 32-column chunk, pairs 0 and 8 (0 / 1 / 2 / 3 / 4 / 6 / 8
+// of 16: 1208 / 1152 / 1141-1156 / 1158 / 1188 / 1245 / 1286 us for 80 layers of 6272 video tokens).
 constexpr int kPolyOf8Lse = 2;
+constexpr uint32_t kPolyMaskColsum = 0x0101u;          // bit i: pair i of a chunk takes the polynomial
 
 // ---------------------------------------------------------------------------------------------
 // Pass 2 on the 5th-generation tensor cores.  CTA = (block of 128 video keys, layer), looping over
@@ -300,8 +302,8 @@ scores_colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
                                      f2_pack(l4.x, l4.y));
           const uint64_t tb = f2_fma(f2_pack(__uint_as_float(v[2 * q + 2]), __uint_as_float(v[2 * q + 3])), sc2,
                                      f2_pack(l4.z, l4.w));
-          acc2[q & 3] = f2_add(acc2[q & 3], f2_exp2_sfu(ta));
-          acc2[(q + 1) & 3] = f2_add(acc2[(q + 1) & 3], f2_exp2_sfu(tb));
+          acc2[q & 3] = f2_add(acc2[q & 3], ((kPolyMaskColsum >> q) & 1) ? f2_exp2_poly(ta) : f2_exp2_sfu(ta));
+          acc2[(q + 1) & 3] = f2_add(acc2[(q + 1) & 3], ((kPolyMaskColsum >> (q + 1)) & 1) ? f2_exp2_poly(tb) : f2_exp2_sfu(tb));
         }
       }
     }
