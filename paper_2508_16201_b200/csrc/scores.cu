@@ -68,10 +68,14 @@ __device__ __forceinline__ void load_key_tile(const CUtensorMap* tm_k, const Sco
 // Some of the exponentials are taken on the FMA pipe (f2_exp2_poly) instead of the special-function
 // unit, which both rating passes nearly saturate.  The polynomial costs about as many FMA-pipe cycles
 // per value as the unit it relieves (8) plus issue slots, so only a small share pays, and the best
-// share is a measured one.  Pass 1: 2 of every 8 pairs (1 / 2 / 3 / 4 of 8: 1144 / 1106 / 1175 /
-// 1224 us).  Pass 2: 2 of the 16 pairs of a 32-column chunk, pairs 0 and 8 (0 / 1 / 2 / 3 / 4 / 6 / 8
-// of 16: 1208 / 1152 / 1141-1156 / 1158 / 1188 / 1245 / 1286 us for 80 layers of 6272 video tokens).
-constexpr int kPolyOf8Lse = 2;
+// share is a measured one (80 layers of 6272 video tokens, same box within a row of figures).
+// Pass 1: 3 of the 16 pairs of a 32-column chunk, pairs 3, 7 and 11 (2 / 4 / 6 / 8 of 16 in an
+// earlier form: 1144 / 1106 / 1175 / 1224 us; then 3 / 4 / 5 / 6 of 16: 1108 / 1143 / 1135 / 1173 us).
+// Which pairs matters to the compiler: under this kernel's 96-register cap pairs {3, 7, 11} compile
+// without a spill, {3, 11} and {2, 7, 12} with 400-850 bytes of spills and run 2-4 times slower.
+// Pass 2: 2 of the 16 pairs, pairs 0 and 8 (0 / 1 / 2 / 3 / 4 / 6 / 8 of 16: 1208 / 1152 / 1141-1156 /
+// 1158 / 1188 / 1245 / 1286 us).
+constexpr uint32_t kPolyMaskLse = 0x0888u;             // bit i: pair i of a chunk takes the polynomial
 constexpr uint32_t kPolyMaskColsum = 0x0101u;          // bit i: pair i of a chunk takes the polynomial
 
 // ---------------------------------------------------------------------------------------------
@@ -513,8 +517,8 @@ scores_lse_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
           const uint64_t t2 = f2_fma(f2_pack(__uint_as_float(v[2 * q]), __uint_as_float(v[2 * q + 1])), sc2, nmu2);
-          // kPolyOf8Lse of every 8 pairs take the polynomial, spread so both kinds interleave
-          const bool poly = ((q & 7) * kPolyOf8Lse) / 8 != (((q & 7) + 1) * kPolyOf8Lse) / 8;
+          // the pairs of kPolyMaskLse take the polynomial, spread so that both kinds interleave
+          const bool poly = (kPolyMaskLse >> q) & 1;
           ps[q & 1] = f2_add(ps[q & 1], poly ? f2_exp2_poly(t2) : f2_exp2_sfu(t2));
         }
         float s0, s1, s2, s3;

@@ -99,3 +99,22 @@ def test_missing_library_raises_and_package_is_oracle_free(monkeypatch, tmp_path
                 with open(os.path.join(root, f)) as fh:
                     src = fh.read()
                 assert not re.search(r"^\s*(import|from)\s+oracle|#include[^\n]*oracle|oracle[./]", src, re.M), f
+
+
+def test_rating_kernels_compile_without_heavy_spills():
+    """The rating kernels run under tight register caps (two CTAs of 320 threads, or 576 threads, per
+    SM) and which exponentials take the polynomial decides whether ptxas fits the loop in them: a
+    choice that spills a few hundred bytes runs two to four times slower.  The build keeps ptxas's
+    report; this reads the spill figures of the two kernels from it."""
+    from paper_2508_16201_b200 import build
+    build.build()
+    log = os.path.join(ROOT, "paper_2508_16201_b200", "_build", "scores.ptxas.log")
+    if not os.path.exists(log):
+        pytest.skip("no ptxas report (the objects were not compiled by this checkout)")
+    text = open(log).read()
+    seen = 0
+    for m in re.finditer(r"Function properties for (\S*scores_(?:lse|colsum)_tc_kernel\S*)\s*\n\s*(\d+) bytes stack frame, "
+                         r"(\d+) bytes spill stores, (\d+) bytes spill loads", text):
+        seen += 1
+        assert int(m.group(3)) <= 64 and int(m.group(4)) <= 64, m.group(0)
+    assert seen >= 4
