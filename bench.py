@@ -57,8 +57,8 @@ def measured_peaks():
 # summarised under profiles/; None where no capture of that launch exists.  Each capture ran a
 # subset of the layers (a many-pass capture has to stay small) and is scaled to the layers one
 # launch processes: traffic is proportional to the layers streamed.  verify: 216.0 MB for 8 of 80 layers; rating
-# passes: 156.5 MB and 153.2 MB for 10 of 80 layers; decode: 43.5 MB, captured whole.
-NCU_TRAFFIC_BYTES = {"verify": 216.0e6 * 10, "decode": 43.5e6, "scores_colsum": 153.2e6 * 8, "scores_lse": 156.5e6 * 8}
+# passes: 155.8 MB and 153.3 MB for 10 of 80 layers; decode: 43.5 MB, captured whole.
+NCU_TRAFFIC_BYTES = {"verify": 216.0e6 * 10, "decode": 43.5e6, "scores_colsum": 153.3e6 * 8, "scores_lse": 155.8e6 * 8}
 
 
 class ClockSampler:
