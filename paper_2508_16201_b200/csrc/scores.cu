@@ -74,7 +74,8 @@ __device__ __forceinline__ void load_key_tile(const CUtensorMap* tm_k, const Sco
 // Which pairs matters to the compiler: under this kernel's 96-register cap pairs {3, 7, 11} compile
 // without a spill, {3, 11} and {2, 7, 12} with 400-850 bytes of spills and run 2-4 times slower.
 // Pass 2: 2 of the 16 pairs, pairs 0 and 8 (0 / 1 / 2 / 3 / 4 / 6 / 8 of 16: 1208 / 1152 / 1141-1156 /
-// 1158 / 1188 / 1245 / 1286 us).
+// 1158 / 1188 / 1245 / 1286 us); the place matters here too: pairs {3, 11} or {5, 13} take 1254 us,
+// {7, 15} 1166, {0, 2} 1174, {0, 14} 1125 against 1133-1137 for {0, 8} on the same box.
 constexpr uint32_t kPolyMaskLse = 0x0888u;             // bit i: pair i of a chunk takes the polynomial
 constexpr uint32_t kPolyMaskColsum = 0x0101u;          // bit i: pair i of a chunk takes the polynomial
 
